@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the multi-Bulyan aggregation path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+A step is one whole aggregation GAR(f, [G_1..G_n]) (distances -> selection ->
+coordinate phase) of one synthetic workload resident in HBM.  One JSON line is
+printed by rank 0.  With N > 1 (torchrun) every rank aggregates its own replica
+of the workload on its own GPU: the path has no inter-GPU step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "multi_bulyan_aggregations_per_sec"
+UNIT = "aggregations/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
+
+    def __init__(self, index: int, period: float = 0.02):
+        self.index, self.period = index, period
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+
+    def _run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+                getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+            }
+            while not self._stop.is_set():
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                    for bit, name in names.items():
+                        if mask & bit:
+                            self.reasons.add(name)
+                except Exception:
+                    pass
+                time.sleep(self.period)
+        except Exception as exc:  # pragma: no cover
+            self.reasons.add(f"sampler_error:{type(exc).__name__}")
+
+    def __enter__(self):
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thr.join(timeout=2)
+
+    def summary(self):
+        s = sorted(self.samples)
+        med = s[len(s) // 2] if s else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def oracle_sample_time(cfg: int, d_sample: int):
+    """Times the CPU oracle, as it stands, on a d_sample-column sample of the workload."""
+    import numpy as np
+    from oracle import gar_oracle as O
+    from paper_1905_04374_b200 import workloads
+    wl = workloads.WORKLOADS[cfg]
+    G, _ = workloads.make_gradients(cfg, d=d_sample, device="cpu")
+    Gh = G.numpy()
+    t0 = time.perf_counter()
+    out, _, _ = O.multi_bulyan(Gh, wl.f)
+    dt = time.perf_counter() - t0
+    assert np.all(np.isfinite(out))
+    return dt, wl
+
+
+def cpu_baseline(cfg: int, d_sample: int):
+    dt, wl = oracle_sample_time(cfg, d_sample)
+    per_full = dt * (wl.d / d_sample)
+    return {"value": 1.0 / per_full, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"numpy fp64 oracle on the first {d_sample} of {wl.d} coordinates of {wl.name} "
+                      f"({dt:.2f} s), scaled by d/sample", "seconds_sample": dt}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1905_04374_b200 import workloads
+    wl = workloads.WORKLOADS[args.config]
+    d_sample = args.ref_sample
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt, _ = oracle_sample_time(args.config, d_sample)
+        if i >= args.warmup:
+            times.append(dt)
+    per_step_full = (sum(times) / len(times)) * (wl.d / d_sample)
+    value = 1.0 / per_step_full
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step_full * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "n": wl.n, "f": wl.f, "d": wl.d, "rule": "multi_bulyan"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"each step: numpy fp64 oracle on the first {d_sample} of {wl.d} coordinates, "
+                                   f"scaled by d/sample"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def event_time_ms(fn, reps, stream):
+    import torch
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    start.record(stream)
+    for _ in range(reps):
+        fn()
+    stop.record(stream)
+    torch.cuda.synchronize()
+    return start.elapsed_time(stop) / reps
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1905_04374_b200 as pkg
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = pkg.workloads.WORKLOADS[args.config]
+    n, f, d = wl.n, wl.f, wl.d
+    theta_a = pkg.gar_theta("multi_bulyan", n, f)
+    theta_b = pkg.gar_theta("bulyan", n, f)
+    G, _ = pkg.workloads.make_gradients(args.config, device=dev)
+    out = torch.empty(d, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pkg.gar_aggregate("multi_bulyan", G, f, out=out)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(physical_gpu_index(local)) as clocks:
+        torch.cuda.synchronize()
+        start.record(stream)
+        for _ in range(args.steps):
+            step()
+        stop.record(stream)
+        torch.cuda.synchronize()
+    elapsed_ms = start.elapsed_time(stop)
+    if world > 1:
+        t = torch.tensor([elapsed_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.barrier()
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * args.steps / (elapsed_ms * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-kernel durations, measured live with CUDA events on the launch stream
+    reps = max(5, min(50, args.steps))
+    dmat = torch.empty(n, n, dtype=torch.float64, device=dev)
+    sel = pkg.new_selection(dev)
+    pkg.gar_pairwise_distances(G, dist=dmat)
+    pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel)
+    k1_ms = event_time_ms(lambda: pkg.gar_pairwise_distances(G, dist=dmat), reps, stream)
+    k2_ms = event_time_ms(lambda: pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel), reps, stream)
+    k3_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, sel, theta_a, 1, out=out), reps, stream)
+    selh = pkg.read_selection(sel)
+    rows_k3 = bin(selh.sets[0]).count("1") if selh.nested else None
+    peak, peak_kind = measured_hbm_peak()
+    k1_bytes = 4.0 * n * d
+    k3_bytes = 4.0 * d * ((rows_k3 if rows_k3 else theta_a) + 1)
+    kernels = {
+        "k1_distances": {"ms": k1_ms, "algorithmic_bytes": k1_bytes, "gbs": k1_bytes / (k1_ms * 1e-3) / 1e9},
+        "k2_select": {"ms": k2_ms},
+        "k3_coordinate": {"ms": k3_ms, "algorithmic_bytes": k3_bytes, "gbs": k3_bytes / (k3_ms * 1e-3) / 1e9,
+                          "rows_read": rows_k3},
+    }
+    dom = "k1_distances" if k1_ms >= k3_ms else "k3_coordinate"
+    achieved = kernels[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None}
+    # whole-path effective bandwidth against the minimum traffic (n + theta + 1) * 4 d
+    path_bytes_northstar = 4.0 * d * (n + theta_b + 1)
+    path_bytes_own = 4.0 * d * (n + (rows_k3 if rows_k3 else theta_a) + 1)
+    path = {
+        "bytes_min_n_plus_theta_plus_1": path_bytes_northstar,
+        "bytes_min_this_rule": path_bytes_own,
+        "effective_gbs": path_bytes_northstar / (ms_per_step * 1e-3) / 1e9,
+        "effective_gbs_this_rule": path_bytes_own / (ms_per_step * 1e-3) / 1e9,
+    }
+    path["frac_of_nominal_8TBs"] = path["effective_gbs"] / NOMINAL_HBM_GBS
+    path["frac_of_measured_peak"] = path["effective_gbs"] / peak
+
+    # ---- end to end through the host entry point (pinned host buffers, copies timed)
+    e2e = None
+    if not args.no_e2e:
+        host = torch.empty(n, d, dtype=torch.float32, pin_memory=True)
+        host.copy_(G)
+        hout = torch.empty(d, dtype=torch.float32, pin_memory=True)
+        e2e_steps = max(2, min(args.steps, args.e2e_steps))
+        pkg.gar_aggregate_host("multi_bulyan", host, f, out=hout)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            pkg.gar_aggregate_host("multi_bulyan", host, f, out=hout)
+        t1 = time.perf_counter()
+        e2e = {"value": e2e_steps / (t1 - t0), "unit": UNIT, "h2d_bytes_per_step": int(4 * n * d),
+               "d2h_bytes_per_step": int(4 * d), "steps": e2e_steps,
+               "api": "gar_aggregate_host (pinned host buffers, synchronous)"}
+        del host, hout
+
+    cpu = None if args.no_cpu_baseline else cpu_baseline(args.config, args.cpu_sample)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "n": n, "f": f, "d": d, "rule": "multi_bulyan", "theta": theta_a,
+                   "beta": pkg.gar_beta("multi_bulyan", n, f), "parallelism": f"replicas x{world}",
+                   "l2": "input (%.2f GB) larger than L2; no flush" % (4e-9 * n * d) if 4 * n * d > 2.6e8
+                   else "input fits L2; not flushed between steps"},
+        "roofline": roofline, "path": path, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": 3 * args.steps, "clocks": clocks.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3, help="workload 1..5 (default 3: n=39, f=9, d=25.6M)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="columns of the CPU-baseline sample")
+    ap.add_argument("--ref-sample", type=int, default=1 << 18, help="columns per step of --impl reference")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,200 @@
+/*
+ * gar.h -- C ABI of the gradient aggregation rule (GAR) library for NVIDIA B200
+ * (sm_100a): averaging, coordinate-wise median, Krum, multi-Krum, Bulyan and
+ * multi-Bulyan of n worker gradients of dimension d, 1 <= n <= 64, fp32.
+ *
+ * The operations follow "Fast and Robust Distributed Learning in High
+ * Dimension" (the multi-Bulyan paper): Eq. 4 and Algorithm 1 (functions
+ * multi-Krum, multi-Bulyan and GAR), the one-sentence Bulyan of Section 2.2,
+ * the averaging rule of the Introduction and the Median rule of Section 5.
+ *
+ * General conventions
+ *  - "dev" pointers are device pointers of the current CUDA device, "host"
+ *    pointers are host pointers.  All buffers are owned by the caller.
+ *  - Gradients are row-major: worker i occupies grads[i*ld .. i*ld + d).
+ *    Any alignment and any ld >= d are accepted; the vectorised kernels are
+ *    used when grads and out are 16-byte aligned and ld is a multiple of 4.
+ *  - Every call is asynchronous on `stream` (a cudaStream_t passed as void*;
+ *    NULL is the legacy default stream) unless stated otherwise.  There is no
+ *    host synchronisation and no host round trip between the kernels.
+ *  - Argument and precondition errors are returned before anything is
+ *    launched; launch failures are returned as GAR_ERR_CUDA.  No exceptions
+ *    cross this boundary.  There is no CPU fallback.
+ *  - Results are deterministic: the same input gives bit-identical output.
+ *  - Ties (equal scores, equal distances to the median) are broken towards the
+ *    lowest worker index, in the coordinate phase towards the earliest round.
+ *    The median of an even count is the lower of the two middle values.
+ *    A non-finite distance is treated as +infinity.
+ */
+#ifndef GAR_H_
+#define GAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GAR_MAX_N 64
+#define GAR_VERSION 100
+
+typedef enum {
+    GAR_AVERAGE      = 0, /* (1/n) sum_i G_i                       (Introduction)            */
+    GAR_MEDIAN       = 1, /* coordinate-wise median                (Section 5, "Median")     */
+    GAR_KRUM         = 2, /* smallest-score gradient               (Eq. 4 with m = 1)        */
+    GAR_MULTI_KRUM   = 3, /* average of the m best-scored          (Eq. 4; Alg. 1 multi-Krum)*/
+    GAR_BULYAN       = 4, /* theta = n-2f Krum winners, median, beta closest (Section 2.2;
+                             iteration count of the proof of Theorem 2 (i))                  */
+    GAR_MULTI_BULYAN = 5  /* Algorithm 1: theta = n-2f-2 rounds, pre-aggregated G^agr,
+                             median of G^ext, beta = theta-2f closest entries of G^agr       */
+} gar_rule_t;
+
+typedef enum {
+    GAR_OK               = 0,
+    GAR_ERR_INVALID_ARG  = 1, /* null pointer, n < 1, f < 0, d < 1, ld < d, unknown rule, bad option */
+    GAR_ERR_PRECONDITION = 2, /* n < 2f+3 (Krum family) or n < 4f+3 (Bulyan family), Section 2.2    */
+    GAR_ERR_UNSUPPORTED  = 3, /* n > GAR_MAX_N                                                       */
+    GAR_ERR_WORKSPACE    = 4, /* workspace missing, misaligned (256 B) or too small                  */
+    GAR_ERR_CUDA         = 5, /* a CUDA runtime call or a launch failed                              */
+    GAR_ERR_TIMEOUT      = 6  /* reserved: a bounded device-side wait gave up                        */
+} gar_status_t;
+
+/*
+ * Result of the scoring / selection step (Eq. 4; Algorithm 1, multi-Krum and
+ * the extraction loop of multi-Bulyan), device resident, consumed by the
+ * coordinate phase.  Rounds are numbered 0..theta-1 in extraction order.
+ *   winners[r]  index of the smallest-score gradient of round r (G^ext[r])
+ *   sets[r]     bit i set <=> gradient i is averaged into G^agr[r]
+ *   m[r]        number of bits in sets[r]
+ *   scores[r][i] score of gradient i in round r (+inf if already extracted)
+ *   gap_winner[r], gap_set[r]  relative gaps (s2-s1)/s2 between the two
+ *               smallest scores and between the m-th and (m+1)-th score
+ * The fields from `nested` on are the summation schedule the coordinate kernel
+ * executes (private layout, documented in the design notes).
+ */
+typedef struct {
+    int32_t  n, f, rule, theta, beta;
+    int32_t  preagg;              /* 1: G^agr[r] = mean over sets[r]; 0: G^agr = G^ext */
+    int32_t  median_of_agr;       /* 1: median taken over G^agr instead of G^ext       */
+    int32_t  status;              /* gar_status_t written by the selection kernel      */
+    int32_t  winners[GAR_MAX_N];
+    int32_t  m[GAR_MAX_N];
+    uint64_t sets[GAR_MAX_N];
+    double   gap_winner[GAR_MAX_N];
+    double   gap_set[GAR_MAX_N];
+    /* schedule */
+    int32_t  nested;              /* 1: sets[r] = sets[r+1] + {winners[r]} for every r  */
+    int32_t  base_count;          /* rows summed for the last round                     */
+    int32_t  base_rows[GAR_MAX_N];/* winners[theta-1] first, then ascending             */
+    int32_t  seg_start[GAR_MAX_N + 1]; /* general schedule: rows added at slot s are
+                                     prog_rows[seg_start[s] .. seg_start[s+1])           */
+    uint8_t  restart[GAR_MAX_N];  /* running sum restarts from zero at slot s           */
+    uint8_t  prog_rows[GAR_MAX_N * GAR_MAX_N];
+    double   scores[GAR_MAX_N][GAR_MAX_N];
+} gar_selection_t;
+
+/* Extended call.  Zero-initialise, then set what you need. */
+typedef struct {
+    int32_t       rule;           /* gar_rule_t */
+    int32_t       n, f;
+    int64_t       d;
+    int64_t       ld;             /* row stride in elements; 0 means d */
+    const float*  grads;          /* dev, n rows */
+    float*        out;            /* dev, d values; must not overlap grads */
+    void*         stream;         /* cudaStream_t */
+    void*         workspace;      /* dev, 256-byte aligned, >= gar_workspace_bytes(), its first 256
+                                     bytes zeroed once before the first use (the kernels restore
+                                     them); NULL: the library's cached per-device workspace
+                                     (allocated on first use) */
+    size_t        workspace_bytes;
+    int32_t       m;              /* multi-Krum only: number of averaged gradients, 1..n-f-2; 0 = n-f-2
+                                     (Section 3 allows any m <= n-f-2) */
+    int32_t       theta;          /* multi-Bulyan only: number of rounds, 2f+1..n-2f-2; 0 = n-2f-2 */
+    int32_t       median_of_agr;  /* multi-Bulyan only: 1 = median over G^agr (reading of Section 5.2's
+                                     "median ... over ... pre-aggregated gradients"); 0 = Algorithm 1 */
+    int32_t       reserved;
+    double*       dist_out;       /* optional dev [n*n]: the distance matrix */
+    gar_selection_t* selection_out; /* optional dev: the selection result */
+} gar_params_t;
+
+/* Library version (GAR_VERSION).  The paper has no counterpart. */
+int gar_version(void);
+
+/* Static description of a status code. */
+const char* gar_status_string(int status);
+
+/* theta (number of extraction rounds) and beta (values kept per coordinate) of a
+ * rule: multi-Bulyan n-2f-2 and theta-2f (Algorithm 1); Bulyan n-2f and theta-2f
+ * (Section 2.2 / proof of Theorem 2); Krum, multi-Krum, averaging 1 and 1;
+ * median n and 1.  Returns -1 if the rule's precondition fails. */
+int gar_theta(int rule, int n, int f);
+int gar_beta(int rule, int n, int f);
+
+/* Bytes of device workspace a call needs (host, pure).  0 on invalid arguments. */
+size_t gar_workspace_bytes(int rule, int n, int f, int64_t d);
+
+/*
+ * GAR(f, [G_1..G_n]) of Algorithm 1 for the chosen rule.
+ *   grads dev [n rows, stride d], out dev [d].
+ * Uses a per-device workspace that the library allocates on the first call for
+ * that device and keeps until gar_shutdown().  Not re-entrant across streams
+ * for the same device (the cached workspace is shared); use gar_aggregate_ex
+ * with distinct workspaces for concurrent calls.
+ */
+int gar_aggregate(int rule, const float* grads, int n, int f, int64_t d, float* out, void* stream);
+
+/* Same with explicit row stride, caller workspace, options and optional outputs. */
+int gar_aggregate_ex(const gar_params_t* params);
+
+/*
+ * The same rule on HOST buffers: grads host [n rows, stride d], out host [d].
+ * Copies the rows to a device buffer the library caches (grown on demand, kept
+ * until gar_shutdown), runs the three kernels and copies the result back, all
+ * on one internal stream.  Synchronous: returns when `out` is complete.
+ * Pinned (page-locked) host buffers are copied at full PCIe speed; pageable
+ * ones work but are slower.
+ */
+int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, float* out);
+
+/*
+ * Step 1 alone: D_ij = ||G_i - G_j||^2 (Algorithm 1, multi-Krum, neighbour
+ * distances), all pairs, one streaming pass.  dist dev [n*n] fp64, symmetric,
+ * zero diagonal.  workspace as in gar_params_t (NULL = cached).
+ */
+int gar_pairwise_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Step 2 alone: scoring and iterative selection from a distance matrix
+ * (Eq. 4; Algorithm 1 multi-Krum and the loop of multi-Bulyan).
+ *   dist dev [n*n] fp64; sel dev, written.  m, theta as in gar_params_t (0 = default).
+ */
+int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int median_of_agr,
+               gar_selection_t* sel, void* stream);
+
+/*
+ * Builds the coordinate kernel's schedule for GIVEN winners and sets (e.g. the
+ * oracle's), without scoring: sel dev with n, f, rule, theta, beta, preagg,
+ * median_of_agr, winners, sets filled by the caller; m, nested, base_*,
+ * seg_start, restart, prog_rows are written.  The paper has no counterpart
+ * (test and diagnostic aid).
+ */
+int gar_schedule_from_tables(gar_selection_t* sel, void* stream);
+
+/*
+ * Step 3 alone: the coordinate phase (Algorithm 1, multi-Bulyan: Median of
+ * G^ext, the beta entries of G^agr closest to it, their average) for a
+ * selection already on the device.  theta and preagg repeat sel->theta and
+ * sel->preagg (the host needs them to pick the kernel).  out dev [d].
+ */
+int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld,
+                         const gar_selection_t* sel, int theta, int preagg, float* out, void* stream);
+
+/* Frees every cached device buffer of every device.  Synchronises. */
+void gar_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GAR_H_ */

@@ -1,0 +1,266 @@
+"""Thin ctypes binding of libgar.so: argument marshalling only.
+
+Every function has the name and the argument order of its C entry point in
+include/gar.h; tensors are passed as device (or host) pointers, the current
+torch CUDA stream is used when no stream is given.  Nothing is computed here
+and there is no fallback: if the library is missing, loading fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+GAR_MAX_N = 64
+RULES = {"average": 0, "median": 1, "krum": 2, "multi_krum": 3, "bulyan": 4, "multi_bulyan": 5}
+GAR_OK = 0
+STATUS_NAMES = {0: "GAR_OK", 1: "GAR_ERR_INVALID_ARG", 2: "GAR_ERR_PRECONDITION", 3: "GAR_ERR_UNSUPPORTED",
+                4: "GAR_ERR_WORKSPACE", 5: "GAR_ERR_CUDA", 6: "GAR_ERR_TIMEOUT"}
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libgar.so")
+_lib = None
+
+
+class GarSelection(C.Structure):
+    """Mirror of gar_selection_t."""
+    _fields_ = [
+        ("n", C.c_int32), ("f", C.c_int32), ("rule", C.c_int32), ("theta", C.c_int32), ("beta", C.c_int32),
+        ("preagg", C.c_int32), ("median_of_agr", C.c_int32), ("status", C.c_int32),
+        ("winners", C.c_int32 * GAR_MAX_N),
+        ("m", C.c_int32 * GAR_MAX_N),
+        ("sets", C.c_uint64 * GAR_MAX_N),
+        ("gap_winner", C.c_double * GAR_MAX_N),
+        ("gap_set", C.c_double * GAR_MAX_N),
+        ("nested", C.c_int32), ("base_count", C.c_int32),
+        ("base_rows", C.c_int32 * GAR_MAX_N),
+        ("seg_start", C.c_int32 * (GAR_MAX_N + 1)),
+        ("restart", C.c_uint8 * GAR_MAX_N),
+        ("prog_rows", C.c_uint8 * (GAR_MAX_N * GAR_MAX_N)),
+        ("scores", (C.c_double * GAR_MAX_N) * GAR_MAX_N),
+    ]
+
+
+class GarParams(C.Structure):
+    """Mirror of gar_params_t."""
+    _fields_ = [
+        ("rule", C.c_int32), ("n", C.c_int32), ("f", C.c_int32),
+        ("d", C.c_int64), ("ld", C.c_int64),
+        ("grads", C.c_void_p), ("out", C.c_void_p), ("stream", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("m", C.c_int32), ("theta", C.c_int32), ("median_of_agr", C.c_int32), ("reserved", C.c_int32),
+        ("dist_out", C.c_void_p), ("selection_out", C.c_void_p),
+    ]
+
+
+class GarError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().gar_status_string(status).decode()
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({msg})")
+
+
+def lib():
+    """The loaded library.  Raises if libgar.so has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with "
+                               "`python -m paper_1905_04374_b200.build` (needs nvcc); there is no fallback")
+        L = C.CDLL(_LIB_PATH)
+        L.gar_version.restype = C.c_int
+        L.gar_status_string.restype = C.c_char_p
+        L.gar_status_string.argtypes = [C.c_int]
+        L.gar_theta.argtypes = [C.c_int, C.c_int, C.c_int]
+        L.gar_beta.argtypes = [C.c_int, C.c_int, C.c_int]
+        L.gar_workspace_bytes.restype = C.c_size_t
+        L.gar_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int64]
+        L.gar_aggregate.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_void_p, C.c_void_p]
+        L.gar_aggregate_ex.argtypes = [C.POINTER(GarParams)]
+        L.gar_aggregate_host.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_void_p]
+        L.gar_pairwise_distances.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                             C.c_size_t, C.c_void_p]
+        L.gar_select.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                 C.c_void_p]
+        L.gar_schedule_from_tables.argtypes = [C.c_void_p, C.c_void_p]
+        L.gar_coordinate_phase.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_int,
+                                           C.c_void_p, C.c_void_p]
+        L.gar_shutdown.restype = None
+        _lib = L
+    return _lib
+
+
+def _rule(rule) -> int:
+    return RULES[rule] if isinstance(rule, str) else int(rule)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(status: int, where: str):
+    if status != GAR_OK:
+        raise GarError(status, where)
+
+
+def _dev_f32(t: torch.Tensor, name: str):
+    if not (t.is_cuda and t.dtype == torch.float32):
+        raise TypeError(f"{name} must be a CUDA float32 tensor")
+    return t
+
+
+def gar_version() -> int:
+    return lib().gar_version()
+
+
+def gar_status_string(status: int) -> str:
+    return lib().gar_status_string(status).decode()
+
+
+def gar_theta(rule, n: int, f: int) -> int:
+    return lib().gar_theta(_rule(rule), n, f)
+
+
+def gar_beta(rule, n: int, f: int) -> int:
+    return lib().gar_beta(_rule(rule), n, f)
+
+
+def gar_workspace_bytes(rule, n: int, f: int, d: int) -> int:
+    return lib().gar_workspace_bytes(_rule(rule), n, f, d)
+
+
+def _rows(grads: torch.Tensor):
+    """(n, d, ld) of a 2-D tensor whose rows are contiguous."""
+    if grads.dim() != 2 or grads.stride(1) != 1:
+        raise ValueError("grads must be 2-D with unit column stride")
+    n, d = grads.shape
+    ld = grads.stride(0) if n > 1 else d
+    return n, d, ld
+
+
+def gar_aggregate(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """gar_aggregate: grads CUDA fp32 [n, d] contiguous, returns out [d]."""
+    _dev_f32(grads, "grads")
+    n, d, ld = _rows(grads)
+    if ld != d:
+        raise ValueError("gar_aggregate needs contiguous rows; use gar_aggregate_ex for a row stride")
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=grads.device)
+    _dev_f32(out, "out")
+    with torch.cuda.device(grads.device):
+        st = lib().gar_aggregate(_rule(rule), grads.data_ptr(), n, f, d, out.data_ptr(), _stream(stream))
+    _check(st, "gar_aggregate")
+    return out
+
+
+def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = None, stream=None,
+                     workspace: torch.Tensor | None = None, m: int = 0, theta: int = 0, median_of_agr: int = 0,
+                     dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None):
+    """gar_aggregate_ex: row stride taken from the tensor; optional workspace
+    (uint8 CUDA tensor), options and outputs (dist_out float64 [n, n];
+    selection_out uint8 CUDA tensor of sizeof(gar_selection_t))."""
+    _dev_f32(grads, "grads")
+    n, d, ld = _rows(grads)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=grads.device)
+    p = GarParams()
+    p.rule, p.n, p.f, p.d, p.ld = _rule(rule), n, f, d, ld
+    p.grads, p.out, p.stream = grads.data_ptr(), out.data_ptr(), _stream(stream)
+    if workspace is not None:
+        p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    p.m, p.theta, p.median_of_agr = m, theta, median_of_agr
+    if dist_out is not None:
+        p.dist_out = dist_out.data_ptr()
+    if selection_out is not None:
+        p.selection_out = selection_out.data_ptr()
+    with torch.cuda.device(grads.device):
+        st = lib().gar_aggregate_ex(C.byref(p))
+    _check(st, "gar_aggregate_ex")
+    return out
+
+
+def gar_aggregate_host(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = None) -> torch.Tensor:
+    """gar_aggregate_host: grads and out are HOST fp32 tensors (pinned for speed)."""
+    if grads.is_cuda or grads.dtype != torch.float32 or not grads.is_contiguous():
+        raise TypeError("grads must be a contiguous host float32 tensor")
+    n, d = grads.shape
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, pin_memory=grads.is_pinned())
+    st = lib().gar_aggregate_host(_rule(rule), grads.data_ptr(), n, f, d, out.data_ptr())
+    _check(st, "gar_aggregate_host")
+    return out
+
+
+def gar_pairwise_distances(grads: torch.Tensor, dist: torch.Tensor | None = None, workspace=None,
+                           stream=None) -> torch.Tensor:
+    """gar_pairwise_distances: returns dist float64 [n, n] on the device."""
+    _dev_f32(grads, "grads")
+    n, d, ld = _rows(grads)
+    if dist is None:
+        dist = torch.empty(n, n, dtype=torch.float64, device=grads.device)
+    wp, wb = (workspace.data_ptr(), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
+    with torch.cuda.device(grads.device):
+        st = lib().gar_pairwise_distances(grads.data_ptr(), n, d, ld, dist.data_ptr(), wp, wb, _stream(stream))
+    _check(st, "gar_pairwise_distances")
+    return dist
+
+
+def new_selection(device) -> torch.Tensor:
+    """Device buffer for one gar_selection_t."""
+    return torch.zeros(C.sizeof(GarSelection), dtype=torch.uint8, device=device)
+
+
+def read_selection(sel: torch.Tensor) -> GarSelection:
+    """Copy a device gar_selection_t to the host."""
+    raw = sel.cpu().numpy().tobytes()
+    return GarSelection.from_buffer_copy(raw)
+
+
+def write_selection(host: GarSelection, device) -> torch.Tensor:
+    """Upload a host gar_selection_t."""
+    import numpy as np
+    arr = np.frombuffer(bytes(host), dtype=np.uint8).copy()
+    return torch.from_numpy(arr).to(device)
+
+
+def gar_select(rule, dist: torch.Tensor | None, n: int, f: int, m: int = 0, theta: int = 0, median_of_agr: int = 0,
+               sel: torch.Tensor | None = None, stream=None, device=None) -> torch.Tensor:
+    """gar_select: dist CUDA float64 [n, n]; returns the device gar_selection_t buffer."""
+    device = dist.device if dist is not None else (device or "cuda")
+    if sel is None:
+        sel = new_selection(device)
+    dp = None
+    if dist is not None:
+        if not (dist.is_cuda and dist.dtype == torch.float64 and dist.is_contiguous()):
+            raise TypeError("dist must be a contiguous CUDA float64 tensor")
+        dp = dist.data_ptr()
+    with torch.cuda.device(sel.device):
+        st = lib().gar_select(_rule(rule), dp, n, f, m, theta, median_of_agr, sel.data_ptr(), _stream(stream))
+    _check(st, "gar_select")
+    return sel
+
+
+def gar_schedule_from_tables(sel: torch.Tensor, stream=None) -> torch.Tensor:
+    with torch.cuda.device(sel.device):
+        st = lib().gar_schedule_from_tables(sel.data_ptr(), _stream(stream))
+    _check(st, "gar_schedule_from_tables")
+    return sel
+
+
+def gar_coordinate_phase(grads: torch.Tensor, sel: torch.Tensor, theta: int, preagg: int,
+                         out: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    _dev_f32(grads, "grads")
+    n, d, ld = _rows(grads)
+    if out is None:
+        out = torch.empty(d, dtype=torch.float32, device=grads.device)
+    with torch.cuda.device(grads.device):
+        st = lib().gar_coordinate_phase(grads.data_ptr(), n, d, ld, sel.data_ptr(), theta, preagg, out.data_ptr(),
+                                        _stream(stream))
+    _check(st, "gar_coordinate_phase")
+    return out
+
+
+def gar_shutdown() -> None:
+    lib().gar_shutdown()

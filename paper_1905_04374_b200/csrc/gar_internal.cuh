@@ -1,0 +1,54 @@
+// Internal declarations shared by the translation units of libgar.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gar.h"
+
+namespace gar {
+
+// ---- workspace layout (device) -------------------------------------------
+// [0, 256)                control block (ticket counter of the distance kernel)
+// [256, +partials)        per-CTA partial distance sums, fp64
+// [.., +n*n doubles)      distance matrix
+// [.., +sizeof(selection)) selection result / coordinate-phase schedule
+constexpr int    kMaxCtasK1      = 592;                 // upper bound on the distance kernel's grid
+constexpr int    kMaxTiles       = 36;                  // 8x8 row-block pairs at n = 64
+constexpr int    kPairSlots      = kMaxTiles * 64;      // fp64 slots per CTA partial
+constexpr size_t kCtrlBytes      = 256;
+constexpr size_t kPartialBytes   = size_t(kMaxCtasK1) * kPairSlots * sizeof(double);
+constexpr size_t kDistBytes      = size_t(GAR_MAX_N) * GAR_MAX_N * sizeof(double);
+
+constexpr size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+constexpr size_t kOffPartials  = kCtrlBytes;
+constexpr size_t kOffDist      = kOffPartials + align256(kPartialBytes);
+constexpr size_t kOffSelection = kOffDist + align256(kDistBytes);
+constexpr size_t kWorkspaceBytes = kOffSelection + align256(sizeof(gar_selection_t));
+
+struct Workspace {
+    char* base;
+    unsigned int*    ticket()    const { return reinterpret_cast<unsigned int*>(base); }
+    double*          partials()  const { return reinterpret_cast<double*>(base + kOffPartials); }
+    double*          dist()      const { return reinterpret_cast<double*>(base + kOffDist); }
+    gar_selection_t* selection() const { return reinterpret_cast<gar_selection_t*>(base + kOffSelection); }
+};
+
+// ---- kernel launchers (one per translation unit) --------------------------
+// Pairwise squared distances of n rows over columns [0, d); result in dist[n*n].
+// `accumulate_only`/`finalize` allow the host path to feed column slabs:
+// slab calls add into the workspace partials, the last one finalises.
+cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
+                             const Workspace& ws, int sm_count, cudaStream_t stream);
+
+// Scoring + iterative selection (and schedule construction) into *sel.
+cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,
+                          int median_of_agr, gar_selection_t* sel, cudaStream_t stream);
+cudaError_t launch_schedule_only(gar_selection_t* sel, cudaStream_t stream);
+
+// Coordinate phase.
+cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
+                              const gar_selection_t* sel, int theta, int preagg, float* out,
+                              int sm_count, cudaStream_t stream);
+
+}  // namespace gar
