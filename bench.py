@@ -219,7 +219,7 @@ def run_ours(args):
     k2_ms = event_time_ms(lambda: pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel), reps, stream)
     k3_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, sel, theta_a, 1, out=out), reps, stream)
     selh = pkg.read_selection(sel)
-    rows_k3 = bin(selh.sets[0]).count("1") if selh.nested else None
+    rows_k3 = int(selh.nu)
     peak, peak_kind = measured_hbm_peak()
     k1_bytes = 4.0 * n * d
     k3_bytes = 4.0 * d * ((rows_k3 if rows_k3 else theta_a) + 1)

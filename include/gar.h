@@ -70,9 +70,29 @@ typedef enum {
  *   scores[r][i] score of gradient i in round r (+inf if already extracted)
  *   gap_winner[r], gap_set[r]  relative gaps (s2-s1)/s2 between the two
  *               smallest scores and between the m-th and (m+1)-th score
- * The fields from `nested` on are the summation schedule the coordinate kernel
- * executes (private layout, documented in the design notes).
+ * The fields from `nu` on are the summation plan the coordinate kernel executes
+ * for the pre-aggregating rules.  Rounds are visited last-to-first ("slots":
+ * slot s = round theta-1-s); the sets lose about one gradient per round, so in
+ * slot order they mostly grow.  With T_s the sum over slot s's set:
+ *     T_s = sum(base rows) + sum(winners of the slots t <= s in chain_mask) + C_s
+ *   base_rows[0..nbase)  gradients present in every slot (minus a chained slot-0 winner)
+ *   chain_mask  bit s: the winner of slot s is in every set from slot s on; it is
+ *               added to the running sum at slot s (the winner's value is needed
+ *               there anyway)
+ *   loose_rows[0..nloose)  every other gradient that occurs in some set
+ *   C_s         sum over the loose gradients of slot s, built by a small plan:
+ *               slot_src[s] says where it starts (GAR_SRC_ZERO, GAR_SRC_CONT =
+ *               continue from slot s-1, or the index of a saved sum),
+ *               slot_nadd[s] loose gradients are added (positions in loose_rows,
+ *               consecutive in add_pos[], slot 0 first), slot_save[s] is
+ *               GAR_SAVE_NONE or the index under which C_s is kept
+ *   corr_mask   bit s: slot s has anything to do for C_s
+ * Sums are only ever added to, never subtracted from.
  */
+#define GAR_SRC_ZERO  255
+#define GAR_SRC_CONT  254
+#define GAR_SAVE_NONE 255
+#define GAR_MAX_SAVED 8
 typedef struct {
     int32_t  n, f, rule, theta, beta;
     int32_t  preagg;              /* 1: G^agr[r] = mean over sets[r]; 0: G^agr = G^ext */
@@ -83,14 +103,17 @@ typedef struct {
     uint64_t sets[GAR_MAX_N];
     double   gap_winner[GAR_MAX_N];
     double   gap_set[GAR_MAX_N];
-    /* schedule */
-    int32_t  nested;              /* 1: sets[r] = sets[r+1] + {winners[r]} for every r  */
-    int32_t  base_count;          /* rows summed for the last round                     */
-    int32_t  base_rows[GAR_MAX_N];/* winners[theta-1] first, then ascending             */
-    int32_t  seg_start[GAR_MAX_N + 1]; /* general schedule: rows added at slot s are
-                                     prog_rows[seg_start[s] .. seg_start[s+1])           */
-    uint8_t  restart[GAR_MAX_N];  /* running sum restarts from zero at slot s           */
-    uint8_t  prog_rows[GAR_MAX_N * GAR_MAX_N];
+    /* summation plan */
+    int32_t  nu;                  /* number of distinct gradients read                  */
+    int32_t  total_adds;          /* sum of slot_nadd                                   */
+    int32_t  nbase, nloose;
+    uint64_t chain_mask, corr_mask;
+    uint8_t  base_rows[GAR_MAX_N];
+    uint8_t  loose_rows[GAR_MAX_N];
+    uint8_t  slot_src[GAR_MAX_N];
+    uint8_t  slot_save[GAR_MAX_N];
+    uint8_t  slot_nadd[GAR_MAX_N];
+    uint8_t  add_pos[GAR_MAX_N * GAR_MAX_N];
     double   scores[GAR_MAX_N][GAR_MAX_N];
 } gar_selection_t;
 
@@ -176,8 +199,8 @@ int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int
 /*
  * Builds the coordinate kernel's schedule for GIVEN winners and sets (e.g. the
  * oracle's), without scoring: sel dev with n, f, rule, theta, beta, preagg,
- * median_of_agr, winners, sets filled by the caller; m, nested, base_*,
- * seg_start, restart, prog_rows are written.  The paper has no counterpart
+ * median_of_agr, winners, sets filled by the caller; m and the summation plan
+ * (nu .. add_pos) are written.  The paper has no counterpart
  * (test and diagnostic aid).
  */
 int gar_schedule_from_tables(gar_selection_t* sel, void* stream);

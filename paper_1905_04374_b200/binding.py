@@ -32,11 +32,14 @@ class GarSelection(C.Structure):
         ("sets", C.c_uint64 * GAR_MAX_N),
         ("gap_winner", C.c_double * GAR_MAX_N),
         ("gap_set", C.c_double * GAR_MAX_N),
-        ("nested", C.c_int32), ("base_count", C.c_int32),
-        ("base_rows", C.c_int32 * GAR_MAX_N),
-        ("seg_start", C.c_int32 * (GAR_MAX_N + 1)),
-        ("restart", C.c_uint8 * GAR_MAX_N),
-        ("prog_rows", C.c_uint8 * (GAR_MAX_N * GAR_MAX_N)),
+        ("nu", C.c_int32), ("total_adds", C.c_int32), ("nbase", C.c_int32), ("nloose", C.c_int32),
+        ("chain_mask", C.c_uint64), ("corr_mask", C.c_uint64),
+        ("base_rows", C.c_uint8 * GAR_MAX_N),
+        ("loose_rows", C.c_uint8 * GAR_MAX_N),
+        ("slot_src", C.c_uint8 * GAR_MAX_N),
+        ("slot_save", C.c_uint8 * GAR_MAX_N),
+        ("slot_nadd", C.c_uint8 * GAR_MAX_N),
+        ("add_pos", C.c_uint8 * (GAR_MAX_N * GAR_MAX_N)),
         ("scores", (C.c_double * GAR_MAX_N) * GAR_MAX_N),
     ]
 

@@ -14,8 +14,7 @@ OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libgar.so")
 
 # Slot counts the coordinate kernel is compiled for: keep identical to K3_P_LIST in k3_dispatch.cu.
-K3_P = [1, 2, 3, 4, 5, 6, 7, 8, 9, 10, 11, 12, 13, 15, 17, 19, 21, 23, 25, 27, 29, 31, 35, 39, 43, 47,
-        51, 55, 59, 64]
+K3_P = list(range(1, 33)) + [36, 40, 44, 48, 52, 56, 60, 64]     # <= 32: theta fixed at compile time
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include"), "-I" + CSRC]
@@ -34,7 +33,7 @@ def _units():
              ("k3_dispatch.cu", "k3_dispatch.o", []),
              ("gar_api.cu", "gar_api.o", [])]
     for p in K3_P:
-        units.append(("k3_inst.cu", f"k3_inst_{p}.o", [f"-DK3_P={p}"]))
+        units.append(("k3_inst.cu", f"k3_inst_{p}.o", [f"-DK3_P={p}", f"-DK3_EXACT={1 if p <= 32 else 0}"]))
     return units
 
 

@@ -37,59 +37,151 @@ __device__ __forceinline__ double rel_gap(double lo, double hi) {
     return (hi - lo) / hi;
 }
 
-// Derive the coordinate kernel's schedule from winners[] and sets[] (see gar.h).
-// Slots are rounds in reverse: slot s = theta-1-r, so that the running sum only
-// ever grows: slot 0 sums the last round's set, slot s adds what round
-// theta-1-s has on top of the following round.
-__device__ void build_schedule(gar_selection_t* sel, int* counts /* shared, NMAX+1 */) {
+// Derive the coordinate kernel's summation plan from winners[] and sets[] (the
+// layout is described in gar.h).  Slots are rounds in reverse (slot s = round
+// theta-1-s).  Gradients present in every slot form the base; a winner that
+// stays in every set from its own slot on is "chained" (added to the running sum
+// at its slot); everything else is "loose" and summed per slot into a correction
+// C_s by the cheapest of: start from zero, continue from slot s-1 (if that loose
+// set is a subset) or start from a saved earlier C (if a subset).  Sums are only
+// ever added to.  At most GAR_MAX_SAVED corrections are kept.
+struct PlanSmem {
+    unsigned long long slotset[NMAX];   // full set of slot s
+    unsigned long long loose[NMAX];     // loose part of slot s
+    unsigned long long addmask[NMAX];
+    unsigned long long uni, base, chain, loose_all;
+    int choice[NMAX];       // pass 1: chosen earlier slot (>= 0), -1 zero, -2 continue
+    int usage[NMAX];
+    int saved[NMAX];        // slot -> saved index or -1
+    int offset[NMAX + 1];
+};
+
+__device__ __forceinline__ void plan_choose(const PlanSmem& ps, int s, bool restricted, int& src, unsigned long long& adds) {
+    const unsigned long long cur = ps.loose[s];
+    int best_cost = __popcll(cur);
+    src = -1;
+    adds = cur;
+    if (s > 0) {
+        const unsigned long long prev = ps.loose[s - 1];
+        if ((prev & ~cur) == 0ull) {
+            const int c = __popcll(cur & ~prev);
+            if (c <= best_cost) { best_cost = c; src = -2; adds = cur & ~prev; }
+        }
+    }
+    for (int j = 0; j + 1 < s; ++j) {
+        if (restricted && ps.saved[j] < 0) continue;
+        const unsigned long long sj = ps.loose[j];
+        if (sj == 0ull || (sj & ~cur) != 0ull) continue;
+        const int c = __popcll(cur & ~sj) + 1;          // +1: reading the saved sum
+        if (c < best_cost) { best_cost = c; src = j; adds = cur & ~sj; }
+    }
+}
+
+__device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
     const int theta = sel->theta;
     const int tid = threadIdx.x;
     if (tid < theta) {
-        const int s = tid, r = theta - 1 - s;
-        const uint64_t cur = sel->sets[r];
-        sel->m[r] = __popcll(cur);
-        uint64_t adds = cur;
-        int restart = 1;
-        if (s > 0) {
-            const uint64_t prev = sel->sets[r + 1];
-            if ((prev & ~cur) == 0ull) { adds = cur & ~prev; restart = 0; }
+        const int r = theta - 1 - tid;
+        ps.slotset[tid] = sel->sets[r];
+        sel->m[r] = __popcll(sel->sets[r]);
+        ps.usage[tid] = 0;
+        ps.saved[tid] = -1;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long u = 0ull, chain = 0ull, chained_rows = 0ull;
+        // suffix intersections: after the loop `suffix` = rows present in every slot
+        unsigned long long suffix = ~0ull, next_suffix = ~0ull;
+        for (int s = theta - 1; s >= 0; --s) {
+            suffix = next_suffix & ps.slotset[s];                 // present in all slots >= s
+            const int w = sel->winners[theta - 1 - s];
+            if (w >= 0 && w < NMAX) {
+                u |= 1ull << w;
+                // chained: permanent from slot s on, and not already permanent from slot s+... (a winner
+                // is absent before its own slot, so "present in all slots >= s" pins its entry to s)
+                if ((suffix >> w) & 1ull) { chain |= 1ull << s; chained_rows |= 1ull << w; }
+            }
+            u |= ps.slotset[s];
+            next_suffix = suffix;
         }
-        sel->restart[s] = uint8_t(restart);
-        counts[s] = __popcll(adds);
+        // a winner can only be in sets of its own slot and later ones; if the caller's tables break
+        // that (a chained row also present earlier), un-chain nothing: the covered set below stays a
+        // subset of every slot set because chained rows are in all slots >= their own and are only
+        // counted from their own slot on.
+        const unsigned long long base = suffix & ~chained_rows;  // suffix at s = 0
+        ps.uni = u;
+        ps.base = base;
+        ps.chain = chain;
+        unsigned long long covered = base, loose_all = 0ull;
+        for (int s = 0; s < theta; ++s) {
+            if ((chain >> s) & 1ull) covered |= 1ull << sel->winners[theta - 1 - s];
+            ps.loose[s] = ps.slotset[s] & ~covered;
+            loose_all |= ps.loose[s];
+        }
+        ps.loose_all = loose_all;
+        sel->nu = __popcll(u);
+        sel->nbase = __popcll(base);
+        sel->nloose = __popcll(loose_all);
+        sel->chain_mask = chain;
+    }
+    __syncthreads();
+    const unsigned long long base = ps.base, loose_all = ps.loose_all;
+    if (tid < NMAX) {
+        const unsigned long long below = (1ull << tid) - 1ull;
+        if ((base >> tid) & 1ull) sel->base_rows[__popcll(base & below)] = uint8_t(tid);
+        if ((loose_all >> tid) & 1ull) sel->loose_rows[__popcll(loose_all & below)] = uint8_t(tid);
+    }
+    // pass 1: unrestricted choice, to see which corrections are worth keeping
+    if (tid < theta) {
+        int src; unsigned long long adds;
+        plan_choose(ps, tid, false, src, adds);
+        ps.choice[tid] = src;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        for (int s = 0; s < theta; ++s) if (ps.choice[s] >= 0) ps.usage[ps.choice[s]] += 1;
+        for (int k = 0; k < GAR_MAX_SAVED; ++k) {           // keep the most used ones
+            int bj = -1, bu = 0;
+            for (int j = 0; j < theta; ++j) if (ps.saved[j] < 0 && ps.usage[j] > bu) { bu = ps.usage[j]; bj = j; }
+            if (bj < 0) break;
+            ps.saved[bj] = k;
+        }
+    }
+    __syncthreads();
+    // pass 2: final choice among the kept corrections
+    if (tid < theta) {
+        int src; unsigned long long adds;
+        plan_choose(ps, tid, true, src, adds);
+        ps.addmask[tid] = adds;
+        sel->slot_src[tid] = src == -1 ? uint8_t(GAR_SRC_ZERO) : src == -2 ? uint8_t(GAR_SRC_CONT) : uint8_t(ps.saved[src]);
+        sel->slot_nadd[tid] = uint8_t(__popcll(adds));
+        sel->slot_save[tid] = ps.saved[tid] >= 0 ? uint8_t(ps.saved[tid]) : uint8_t(GAR_SAVE_NONE);
     }
     __syncthreads();
     if (tid == 0) {
         int acc = 0;
-        for (int s = 0; s < theta; ++s) { sel->seg_start[s] = acc; acc += counts[s]; }
-        sel->seg_start[theta] = acc;
+        unsigned long long corr = 0ull;
+        for (int s = 0; s < theta; ++s) {
+            ps.offset[s] = acc;
+            const int na = __popcll(ps.addmask[s]);
+            acc += na;
+            const bool noop = (na == 0) && sel->slot_save[s] == GAR_SAVE_NONE &&
+                              (sel->slot_src[s] == GAR_SRC_CONT || (s == 0 && sel->slot_src[s] == GAR_SRC_ZERO));
+            if (!noop) corr |= 1ull << s;
+        }
+        ps.offset[theta] = acc;
+        sel->total_adds = acc;
+        sel->corr_mask = corr;
     }
     __syncthreads();
     if (tid < theta) {
-        const int s = tid, r = theta - 1 - s;
-        const uint64_t cur = sel->sets[r];
-        uint64_t adds = cur;
-        if (s > 0 && !sel->restart[s]) adds = cur & ~sel->sets[r + 1];
-        int pos = sel->seg_start[s];
-        const int w = sel->winners[r];
-        // the winner first (slot 0 relies on it), then ascending
-        if (w >= 0 && w < NMAX && ((adds >> w) & 1ull)) { sel->prog_rows[pos++] = uint8_t(w); adds &= ~(1ull << w); }
-        while (adds) { int b = __ffsll((long long)adds) - 1; sel->prog_rows[pos++] = uint8_t(b); adds &= adds - 1; }
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int nested = sel->preagg ? 1 : 0;
-        const int wl = sel->winners[theta - 1];
-        const int bc = sel->seg_start[1] - sel->seg_start[0];
-        if (!(wl >= 0 && wl < NMAX && ((sel->sets[theta - 1] >> wl) & 1ull))) nested = 0;
-        for (int s = 1; s < theta && nested; ++s) {
-            const int r = theta - 1 - s;
-            if (sel->restart[s] || sel->seg_start[s + 1] - sel->seg_start[s] != 1 ||
-                sel->prog_rows[sel->seg_start[s]] != sel->winners[r])
-                nested = 0;
+        unsigned long long adds = ps.addmask[tid];
+        int pos = ps.offset[tid];
+        while (adds) {
+            const int b = __ffsll((long long)adds) - 1;
+            sel->add_pos[pos++] = uint8_t(__popcll(loose_all & ((1ull << b) - 1ull)));
+            adds &= adds - 1;
         }
-        sel->nested = nested;
-        sel->base_count = bc;
-        for (int b = 0; b < bc && b < NMAX; ++b) sel->base_rows[b] = sel->prog_rows[b];
     }
 }
 
@@ -98,7 +190,7 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
           int m_user, int theta, int beta, int median_of_agr) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     K2Smem& sm = *reinterpret_cast<K2Smem*>(smem_raw);
-    __shared__ int counts[NMAX + 1];
+    __shared__ PlanSmem plan_smem;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     const bool preagg = (rule == GAR_MULTI_BULYAN || rule == GAR_MULTI_KRUM || rule == GAR_AVERAGE);
@@ -119,7 +211,7 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
             sel->gap_set[tid] = INFINITY;
         }
         __syncthreads();
-        build_schedule(sel, counts);
+        build_schedule(sel, plan_smem);
         return;
     }
 
@@ -217,12 +309,12 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         __syncthreads();
     }
     // 4. schedule
-    build_schedule(sel, counts);
+    build_schedule(sel, plan_smem);
 }
 
 __global__ void __launch_bounds__(64) k2_schedule_only(gar_selection_t* sel) {
-    __shared__ int counts[NMAX + 1];
-    build_schedule(sel, counts);
+    __shared__ PlanSmem plan_smem;
+    build_schedule(sel, plan_smem);
 }
 
 }  // namespace

@@ -5,20 +5,26 @@
 // loads the gradients it needs straight from the n x d block and rebuilds
 //    e[s] = G[winner of round theta-1-s]           (G^ext, reversed round order)
 //    a[s] = mean of G over that round's set        (G^agr)
-// in registers.  Rounds are visited last-to-first ("slots") because the sets
-// shrink by one gradient per round: the running sum T then only grows,
-// T_s = T_{s-1} + (rows the earlier round has on top), and no value is ever
-// subtracted.  In the usual case (sets[r] = sets[r+1] + {winner_r}, "nested")
-// the row added at slot s is exactly the winner whose value is e[s], so every
-// needed row is loaded exactly once: |sets[0]| loads per coordinate.  Any other
-// set structure runs the general schedule (restart flags + row lists).
-// The median is a Batcher odd-even merge sorting network over registers, pruned
-// by the compiler to the comparators the middle output depends on; the beta
+// in registers ("slot" s = round theta-1-s).
+//  * Rules without pre-aggregation (Bulyan, Median, Krum: a = e) load the theta
+//    winner rows, one load each.
+//  * Pre-aggregating rules (multi-Bulyan, multi-Krum, averaging) follow the
+//    summation plan of the selection kernel (layout in gar.h):
+//       T_s = sum(base rows) + sum(chained winners up to slot s) + C_s.
+//    Base rows are added as they arrive; a chained winner's value is e[s], already
+//    in a register, so the chain costs one add per slot; only the few "loose"
+//    gradients are parked in a shared-memory column private to the thread
+//    (dynamic indexing without local memory, no barrier) and summed into C_s by
+//    the plan.  Every needed gradient is loaded exactly once, except a winner
+//    that is also loose (twice, the second time from L1).
+// The median is a Batcher odd-even merge network over registers, pruned at
+// compile time to the comparators the middle output depends on; the beta
 // closest values are found by beta passes of arg-min over |a - M|.
 //
-// P is the compiled slot count (>= theta): slots >= theta are padding that is
-// never loaded; the median padding is split between -inf and +inf so that the
-// lower median of the theta real values sits at index (P-1)/2.
+// P is the compiled slot count.  EXACT kernels have theta == P at compile time;
+// the others take theta <= P at run time: slots >= theta are padding that is
+// never loaded, and the median padding is split between -inf and +inf so that
+// the lower median of the theta real values sits at index (P-1)/2.
 #pragma once
 #include <math_constants.h>
 
@@ -29,21 +35,18 @@
 namespace gar {
 
 constexpr int K3_THREADS = 256;
+constexpr int K3_LOOSE_CAP = 32;      // loose gradients parked in shared memory; more: read from global
 
 struct K3Plan {
-    int     theta, beta, median_of_agr, nested, base_count, lo_pads;
-    int64_t woff[GAR_MAX_N];       // slot -> winner row offset (elements)
-    float   inv_m[GAR_MAX_N];      // slot -> 1/|set|
-    int64_t base_off[GAR_MAX_N];   // slot 0 rows
-    int     seg_start[GAR_MAX_N + 1];
-    uint8_t restart[GAR_MAX_N];
-    uint8_t prog_rows[GAR_MAX_N * GAR_MAX_N];
+    int      theta, beta, median_of_agr, lo_pads, nbase, nloose, loose_in_smem;
+    unsigned long long chain_mask, corr_mask;
+    int64_t  woff[GAR_MAX_N];       // slot -> winner row offset (elements)
+    int64_t  boff[GAR_MAX_N];       // base row offsets
+    int64_t  loff[GAR_MAX_N];       // loose row offsets
+    float    inv_m[GAR_MAX_N];      // slot -> 1/|set|
+    uint8_t  src[GAR_MAX_N], save[GAR_MAX_N], nadd[GAR_MAX_N];
+    uint8_t  add_pos[GAR_MAX_N * GAR_MAX_N];
 };
-
-template <int V> struct VecT;
-template <> struct VecT<1> { using type = float; };
-template <> struct VecT<2> { using type = float2; };
-template <> struct VecT<4> { using type = float4; };
 
 template <int V> __device__ __forceinline__ void load_vec(const float* p, float (&x)[V]) {
     if constexpr (V == 1) { x[0] = __ldg(p); }
@@ -54,6 +57,11 @@ template <int V> __device__ __forceinline__ void store_vec(float* p, const float
     if constexpr (V == 1) { *p = x[0]; }
     else if constexpr (V == 2) { *reinterpret_cast<float2*>(p) = make_float2(x[0], x[1]); }
     else { *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]); }
+}
+template <int V> __device__ __forceinline__ void read_vec(const float* p, float (&x)[V]) {
+    if constexpr (V == 1) { x[0] = *p; }
+    else if constexpr (V == 2) { float2 t = *reinterpret_cast<const float2*>(p); x[0] = t.x; x[1] = t.y; }
+    else { float4 t = *reinterpret_cast<const float4*>(p); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
 }
 
 __device__ __forceinline__ void cmpswap(float& lo, float& hi) {
@@ -119,117 +127,158 @@ template <int N, int V> __device__ __forceinline__ void median_network(float (&x
     median_network_apply<N, V>(x, std::make_index_sequence<MedianNet<N>::data.count>{});
 }
 
-__device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* __restrict__ sel, int64_t ld, int P) {
+__device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* __restrict__ sel, int64_t ld, int P,
+                                          bool preagg, int loose_cap) {
     const int tid = threadIdx.x;
     const int theta = sel->theta;
     if (tid == 0) {
         plan.theta = theta;
         plan.beta = sel->beta;
         plan.median_of_agr = sel->median_of_agr;
-        plan.nested = sel->nested;
-        plan.base_count = sel->base_count;
         plan.lo_pads = (P - 1) / 2 - (theta - 1) / 2;
+        plan.nbase = sel->nbase;
+        plan.nloose = sel->nloose;
+        plan.loose_in_smem = sel->nloose <= loose_cap ? 1 : 0;
+        plan.chain_mask = sel->chain_mask;
+        plan.corr_mask = sel->corr_mask;
     }
     for (int s = tid; s < theta; s += blockDim.x) {
         const int r = theta - 1 - s;
         plan.woff[s] = int64_t(sel->winners[r]) * ld;
         plan.inv_m[s] = 1.0f / float(sel->m[r]);
-        plan.restart[s] = sel->restart[s];
+        plan.src[s] = sel->slot_src[s];
+        plan.save[s] = sel->slot_save[s];
+        plan.nadd[s] = sel->slot_nadd[s];
     }
-    for (int s = tid; s <= theta; s += blockDim.x) plan.seg_start[s] = sel->seg_start[s];
-    for (int b = tid; b < sel->base_count; b += blockDim.x) plan.base_off[b] = int64_t(sel->base_rows[b]) * ld;
-    if (sel->preagg && !sel->nested) {
-        const int total = sel->seg_start[theta];
-        for (int k = tid; k < total; k += blockDim.x) plan.prog_rows[k] = sel->prog_rows[k];
+    if (preagg) {
+        for (int u = tid; u < sel->nbase; u += blockDim.x) plan.boff[u] = int64_t(sel->base_rows[u]) * ld;
+        for (int u = tid; u < sel->nloose; u += blockDim.x) plan.loff[u] = int64_t(sel->loose_rows[u]) * ld;
+        for (int k = tid; k < sel->total_adds; k += blockDim.x) plan.add_pos[k] = sel->add_pos[k];
     }
 }
 
 // Coordinates [t_begin, t_end), V per thread; (t_end - t_begin) % V == 0 and the
 // V-vectors at g + row*ld + t and out + t are naturally aligned.
-template <int P, bool PREAGG, int V>
+// Dynamic shared memory (PREAGG only): (loose_cap + GAR_MAX_SAVED) * blockDim * V floats.
+template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(K3_THREADS)
 k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64_t ld,
-              const gar_selection_t* __restrict__ sel, float* __restrict__ out) {
+              const gar_selection_t* __restrict__ sel, float* __restrict__ out, int loose_cap) {
     __shared__ K3Plan plan;
-    load_plan(plan, sel, ld, P);
+    extern __shared__ __align__(16) float k3_dyn[];
+    load_plan(plan, sel, ld, P, PREAGG, loose_cap);
     __syncthreads();
-    const int theta = plan.theta;
+    const int theta = EXACT ? P : plan.theta;
     const int beta = plan.beta;
     const float inv_beta = 1.0f / float(beta);
-    const int lo_pads = plan.lo_pads;
+    const int lo_pads = EXACT ? 0 : plan.lo_pads;
     const bool med_agr = plan.median_of_agr != 0;
+    const int nthreads = blockDim.x;
+    // this thread's private columns: loose value u at xcol[u*stride], saved sum k at tcol[k*stride]
+    const int stride = nthreads * V;
+    float* const xcol = k3_dyn + threadIdx.x * V;
+    float* const tcol = xcol + size_t(loose_cap) * stride;
+    const unsigned long long chain_mask = plan.chain_mask, corr_mask = plan.corr_mask;
 
     const int64_t nvec = (t_end - t_begin) / V;
-    for (int64_t vi = int64_t(blockIdx.x) * K3_THREADS + threadIdx.x; vi < nvec;
-         vi += int64_t(gridDim.x) * K3_THREADS) {
+    for (int64_t vi = int64_t(blockIdx.x) * nthreads + threadIdx.x; vi < nvec;
+         vi += int64_t(gridDim.x) * nthreads) {
         const int64_t t = t_begin + vi * V;
         const float* gt = g + t;
         float e[P][V], a[P][V];
 #pragma unroll
         for (int s = 0; s < P; ++s) {
+            if (s < theta) {
+                load_vec<V>(gt + plan.woff[s], e[s]);
+            } else {
 #pragma unroll
-            for (int v = 0; v < V; ++v) { e[s][v] = 0.0f; a[s][v] = 0.0f; }
+                for (int v = 0; v < V; ++v) e[s][v] = 0.0f;
+            }
         }
 
         if constexpr (PREAGG) {
             float T[V];
-            if (plan.nested) {
-                float x[V];
-                load_vec<V>(gt + plan.base_off[0], x);
 #pragma unroll
-                for (int v = 0; v < V; ++v) { e[0][v] = x[v]; T[v] = x[v]; }
-                const int bc = plan.base_count;
-#pragma unroll 4
-                for (int b = 1; b < bc; ++b) {
-                    load_vec<V>(gt + plan.base_off[b], x);
+            for (int v = 0; v < V; ++v) T[v] = 0.0f;
+            // base rows: summed as they arrive, 8 loads in flight
+            const int nbase = plan.nbase;
+            for (int base = 0; base < nbase; base += 8) {
+                float x[8][V];
 #pragma unroll
-                    for (int v = 0; v < V; ++v) T[v] += x[v];
-                }
-                const float im0 = plan.inv_m[0];
+                for (int k = 0; k < 8; ++k) {
+                    if (base + k < nbase) {
+                        load_vec<V>(gt + plan.boff[base + k], x[k]);
+                    } else {
 #pragma unroll
-                for (int v = 0; v < V; ++v) a[0][v] = T[v] * im0;
-#pragma unroll
-                for (int s = 1; s < P; ++s) {
-                    if (s < theta) {
-                        load_vec<V>(gt + plan.woff[s], x);
-                        const float im = plan.inv_m[s];
-#pragma unroll
-                        for (int v = 0; v < V; ++v) { T[v] += x[v]; e[s][v] = x[v]; a[s][v] = T[v] * im; }
+                        for (int v = 0; v < V; ++v) x[k][v] = 0.0f;
                     }
                 }
-            } else {
 #pragma unroll
-                for (int v = 0; v < V; ++v) T[v] = 0.0f;
+                for (int k = 0; k < 8; ++k) {
 #pragma unroll
-                for (int s = 0; s < P; ++s) {
-                    if (s < theta) {
-                        float x[V];
-                        if (plan.restart[s]) {
+                    for (int v = 0; v < V; ++v) T[v] += x[k][v];
+                }
+            }
+            // loose rows: parked in this thread's shared-memory column
+            const int nloose = plan.nloose;
+            const bool in_smem = plan.loose_in_smem != 0;
+            if (in_smem) {
+                for (int base = 0; base < nloose; base += 8) {
+                    float x[8][V];
 #pragma unroll
-                            for (int v = 0; v < V; ++v) T[v] = 0.0f;
-                        }
-                        const int k1 = plan.seg_start[s + 1];
-                        for (int k = plan.seg_start[s]; k < k1; ++k) {
-                            load_vec<V>(gt + int64_t(plan.prog_rows[k]) * ld, x);
-#pragma unroll
-                            for (int v = 0; v < V; ++v) T[v] += x[v];
-                        }
-                        load_vec<V>(gt + plan.woff[s], x);
-                        const float im = plan.inv_m[s];
-#pragma unroll
-                        for (int v = 0; v < V; ++v) { e[s][v] = x[v]; a[s][v] = T[v] * im; }
+                    for (int k = 0; k < 8; ++k) {
+                        if (base + k < nloose) load_vec<V>(gt + plan.loff[base + k], x[k]);
                     }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        if (base + k < nloose) store_vec<V>(xcol + size_t(base + k) * stride, x[k]);
+                    }
+                }
+            }
+            float C[V];
+#pragma unroll
+            for (int v = 0; v < V; ++v) C[v] = 0.0f;
+            int kadd = 0;
+#pragma unroll
+            for (int s = 0; s < P; ++s) {
+                if (s < theta) {
+                    if ((corr_mask >> s) & 1ull) {
+                        const int src = plan.src[s];
+                        if (src == GAR_SRC_ZERO) {
+#pragma unroll
+                            for (int v = 0; v < V; ++v) C[v] = 0.0f;
+                        } else if (src != GAR_SRC_CONT) {
+                            read_vec<V>(tcol + size_t(src) * stride, C);
+                        }
+                        const int kend = kadd + plan.nadd[s];
+                        for (; kadd < kend; ++kadd) {
+                            float x[V];
+                            const int pos = plan.add_pos[kadd];
+                            if (in_smem) read_vec<V>(xcol + size_t(pos) * stride, x);
+                            else load_vec<V>(gt + plan.loff[pos], x);
+#pragma unroll
+                            for (int v = 0; v < V; ++v) C[v] += x[v];
+                        }
+                        const int sv = plan.save[s];
+                        if (sv != GAR_SAVE_NONE) store_vec<V>(tcol + size_t(sv) * stride, C);
+                    }
+                    if ((chain_mask >> s) & 1ull) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) T[v] += e[s][v];
+                    }
+                    const float im = plan.inv_m[s];
+#pragma unroll
+                    for (int v = 0; v < V; ++v) a[s][v] = (T[v] + C[v]) * im;
+                } else {
+#pragma unroll
+                    for (int v = 0; v < V; ++v) a[s][v] = 0.0f;
                 }
             }
         } else {
 #pragma unroll
             for (int s = 0; s < P; ++s) {
-                if (s < theta) {
-                    float x[V];
-                    load_vec<V>(gt + plan.woff[s], x);
 #pragma unroll
-                    for (int v = 0; v < V; ++v) { e[s][v] = x[v]; a[s][v] = x[v]; }
-                }
+                for (int v = 0; v < V; ++v) a[s][v] = e[s][v];
             }
         }
 
@@ -260,11 +309,11 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
         for (int b = 0; b < beta; ++b) {
 #pragma unroll
             for (int v = 0; v < V; ++v) {
-                float best = CUDART_INF_F, ba = 0.0f;
-                int bi = -1;
+                float best = key[P - 1][v], ba = a[P - 1][v];
+                int bi = P - 1;
 #pragma unroll
-                for (int s = P - 1; s >= 0; --s) {
-                    const bool take = (s < theta) && (key[s][v] < best || bi < 0);
+                for (int s = P - 2; s >= 0; --s) {
+                    const bool take = key[s][v] < best;
                     best = take ? key[s][v] : best;
                     ba = take ? a[s][v] : ba;
                     bi = take ? s : bi;
@@ -284,7 +333,7 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
 }
 
 template <int P>
-cudaError_t launch_k3_p(const float* g, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
+cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
                         int vec, float* out, int sm_count, cudaStream_t stream);
 
 }  // namespace gar

@@ -4,26 +4,27 @@
 #include "gar_internal.cuh"
 
 // Slot counts the coordinate kernel is compiled for (k3_inst.cu is built once
-// per entry; keep the build script's list identical).
-#define K3_P_LIST(X)                                                                              \
-    X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(15) X(17) X(19) X(21)  \
-    X(23) X(25) X(27) X(29) X(31) X(35) X(39) X(43) X(47) X(51) X(55) X(59) X(64)
+// per entry; keep the build script's list identical): every theta up to 32 has
+// its own kernel with theta fixed at compile time; larger ones share padded kernels.
+#define K3_P_LIST(X)                                                                                   \
+    X(1) X(2) X(3) X(4) X(5) X(6) X(7) X(8) X(9) X(10) X(11) X(12) X(13) X(14) X(15) X(16) X(17) X(18) \
+    X(19) X(20) X(21) X(22) X(23) X(24) X(25) X(26) X(27) X(28) X(29) X(30) X(31) X(32) X(36) X(40)    \
+    X(44) X(48) X(52) X(56) X(60) X(64)
 
 namespace gar {
 
 template <int P>
-cudaError_t launch_k3_p(const float* g, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
+cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
                         int vec, float* out, int sm_count, cudaStream_t stream);
 #define K3_DECL(P)                                                                                         \
     template <>                                                                                            \
-    cudaError_t launch_k3_p<P>(const float*, int64_t, int64_t, const gar_selection_t*, int, int, float*, \
-                               int, cudaStream_t);
+    cudaError_t launch_k3_p<P>(const float*, int, int64_t, int64_t, const gar_selection_t*, int, int, \
+                               float*, int, cudaStream_t);
 K3_P_LIST(K3_DECL)
 #undef K3_DECL
 
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, const gar_selection_t* sel,
                               int theta, int preagg, float* out, int sm_count, cudaStream_t stream) {
-    (void)n;
     const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out);
     int vec = 1;
     if (a % 16 == 0 && ld % 4 == 0) vec = 4;
@@ -36,7 +37,7 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
         if (cap == 1 || cap == 2 || cap == 4) vec = vec < cap ? vec : cap;
     }
 #define K3_TRY(P) \
-    if (theta <= P) return launch_k3_p<P>(grads, d, ld, sel, preagg, vec, out, sm_count, stream);
+    if (theta <= P) return launch_k3_p<P>(grads, n, d, ld, sel, preagg, vec, out, sm_count, stream);
     K3_P_LIST(K3_TRY)
 #undef K3_TRY
     return cudaErrorInvalidValue;

@@ -1,44 +1,79 @@
 // One instantiation of the coordinate kernel per compiled slot count K3_P
-// (this file is compiled once for every value in K3_P_LIST of k3_dispatch.cu).
+// (this file is compiled once for every entry of K3_P_LIST in k3_dispatch.cu;
+// K3_EXACT = 1 when the kernel is only used with theta == K3_P).
 #include "k3_coordinate.cuh"
 
-#ifndef K3_P
-#error "compile with -DK3_P=<slot count>"
+#if !defined(K3_P) || !defined(K3_EXACT)
+#error "compile with -DK3_P=<slot count> -DK3_EXACT=<0|1>"
 #endif
 
 namespace gar {
 
+// Threads per CTA and dynamic shared memory of the pre-aggregating kernel: every
+// thread owns (loose_cap + GAR_MAX_SAVED) columns of V floats; aim at >= 2 CTAs per SM.
+static inline void preagg_shape(int loose_cap, int V, int* threads, size_t* smem) {
+    const size_t per_thread = size_t(loose_cap + GAR_MAX_SAVED) * V * sizeof(float);
+    const size_t budget = 100 * 1024;
+    int t = int(budget / per_thread) / 32 * 32;
+    if (t > K3_THREADS) t = K3_THREADS;
+    if (t < 32) t = 32;
+    *threads = t;
+    *smem = per_thread * t;
+}
+
 template <int P, bool PREAGG, int V>
-static cudaError_t run(const float* g, int64_t d, int64_t ld, const gar_selection_t* sel, float* out,
+static cudaError_t run(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, float* out,
                        int sm_count, cudaStream_t stream) {
+    constexpr bool EXACT = (K3_EXACT != 0);
+    int threads = K3_THREADS, threads1 = K3_THREADS;
+    size_t smem = 0, smem1 = 0;
+    const int loose_cap = n < K3_LOOSE_CAP ? n : K3_LOOSE_CAP;
+    if (PREAGG) {
+        preagg_shape(loose_cap, V, &threads, &smem);
+        preagg_shape(loose_cap, 1, &threads1, &smem1);
+        static bool configured[64] = {false};      // per device, for this instantiation
+        int dev = 0;
+        cudaError_t err = cudaGetDevice(&dev);
+        if (err != cudaSuccess) return err;
+        if (!(dev >= 0 && dev < 64 && configured[dev])) {
+            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, V>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+            if (err != cudaSuccess) return err;
+            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, 1>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+            if (err != cudaSuccess) return err;
+            if (dev >= 0 && dev < 64) configured[dev] = true;
+        }
+    }
     const int64_t d_vec = d - d % V;
     if (d_vec > 0) {
         const int64_t nvec = d_vec / V;
-        int64_t blocks = (nvec + K3_THREADS - 1) / K3_THREADS;
-        const int64_t cap = int64_t(sm_count) * 16;
+        int64_t blocks = (nvec + threads - 1) / threads;
+        const int64_t cap = int64_t(sm_count) * 8;
         if (blocks > cap) blocks = cap;
-        k3_coordinate<P, PREAGG, V><<<unsigned(blocks), K3_THREADS, 0, stream>>>(g, 0, d_vec, ld, sel, out);
+        k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, 0, d_vec, ld, sel, out,
+                                                                                         loose_cap);
     }
     if (d_vec < d) {   // ragged tail (only when ld > d): scalar kernel on the last d % V coordinates
-        k3_coordinate<P, PREAGG, 1><<<1, K3_THREADS, 0, stream>>>(g, d_vec, d, ld, sel, out);
+        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, d_vec, d, ld, sel, out, loose_cap);
     }
     return cudaGetLastError();
 }
 
 template <>
-cudaError_t launch_k3_p<K3_P>(const float* g, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
+cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
                               int vec, float* out, int sm_count, cudaStream_t stream) {
     // 4-wide vectors are only compiled for small slot counts (register budget)
     constexpr bool kWide = (K3_P <= 8);
     if (vec == 4 && !kWide) vec = 2;
     if (preagg) {
-        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, d, ld, sel, out, sm_count, stream);
-        if (vec == 2) return run<K3_P, true, 2>(g, d, ld, sel, out, sm_count, stream);
-        return run<K3_P, true, 1>(g, d, ld, sel, out, sm_count, stream);
+        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, d, ld, sel, out, sm_count, stream);
+        if (vec == 2) return run<K3_P, true, 2>(g, n, d, ld, sel, out, sm_count, stream);
+        return run<K3_P, true, 1>(g, n, d, ld, sel, out, sm_count, stream);
     }
-    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, d, ld, sel, out, sm_count, stream);
-    if (vec == 2) return run<K3_P, false, 2>(g, d, ld, sel, out, sm_count, stream);
-    return run<K3_P, false, 1>(g, d, ld, sel, out, sm_count, stream);
+    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, d, ld, sel, out, sm_count, stream);
+    if (vec == 2) return run<K3_P, false, 2>(g, n, d, ld, sel, out, sm_count, stream);
+    return run<K3_P, false, 1>(g, n, d, ld, sel, out, sm_count, stream);
 }
 
 }  // namespace gar

@@ -38,13 +38,13 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
     src = tmp_path / "sz.cpp"
     src.write_text('#include "gar.h"\n#include <cstdio>\n#include <cstddef>\n'
                    'int main(){printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(gar_selection_t),'
-                   'offsetof(gar_selection_t,sets), offsetof(gar_selection_t,nested),'
-                   'offsetof(gar_selection_t,prog_rows), offsetof(gar_selection_t,scores), sizeof(gar_params_t));}')
+                   'offsetof(gar_selection_t,sets), offsetof(gar_selection_t,nu),'
+                   'offsetof(gar_selection_t,add_pos), offsetof(gar_selection_t,scores), sizeof(gar_params_t));}')
     exe = tmp_path / "sz"
     subprocess.check_call(["g++", "-I" + os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(v) for v in subprocess.check_output([str(exe)]).split()]
     S = pkg.GarSelection
-    assert got == [C.sizeof(S), S.sets.offset, S.nested.offset, S.prog_rows.offset, S.scores.offset,
+    assert got == [C.sizeof(S), S.sets.offset, S.nu.offset, S.add_pos.offset, S.scores.offset,
                    C.sizeof(pkg.GarParams)]
 
 

@@ -100,7 +100,7 @@ def test_selection_given_oracle_distances(pkg, rule, cfg, n, f):
             assert sel.sets[r] == sum(1 << i for i in rnd.selected)
         if np.isfinite(rnd.gap_winner):
             assert abs(sel.gap_winner[r] - rnd.gap_winner) <= 1e-9
-    assert sel.nested in (0, 1)
+    assert 1 <= sel.nu <= n
 
 
 def test_selection_integer_ties(pkg):
@@ -144,7 +144,7 @@ def test_coordinate_phase_given_oracle_tables(pkg, cfg, n, f, rule, d):
 
 def test_coordinate_phase_general_schedule(pkg):
     # sets that are NOT nested (a later round holds a row the earlier one lacks):
-    # the kernel must fall back to its general schedule
+    # the summation plan must restart or reuse a saved sum
     n, f, d = 15, 3, 30_011
     G, Gh, _ = draw(pkg, 5, d)
     winners = [4, 9, 1, 12, 6, 0, 7]
@@ -154,7 +154,8 @@ def test_coordinate_phase_general_schedule(pkg):
     ext, agr = O.extracted_and_aggregated(Gh, winners, sets)
     want, _, gap = O.closest_to_median_average(ext, agr, beta)
     dev = _upload_tables(pkg, n, f, 5, winners, sets, beta, 1)
-    assert pkg.read_selection(dev).nested == 0
+    plan = pkg.read_selection(dev)
+    assert plan.nu == 9 and any(plan.slot_src[s] != 254 for s in range(1, 7))   # some slot cannot just continue
     out = pkg.gar_coordinate_phase(G, dev, len(winners), 1).cpu().numpy()
     assert_outputs_match(out, want, G=Gh, tables=dict(winners=winners, sets=sets, beta=beta, gap=gap))
 
@@ -196,7 +197,9 @@ def test_rules_end_to_end(pkg, rule, cfg, n, f, d):
         sets = [[i for i in range(n) if (sel.sets[r] >> i) & 1] for r in range(sel.theta)] if preagg else None
         want2, gap2 = O.coordinate_phase(Gh, winners, sets, sel.beta)
         assert_outputs_match(out, want2, G=Gh, tables=dict(winners=winners, sets=sets, beta=sel.beta, gap=gap2))
-    if rule in ("multi_bulyan", "multi_krum"):
+    if rule in ("multi_bulyan", "multi_krum") and cfg in (1, 3, 5):
+        # far-away Byzantine rows are never averaged (the small-perturbation rows of
+        # workloads 2 and 4 are built to blend in and may be)
         for r in range(sel.theta):
             assert not any((sel.sets[r] >> b) & 1 for b in byz), "a Byzantine row was averaged"
 
@@ -241,9 +244,8 @@ def test_equal_honest_rows_give_that_row(pkg):
     v = torch.randn(d, device=DEV)
     G = v.repeat(n, 1).contiguous()
     G[[2, 8, 13]] = torch.randn(3, d, device=DEV) * 1e3
-    for rule in ("krum", "bulyan"):
-        assert torch.equal(pkg.gar_aggregate(rule, G, f), v)
-    for rule in ("multi_krum", "multi_bulyan"):      # fp32 mean of m equal values: a rounding or two
+    assert torch.equal(pkg.gar_aggregate("krum", G, f), v)
+    for rule in ("bulyan", "multi_krum", "multi_bulyan"):      # fp32 mean of equal values: a rounding or two
         out = pkg.gar_aggregate(rule, G, f)
         assert torch.all((out - v).abs() <= 4e-7 * v.abs())
 
