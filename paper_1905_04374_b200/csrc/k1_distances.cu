@@ -2,66 +2,34 @@
 // streaming pass over the n x d block (Algorithm 1, multi-Krum: the distances
 // to the k-f-2 closest vectors; the only O(n^2 d) step, computed once).
 //
-// Layout of the work
-//  * Rows are grouped in blocks of 8; a "tile" is a pair of row blocks (I <= J).
-//    Off-diagonal tiles hold 64 pairs, diagonal tiles the 28 pairs i < j.
-//  * A CTA walks column slabs of TK coordinates (persistent, slab = cta + k*grid).
-//    A slab of all rows is staged in shared memory through an NSTAGE-deep ring.
-//  * A thread owns one tile and one of 8*G column lanes: it reads 8 + 8 float4
-//    from shared memory and updates 64 (or 28) fp32 accumulators in registers,
-//    (a-b) then fma -- the difference form, exact to fp32 rounding per term.
-//  * fp32 accumulators only ever hold a few dozen terms: every FLUSH slabs they
-//    are reduced over the tile's 8 lanes by shuffles and added to fp64 sums in
-//    shared memory.  CTA sums go to a global partial array; the last CTA to
-//    finish (ticket counter) adds the partials in CTA order in fp64 and writes
-//    the symmetric matrix.  No floating-point atomics: results are
-//    bit-reproducible and D_ij == D_ji by construction.
-#include <cooperative_groups.h>
+// Every pair term is (a-b) then fma in fp32 -- the difference form, exact to
+// fp32 rounding per term.  fp32 accumulators only ever hold a few thousand
+// terms: they are reduced across lanes by shuffles and added to fp64 sums in
+// shared memory.  CTA sums go to a global partial array; the last CTA to finish
+// (ticket counter) adds the partials in CTA order in fp64 and writes the
+// symmetric matrix.  No floating-point atomics: results are bit-reproducible
+// and D_ij == D_ji by construction.
+//
+// Two kernels:
+//  * n <= 16 ("direct"): a thread loads its V coordinates of all n rows straight
+//    from global memory (software-prefetched one iteration ahead) and updates
+//    all n(n-1)/2 accumulators in registers.  No shared-memory staging, no
+//    barrier in the loop; HBM-bound.
+//  * n > 16 ("tiled"): rows are grouped in blocks of 8; a column slab of all rows
+//    is staged in shared memory through a cp.async ring.  A half-warp owns either
+//    one off-diagonal 8x8 tile (64 pairs) or two diagonal tiles (2 x 28 pairs);
+//    warps are homogeneous, so every warp runs one code path and all carry about
+//    the same work.  Every pair sees the same column-to-lane assignment and the
+//    same reduction tree, so identical rows get bit-identical distances.
+//    FMA-pipe-bound.
+#include <cstdlib>
 
 #include "gar_internal.cuh"
 
 namespace gar {
 namespace {
 
-template <int NB> struct K1Shape;
-// G = column-lane groups per tile, KQ = float4 passes per slab, FLUSH = slabs per fp64 flush
-// NSTAGE = depth of the shared-memory ring
-template <> struct K1Shape<1> { static constexpr int G = 32, KQ = 1, FLUSH = 16, NSTAGE = 3; };
-template <> struct K1Shape<2> { static constexpr int G = 12, KQ = 1, FLUSH = 16, NSTAGE = 3; };
-template <> struct K1Shape<3> { static constexpr int G = 6,  KQ = 1, FLUSH = 16, NSTAGE = 4; };
-template <> struct K1Shape<4> { static constexpr int G = 3,  KQ = 2, FLUSH = 8,  NSTAGE = 3; };
-template <> struct K1Shape<5> { static constexpr int G = 2,  KQ = 2, FLUSH = 8,  NSTAGE = 4; };
-template <> struct K1Shape<6> { static constexpr int G = 2,  KQ = 2, FLUSH = 8,  NSTAGE = 4; };
-template <> struct K1Shape<7> { static constexpr int G = 2,  KQ = 2, FLUSH = 8,  NSTAGE = 4; };
-template <> struct K1Shape<8> { static constexpr int G = 1,  KQ = 4, FLUSH = 4,  NSTAGE = 4; };
-
-template <int NB> struct K1Dims {
-    static constexpr int R      = NB * 8;                    // staged rows (zero padded)
-    static constexpr int TILES  = NB * (NB + 1) / 2;
-    static constexpr int OFF    = NB * (NB - 1) / 2;         // off-diagonal tiles come first
-    static constexpr int G      = K1Shape<NB>::G;
-    static constexpr int KQ     = K1Shape<NB>::KQ;
-    static constexpr int FLUSH  = K1Shape<NB>::FLUSH;
-    static constexpr int NSTAGE = K1Shape<NB>::NSTAGE;
-    static constexpr int LANES  = 8 * G;                     // float4 lanes per pass
-    static constexpr int TK4    = LANES * KQ;                // float4 per row per slab
-    static constexpr int TK     = TK4 * 4;                   // coordinates per slab
-    static constexpr int SLOTS  = TILES * G;                 // (tile, group) owners
-    static constexpr int ACTIVE = SLOTS * 8;
-    static constexpr int THREADS = (ACTIVE + 31) / 32 * 32;
-    static constexpr size_t STAGE_BYTES = size_t(R) * TK * 4;
-    static constexpr size_t SUM_BYTES   = size_t(SLOTS) * 64 * sizeof(double);
-    static constexpr size_t SMEM_BYTES  = NSTAGE * STAGE_BYTES + SUM_BYTES;
-};
-
-__device__ __forceinline__ void tile_to_blocks(int p, int nb, int off, int& I, int& J) {
-    if (p >= off) { I = J = p - off; return; }
-    // off-diagonal tiles enumerated row by row: (0,1),(0,2)..(0,nb-1),(1,2)..
-    int i = 0, rem = p;
-    while (rem >= nb - 1 - i) { rem -= nb - 1 - i; ++i; }
-    I = i; J = i + 1 + rem;
-}
-
+// ------------------------------------------------------------------ helpers
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
     unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gsrc), "r"(src_bytes) : "memory");
@@ -69,6 +37,226 @@ __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+// Sum of v[i] over the LANES lanes of a lane group (LANES = 8, 16 or 32, groups
+// aligned), "reduce-scatter" style: each step exchanges half of the remaining
+// values with the partner lane, so the whole reduction costs about COUNT
+// shuffles instead of COUNT*log2(LANES).  COUNT must be a multiple of LANES.
+// On return v[0 .. COUNT/LANES) of lane l holds the totals of the indices
+// scatter_base<COUNT, LANES>(l) + (0 .. COUNT/LANES).
+template <int COUNT, int LANES>
+__device__ __forceinline__ void reduce_scatter(float (&v)[COUNT], int lane) {
+    int len = COUNT;
+#pragma unroll
+    for (int m = LANES / 2; m >= 1; m >>= 1) {
+        const int half = len / 2;
+        const bool upper = (lane & m) != 0;
+#pragma unroll
+        for (int i = 0; i < COUNT / 2; ++i) {
+            if (i < half) {
+                const float lo = v[i], hi = v[i + half];
+                const float send = upper ? lo : hi, keep = upper ? hi : lo;
+                v[i] = keep + __shfl_xor_sync(0xffffffffu, send, m);
+            }
+        }
+        len = half;
+    }
+}
+template <int COUNT, int LANES> __device__ __forceinline__ int scatter_base(int lane) {
+    int base = 0, len = COUNT;
+#pragma unroll
+    for (int m = LANES / 2; m >= 1; m >>= 1) {
+        len /= 2;
+        if (lane & m) base += len;
+    }
+    return base;
+}
+
+// Last-CTA reduction of the per-CTA partial sums (fixed order) -> `combine(slot, sum)`.
+template <typename F>
+__device__ __forceinline__ void reduce_partials(const double* partials, int nslots, int nthreads, F combine) {
+    for (int i = threadIdx.x; i < nslots; i += nthreads) {
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+        unsigned b = 0;
+        for (; b + 4 <= gridDim.x; b += 4) {
+            s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
+            s1 += __ldcg(partials + size_t(b + 1) * kPairSlots + i);
+            s2 += __ldcg(partials + size_t(b + 2) * kPairSlots + i);
+            s3 += __ldcg(partials + size_t(b + 3) * kPairSlots + i);
+        }
+        for (; b < gridDim.x; ++b) s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
+        combine(i, (s0 + s1) + (s2 + s3));
+    }
+}
+
+// Returns true in exactly one CTA: the last one to arrive.  All of this CTA's
+// partial sums must have been written before the call.
+__device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) {
+    __shared__ int is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (is_last) __threadfence();
+    return is_last != 0;
+}
+
+// ======================================================== direct kernel, n <= 16
+constexpr int K1R_THREADS = 128;
+constexpr int K1R_FLUSH = 64;       // iterations between fp64 flushes
+
+template <int N, int V>
+__global__ void __launch_bounds__(K1R_THREADS)
+k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
+          double* __restrict__ partials, unsigned int* __restrict__ ticket) {
+    constexpr int NP = N * (N - 1) / 2;
+    constexpr int NPAD = (NP + 31) / 32 * 32;
+    constexpr int PER_LANE = NPAD / 32;
+    constexpr int WARPS = K1R_THREADS / 32;
+    __shared__ double sums[WARPS][NPAD];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < WARPS * NPAD; i += K1R_THREADS) (&sums[0][0])[i] = 0.0;
+    __syncthreads();
+
+    float acc[NPAD];
+#pragma unroll
+    for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
+    const int sbase = scatter_base<NPAD, 32>(lane);
+
+    auto flush = [&]() {
+        reduce_scatter<NPAD, 32>(acc, lane);
+#pragma unroll
+        for (int i = 0; i < PER_LANE; ++i) sums[warp][sbase + i] += double(acc[i]);
+#pragma unroll
+        for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
+    };
+    // rows of V coordinates at t; a lane past the end gets zeros (they add nothing)
+    auto load_rows = [&](float (&x)[N][V], int64_t t, bool valid) {
+#pragma unroll
+        for (int r = 0; r < N; ++r) {
+            const float* p = g + int64_t(r) * ld + t;
+            if (valid) {
+                if constexpr (V == 4) { float4 q = __ldg(reinterpret_cast<const float4*>(p)); x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w; }
+                else if constexpr (V == 2) { float2 q = __ldg(reinterpret_cast<const float2*>(p)); x[r][0] = q.x; x[r][1] = q.y; }
+                else { x[r][0] = __ldg(p); }
+            } else {
+#pragma unroll
+                for (int v = 0; v < V; ++v) x[r][v] = 0.0f;
+            }
+        }
+    };
+    auto accumulate = [&](const float (&x)[N][V]) {
+        int p = 0;
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+#pragma unroll
+            for (int j = i + 1; j < N; ++j) {
+                float t = acc[p];
+#pragma unroll
+                for (int v = 0; v < V; ++v) { const float df = x[i][v] - x[j][v]; t = fmaf(df, df, t); }
+                acc[p] = t;
+                ++p;
+            }
+        }
+    };
+
+    // the loop bound is per warp, so that the flush (warp-collective) is uniform
+    const int64_t nvec = d / V;
+    const int64_t stride = int64_t(gridDim.x) * K1R_THREADS;
+    int64_t wbase = int64_t(blockIdx.x) * K1R_THREADS + warp * 32;
+    float cur[N][V], nxt[N][V];
+    if (wbase < nvec) load_rows(cur, (wbase + lane) * V, wbase + lane < nvec);
+    int since = 0;
+    while (wbase < nvec) {
+        const int64_t nb = wbase + stride;
+        if (nb < nvec) load_rows(nxt, (nb + lane) * V, nb + lane < nvec);
+        accumulate(cur);
+        if (nb < nvec) {
+#pragma unroll
+            for (int r = 0; r < N; ++r) {
+#pragma unroll
+                for (int v = 0; v < V; ++v) cur[r][v] = nxt[r][v];
+            }
+        }
+        wbase = nb;
+        if (++since == K1R_FLUSH) { flush(); since = 0; }
+    }
+    // ragged tail: the last d % V coordinates, one thread
+    if (V > 1 && blockIdx.x == 0 && tid == 0) {
+        for (int64_t t = nvec * V; t < d; ++t) {
+            float x[N];
+#pragma unroll
+            for (int r = 0; r < N; ++r) x[r] = __ldg(g + int64_t(r) * ld + t);
+            int p = 0;
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+#pragma unroll
+                for (int j = i + 1; j < N; ++j) { const float df = x[i] - x[j]; acc[p] = fmaf(df, df, acc[p]); ++p; }
+            }
+        }
+    }
+    __syncwarp();
+    flush();
+    __syncthreads();
+
+    double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
+    for (int i = tid; i < NP; i += K1R_THREADS) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) s += sums[w][i];
+        my_partial[i] = s;
+    }
+    if (!last_cta_ticket(ticket)) return;
+    reduce_partials(partials, NP, K1R_THREADS, [&](int p, double s) {
+        // pair index -> (i, j), pairs enumerated (0,1),(0,2),..,(0,N-1),(1,2),..
+        int i = 0, rem = p;
+        while (rem >= N - 1 - i) { rem -= N - 1 - i; ++i; }
+        const int j = i + 1 + rem;
+        dist[i * N + j] = s;
+        dist[j * N + i] = s;
+    });
+    for (int i = tid; i < N; i += K1R_THREADS) dist[i * N + i] = 0.0;
+    if (tid == 0) *ticket = 0u;               // ready for the next call
+}
+
+// ========================================================= tiled kernel, n > 16
+template <int NB> struct K1Shape;
+// G = column groups per CTA, KQ = float4 passes of an off-diagonal lane per slab,
+// FLUSH = slabs between fp64 flushes, NSTAGE = depth of the shared-memory ring
+template <> struct K1Shape<3> { static constexpr int G = 3, KQ = 1, FLUSH = 16, NSTAGE = 3; };
+template <> struct K1Shape<4> { static constexpr int G = 2, KQ = 2, FLUSH = 8, NSTAGE = 3; };
+template <> struct K1Shape<5> { static constexpr int G = 1, KQ = 2, FLUSH = 8, NSTAGE = 4; };
+template <> struct K1Shape<6> { static constexpr int G = 1, KQ = 4, FLUSH = 4, NSTAGE = 3; };
+template <> struct K1Shape<7> { static constexpr int G = 1, KQ = 4, FLUSH = 4, NSTAGE = 3; };
+template <> struct K1Shape<8> { static constexpr int G = 1, KQ = 2, FLUSH = 8, NSTAGE = 4; };
+
+template <int NB> struct K1Dims {
+    static constexpr int R       = NB * 8;                   // staged rows (zero padded)
+    static constexpr int OFFJ    = NB * (NB - 1) / 2;        // off-diagonal tiles, half-warp each
+    static constexpr int DIAGJ   = (NB + 1) / 2;             // pairs of diagonal tiles, half-warp each
+    static constexpr int OFFW    = (OFFJ + 1) / 2;           // warps of off-diagonal tiles per group
+    static constexpr int DIAGW   = (DIAGJ + 1) / 2;          // warps of diagonal-tile pairs per group
+    static constexpr int GW      = OFFW + DIAGW;             // warps per group
+    static constexpr int G       = K1Shape<NB>::G;
+    static constexpr int KQ      = K1Shape<NB>::KQ;
+    static constexpr int FLUSH   = K1Shape<NB>::FLUSH;
+    static constexpr int NSTAGE  = K1Shape<NB>::NSTAGE;
+    static constexpr int GQ      = 16 * KQ;                  // float4 columns per group per slab
+    static constexpr int TK4     = G * GQ;                   // float4 per row per slab
+    static constexpr int TK      = TK4 * 4;                  // coordinates per slab
+    static constexpr int THREADS = G * GW * 32;
+    static constexpr int TILES   = OFFJ + DIAGJ;             // tile t < OFFJ: off-diagonal
+    static constexpr size_t STAGE_BYTES = size_t(R) * TK * 4;
+    static constexpr size_t SUM_BYTES   = size_t(G) * TILES * 64 * sizeof(double);
+    static constexpr size_t SMEM_BYTES  = NSTAGE * STAGE_BYTES + SUM_BYTES;
+};
+
+__device__ __forceinline__ void off_tile_blocks(int p, int nb, int& I, int& J) {
+    // off-diagonal tiles enumerated row by row: (0,1),(0,2)..(0,nb-1),(1,2)..
+    int i = 0, rem = p;
+    while (rem >= nb - 1 - i) { rem -= nb - 1 - i; ++i; }
+    I = i; J = i + 1 + rem;
 }
 
 // Stage one slab (all R rows, TK columns from t0) into shared memory.
@@ -79,45 +267,55 @@ __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ 
     using D = K1Dims<NB>;
     if constexpr (VEC) {
         for (int idx = threadIdx.x; idx < D::R * D::TK4; idx += D::THREADS) {
-            int row = idx / D::TK4, c4 = idx - row * D::TK4;
-            int64_t col = t0 + 4 * int64_t(c4);
-            int64_t left = d - col;                       // valid coordinates from col
-            int bytes = (row < n && left > 0) ? (left >= 4 ? 16 : int(left) * 4) : 0;
+            const int row = idx / D::TK4, c4 = idx - row * D::TK4;
+            const int64_t col = t0 + 4 * int64_t(c4);
+            const int64_t left = d - col;                 // valid coordinates from col
+            const int bytes = (row < n && left > 0) ? (left >= 4 ? 16 : int(left) * 4) : 0;
             const float* src = bytes ? g + int64_t(row) * ld + col : g;
             cp_async16(sm + size_t(row) * D::TK + 4 * c4, src, bytes);
         }
     } else {
         for (int idx = threadIdx.x; idx < D::R * D::TK; idx += D::THREADS) {
-            int row = idx / D::TK, c = idx - row * D::TK;
-            int64_t col = t0 + c;
-            float v = (row < n && col < d) ? __ldg(g + int64_t(row) * ld + col) : 0.0f;
-            sm[size_t(row) * D::TK + c] = v;
+            const int row = idx / D::TK, c = idx - row * D::TK;
+            const int64_t col = t0 + c;
+            sm[size_t(row) * D::TK + c] = (row < n && col < d) ? __ldg(g + int64_t(row) * ld + col) : 0.0f;
         }
     }
 }
 
 template <int NB, bool VEC>
 __global__ void __launch_bounds__(K1Dims<NB>::THREADS)
-k1_distances(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
-             double* __restrict__ partials, unsigned int* __restrict__ ticket) {
+k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
+         double* __restrict__ partials, unsigned int* __restrict__ ticket) {
     using D = K1Dims<NB>;
     constexpr int NSTAGE = D::NSTAGE;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float*  stage = reinterpret_cast<float*>(smem_raw);
-    double* sums  = reinterpret_cast<double*>(smem_raw + NSTAGE * D::STAGE_BYTES);
-    __shared__ int is_last;
+    double* sums  = reinterpret_cast<double*>(smem_raw + NSTAGE * D::STAGE_BYTES);   // [G][TILES][64]
 
-    const int tid  = threadIdx.x;
-    const int slot = tid >> 3;                 // (group, tile) owner index
-    const int c    = tid & 7;                  // lane inside the owner
-    const bool active = slot < D::SLOTS;
-    const int grp  = active ? slot / D::TILES : 0;
-    const int p    = active ? slot - grp * D::TILES : 0;
-    int I, J;
-    tile_to_blocks(p, NB, D::OFF, I, J);
-    const bool diag = (p >= D::OFF);
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = tid >> 5;
+    const int grp = warp / D::GW, gw = warp - grp * D::GW;
+    const bool off_warp = gw < D::OFFW;
+    // a half-warp per job: an off-diagonal tile (I, J), or the diagonal tiles I and J = I + 1
+    int tile, I = 0, J = 0;
+    bool active;
+    const int c = lane & 15;
+    if (off_warp) {
+        const int job = gw * 2 + (lane >> 4);
+        active = job < D::OFFJ;
+        tile = active ? job : 0;
+        off_tile_blocks(tile, NB, I, J);
+    } else {
+        const int job = (gw - D::OFFW) * 2 + (lane >> 4);
+        active = job < D::DIAGJ;
+        I = active ? 2 * job : 0;
+        J = (I + 1 < NB) ? I + 1 : I;          // odd block count: the last job repeats its tile (ignored later)
+        tile = D::OFFJ + (active ? job : 0);
+    }
+    double* my_sums = sums + (size_t(grp) * D::TILES + tile) * 64;
 
-    for (int i = tid; i < D::SLOTS * 64; i += D::THREADS) sums[i] = 0.0;
+    for (int i = tid; i < D::G * D::TILES * 64; i += D::THREADS) sums[i] = 0.0;
     __syncthreads();
 
     float acc[64];
@@ -129,16 +327,14 @@ k1_distances(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* 
     const int64_t mine = first < nslabs ? (nslabs - first + step - 1) / step : 0;
 
     auto flush = [&]() {
-        // reduce each accumulator over the tile's 8 lanes, then lane (pair & 7) adds it in fp64
+        reduce_scatter<64, 16>(acc, lane);               // 4 totals per lane
+        const int b = scatter_base<64, 16>(lane);
+        if (active) {
 #pragma unroll
-        for (int i = 0; i < 64; ++i) {
-            float v = acc[i];
-            v += __shfl_xor_sync(0xffffffffu, v, 1);
-            v += __shfl_xor_sync(0xffffffffu, v, 2);
-            v += __shfl_xor_sync(0xffffffffu, v, 4);
-            if (active && (i & 7) == c) sums[slot * 64 + i] += double(v);
-            acc[i] = 0.0f;
+            for (int i = 0; i < 4; ++i) my_sums[b + i] += double(acc[i]);
         }
+#pragma unroll
+        for (int i = 0; i < 64; ++i) acc[i] = 0.0f;
     };
 
     if constexpr (VEC) {
@@ -150,11 +346,11 @@ k1_distances(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* 
 
     int since_flush = 0;
     for (int64_t it = 0; it < mine; ++it) {
-        float* cur;
+        const float* cur;
         if constexpr (VEC) {
             cp_async_wait<NSTAGE - 2>();
             __syncthreads();
-            int64_t nxt = it + NSTAGE - 1;
+            const int64_t nxt = it + NSTAGE - 1;
             if (nxt < mine)
                 stage_slab<NB, true>(stage + size_t(nxt % NSTAGE) * D::R * D::TK, g, n, d, ld, (first + nxt * step) * D::TK);
             cp_async_commit();
@@ -165,37 +361,56 @@ k1_distances(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* 
             __syncthreads();
             cur = stage;
         }
-
-        if (active) {
-            const float4* s4 = reinterpret_cast<const float4*>(cur);
+        const float4* s4 = reinterpret_cast<const float4*>(cur) + grp * D::GQ;
+        if (off_warp) {
+            const float4* pa = s4 + (I * 8) * D::TK4 + c;
+            const float4* pb = s4 + (J * 8) * D::TK4 + c;
 #pragma unroll
             for (int k = 0; k < D::KQ; ++k) {
-                const int q = k * D::LANES + grp * 8 + c;
                 float4 a[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) a[i] = s4[(I * 8 + i) * D::TK4 + q];
-                if (!diag) {
+                for (int i = 0; i < 8; ++i) a[i] = pa[i * D::TK4 + k * 16];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const float4 b = s4[(J * 8 + j) * D::TK4 + q];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            float dx = a[i].x - b.x, dy = a[i].y - b.y, dz = a[i].z - b.z, dw = a[i].w - b.w;
-                            float t = acc[i * 8 + j];
-                            t = fmaf(dx, dx, t); t = fmaf(dy, dy, t); t = fmaf(dz, dz, t); t = fmaf(dw, dw, t);
-                            acc[i * 8 + j] = t;
-                        }
-                    }
-                } else {
+                for (int j = 0; j < 8; ++j) {
+                    const float4 b = pb[j * D::TK4 + k * 16];
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
+                        const float dx = a[i].x - b.x, dy = a[i].y - b.y, dz = a[i].z - b.z, dw = a[i].w - b.w;
+                        float t = acc[i * 8 + j];
+                        t = fmaf(dx, dx, t); t = fmaf(dy, dy, t); t = fmaf(dz, dz, t); t = fmaf(dw, dw, t);
+                        acc[i * 8 + j] = t;
+                    }
+                }
+            }
+        } else {
+            // two diagonal tiles: pairs i < j of tile I at acc[i*8+j], of tile J at acc[j*8+i]
+            const float4* pa = s4 + (I * 8) * D::TK4 + c;
+            const float4* pb = s4 + (J * 8) * D::TK4 + c;
 #pragma unroll
-                        for (int j = i + 1; j < 8; ++j) {
-                            float dx = a[i].x - a[j].x, dy = a[i].y - a[j].y, dz = a[i].z - a[j].z, dw = a[i].w - a[j].w;
-                            float t = acc[i * 8 + j];
-                            t = fmaf(dx, dx, t); t = fmaf(dy, dy, t); t = fmaf(dz, dz, t); t = fmaf(dw, dw, t);
-                            acc[i * 8 + j] = t;
-                        }
+            for (int k = 0; k < D::KQ; ++k) {
+                float4 a[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a[i] = pa[i * D::TK4 + k * 16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+#pragma unroll
+                    for (int j = i + 1; j < 8; ++j) {
+                        const float dx = a[i].x - a[j].x, dy = a[i].y - a[j].y, dz = a[i].z - a[j].z, dw = a[i].w - a[j].w;
+                        float t = acc[i * 8 + j];
+                        t = fmaf(dx, dx, t); t = fmaf(dy, dy, t); t = fmaf(dz, dz, t); t = fmaf(dw, dw, t);
+                        acc[i * 8 + j] = t;
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a[i] = pb[i * D::TK4 + k * 16];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+#pragma unroll
+                    for (int j = i + 1; j < 8; ++j) {
+                        const float dx = a[i].x - a[j].x, dy = a[i].y - a[j].y, dz = a[i].z - a[j].z, dw = a[i].w - a[j].w;
+                        float t = acc[j * 8 + i];
+                        t = fmaf(dx, dx, t); t = fmaf(dy, dy, t); t = fmaf(dz, dz, t); t = fmaf(dw, dw, t);
+                        acc[j * 8 + i] = t;
                     }
                 }
             }
@@ -211,84 +426,130 @@ k1_distances(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* 
     for (int i = tid; i < D::TILES * 64; i += D::THREADS) {
         double s = 0.0;
 #pragma unroll 1
-        for (int gq = 0; gq < D::G; ++gq) s += sums[(gq * D::TILES + (i >> 6)) * 64 + (i & 63)];
+        for (int gq = 0; gq < D::G; ++gq) s += sums[size_t(gq) * D::TILES * 64 + i];
         my_partial[i] = s;
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        unsigned int t = atomicAdd(ticket, 1u);
-        is_last = (t == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-
-    // last CTA: add the partials in CTA order and write the symmetric matrix
-    for (int i = tid; i < D::TILES * 64; i += D::THREADS) {
-        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-        unsigned b = 0;
-        for (; b + 4 <= gridDim.x; b += 4) {
-            s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
-            s1 += __ldcg(partials + size_t(b + 1) * kPairSlots + i);
-            s2 += __ldcg(partials + size_t(b + 2) * kPairSlots + i);
-            s3 += __ldcg(partials + size_t(b + 3) * kPairSlots + i);
+    if (!last_cta_ticket(ticket)) return;
+    reduce_partials(partials, D::TILES * 64, D::THREADS, [&](int i, double s) {
+        const int t = i >> 6, hi = (i & 63) >> 3, lo = i & 7;
+        int ra, rb;
+        if (t < D::OFFJ) {
+            int bi, bj;
+            off_tile_blocks(t, NB, bi, bj);
+            ra = bi * 8 + hi;
+            rb = bj * 8 + lo;
+        } else if (hi < lo) {                      // first diagonal tile of the job
+            ra = 2 * (t - D::OFFJ) * 8 + hi;
+            rb = 2 * (t - D::OFFJ) * 8 + lo;
+        } else if (hi > lo && 2 * (t - D::OFFJ) + 1 < NB) {   // second one
+            ra = (2 * (t - D::OFFJ) + 1) * 8 + lo;
+            rb = (2 * (t - D::OFFJ) + 1) * 8 + hi;
+        } else {
+            ra = rb = n;                           // unused slot
         }
-        for (; b < gridDim.x; ++b) s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
-        const double s = (s0 + s1) + (s2 + s3);
-        int pi = i >> 6, pr = i & 63, bi, bj;
-        tile_to_blocks(pi, NB, D::OFF, bi, bj);
-        const int ra = bi * 8 + (pr >> 3), rb = bj * 8 + (pr & 7);
         if (ra < n && rb < n && ra < rb) {
             dist[ra * n + rb] = s;
             dist[rb * n + ra] = s;
         }
-    }
+    });
     for (int i = tid; i < n; i += D::THREADS) dist[i * n + i] = 0.0;
     if (tid == 0) *ticket = 0u;               // ready for the next call
 }
 
-template <int NB, bool VEC>
-cudaError_t launch_nb(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
-                      int sm_count, cudaStream_t stream) {
-    using D = K1Dims<NB>;
-    auto kern = k1_distances<NB, VEC>;
-    static int per_sm_cache[64] = {0};        // per device: 0 = not configured yet
+// ------------------------------------------------------------------ launchers
+template <typename K>
+cudaError_t persistent_grid(K kern, int threads, size_t smem, int sm_count, int* per_sm_cache, int64_t work_items,
+                            int64_t* grid_out) {
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     int per_sm = (dev >= 0 && dev < 64) ? per_sm_cache[dev] : 0;
     if (per_sm == 0) {
-        err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(D::SMEM_BYTES));
-        if (err != cudaSuccess) return err;
-        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, D::THREADS, D::SMEM_BYTES);
+        if (smem > 48 * 1024) {
+            err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+            if (err != cudaSuccess) return err;
+        }
+        err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
         if (err != cudaSuccess) return err;
         if (per_sm < 1) per_sm = 1;
         if (dev >= 0 && dev < 64) per_sm_cache[dev] = per_sm;
     }
-    int64_t nslabs = (d + D::TK - 1) / D::TK;
     int64_t grid = int64_t(sm_count) * per_sm;
     if (grid > kMaxCtasK1) grid = kMaxCtasK1;
-    if (grid > nslabs) grid = nslabs;
-    kern<<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket());
+    if (grid > work_items) grid = work_items;
+    if (grid < 1) grid = 1;
+    *grid_out = grid;
+    return cudaSuccess;
+}
+
+template <int NB, bool VEC>
+cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
+                         int sm_count, cudaStream_t stream) {
+    using D = K1Dims<NB>;
+    static int per_sm_cache[64] = {0};
+    int64_t grid = 1;
+    cudaError_t err = persistent_grid(k1_tiled<NB, VEC>, D::THREADS, D::SMEM_BYTES, sm_count, per_sm_cache,
+                                      (d + D::TK - 1) / D::TK, &grid);
+    if (err != cudaSuccess) return err;
+    k1_tiled<NB, VEC><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket());
     return cudaGetLastError();
+}
+
+template <int N, int V>
+cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
+                          cudaStream_t stream) {
+    static int per_sm_cache[64] = {0};
+    int64_t grid = 1;
+    const int64_t nvec = d / V > 0 ? d / V : 1;
+    cudaError_t err = persistent_grid(k1_direct<N, V>, K1R_THREADS, 0, sm_count, per_sm_cache,
+                                      (nvec + K1R_THREADS - 1) / K1R_THREADS, &grid);
+    if (err != cudaSuccess) return err;
+    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, 0, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket());
+    return cudaGetLastError();
+}
+
+template <int N>
+cudaError_t launch_direct_n(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
+                            cudaStream_t stream, int vec) {
+    // few rows: wide vectors keep enough bytes in flight; many rows: narrow ones keep the registers in check
+    if constexpr (N <= 8) {
+        if (vec >= 4) return launch_direct<N, 4>(g, d, ld, dist, ws, sm_count, stream);
+    }
+    if (vec >= 2) return launch_direct<N, 2>(g, d, ld, dist, ws, sm_count, stream);
+    return launch_direct<N, 1>(g, d, ld, dist, ws, sm_count, stream);
 }
 
 }  // namespace
 
 cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
                              const Workspace& ws, int sm_count, cudaStream_t stream) {
-    const bool vec = (reinterpret_cast<uintptr_t>(grads) % 16 == 0) && (ld % 4 == 0);
-    const int nb = (n + 7) / 8;
-#define GAR_K1_CASE(NBV)                                                                      \
-    case NBV:                                                                                 \
-        return vec ? launch_nb<NBV, true>(grads, n, d, ld, dist, ws, sm_count, stream)        \
-                   : launch_nb<NBV, false>(grads, n, d, ld, dist, ws, sm_count, stream);
-    switch (nb) {
-        GAR_K1_CASE(1) GAR_K1_CASE(2) GAR_K1_CASE(3) GAR_K1_CASE(4)
-        GAR_K1_CASE(5) GAR_K1_CASE(6) GAR_K1_CASE(7) GAR_K1_CASE(8)
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(grads);
+    int vec = 1;
+    if (addr % 16 == 0 && ld % 4 == 0) vec = 4;
+    else if (addr % 8 == 0 && ld % 2 == 0) vec = 2;
+    static const char* env = std::getenv("GAR_K1_VEC");   // tuning aid: cap the vector width
+    if (env) {
+        const int cap = std::atoi(env);
+        if ((cap == 1 || cap == 2) && n <= 16) vec = vec < cap ? vec : cap;
     }
-#undef GAR_K1_CASE
+    if (n == 1) return cudaMemsetAsync(dist, 0, sizeof(double), stream);
+#define GAR_K1_DIRECT(NV) case NV: return launch_direct_n<NV>(grads, d, ld, dist, ws, sm_count, stream, vec);
+#define GAR_K1_TILED(NBV)                                                                          \
+    case NBV:                                                                                      \
+        return vec == 4 ? launch_tiled<NBV, true>(grads, n, d, ld, dist, ws, sm_count, stream)      \
+                        : launch_tiled<NBV, false>(grads, n, d, ld, dist, ws, sm_count, stream);
+    if (n <= 16) {
+        switch (n) {
+            GAR_K1_DIRECT(2) GAR_K1_DIRECT(3) GAR_K1_DIRECT(4) GAR_K1_DIRECT(5) GAR_K1_DIRECT(6) GAR_K1_DIRECT(7)
+            GAR_K1_DIRECT(8) GAR_K1_DIRECT(9) GAR_K1_DIRECT(10) GAR_K1_DIRECT(11) GAR_K1_DIRECT(12)
+            GAR_K1_DIRECT(13) GAR_K1_DIRECT(14) GAR_K1_DIRECT(15) GAR_K1_DIRECT(16)
+        }
+    }
+    switch ((n + 7) / 8) {
+        GAR_K1_TILED(3) GAR_K1_TILED(4) GAR_K1_TILED(5) GAR_K1_TILED(6) GAR_K1_TILED(7) GAR_K1_TILED(8)
+    }
+#undef GAR_K1_DIRECT
+#undef GAR_K1_TILED
     return cudaErrorInvalidValue;
 }
 
