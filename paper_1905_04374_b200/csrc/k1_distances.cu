@@ -105,7 +105,23 @@ __device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) {
 // ======================================================== direct kernel, n <= 16
 constexpr int K1R_THREADS = 128;
 constexpr int K1R_FLUSH = 64;       // iterations between fp64 flushes
+constexpr int K1R_STAGES = 4;       // depth of the per-thread cp.async ring
 
+template <int BYTES>
+__device__ __forceinline__ void cp_async_small(void* smem_dst, const void* gsrc) {
+    unsigned s = static_cast<unsigned>(__cvta_generic_to_shared(smem_dst));
+    if constexpr (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gsrc) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], %2;\n" ::"r"(s), "l"(gsrc), "n"(BYTES) : "memory");
+}
+
+template <int N, int V> struct K1RDims {
+    static constexpr size_t RING_BYTES = size_t(K1R_STAGES) * N * K1R_THREADS * V * sizeof(float);
+};
+
+// Each thread owns V coordinates of all N rows per iteration.  The rows travel
+// through a ring of cp.async copies into shared-memory slots private to the
+// thread (K1R_STAGES - 1 iterations in flight, no barrier, no register staging),
+// so many bytes are in flight per SM while the registers hold the accumulators.
 template <int N, int V>
 __global__ void __launch_bounds__(K1R_THREADS)
 k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
@@ -114,6 +130,7 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     constexpr int NPAD = (NP + 31) / 32 * 32;
     constexpr int PER_LANE = NPAD / 32;
     constexpr int WARPS = K1R_THREADS / 32;
+    extern __shared__ __align__(16) float ring[];            // [stage][row][thread][V]
     __shared__ double sums[WARPS][NPAD];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int i = tid; i < WARPS * NPAD; i += K1R_THREADS) (&sums[0][0])[i] = 0.0;
@@ -131,22 +148,30 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
 #pragma unroll
         for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
     };
-    // rows of V coordinates at t; a lane past the end gets zeros (they add nothing)
-    auto load_rows = [&](float (&x)[N][V], int64_t t, bool valid) {
+    // request the rows of vector index vi into ring stage st (zeros past the end)
+    auto request = [&](int st, int64_t vi, bool valid) {
+        float* slot = ring + (size_t(st) * N * K1R_THREADS + tid) * V;
 #pragma unroll
         for (int r = 0; r < N; ++r) {
-            const float* p = g + int64_t(r) * ld + t;
+            float* dst = slot + size_t(r) * K1R_THREADS * V;
             if (valid) {
-                if constexpr (V == 4) { float4 q = __ldg(reinterpret_cast<const float4*>(p)); x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w; }
-                else if constexpr (V == 2) { float2 q = __ldg(reinterpret_cast<const float2*>(p)); x[r][0] = q.x; x[r][1] = q.y; }
-                else { x[r][0] = __ldg(p); }
+                cp_async_small<4 * V>(dst, g + int64_t(r) * ld + vi * V);
             } else {
 #pragma unroll
-                for (int v = 0; v < V; ++v) x[r][v] = 0.0f;
+                for (int v = 0; v < V; ++v) dst[v] = 0.0f;
             }
         }
     };
-    auto accumulate = [&](const float (&x)[N][V]) {
+    auto consume = [&](int st) {
+        const float* slot = ring + (size_t(st) * N * K1R_THREADS + tid) * V;
+        float x[N][V];
+#pragma unroll
+        for (int r = 0; r < N; ++r) {
+            const float* src = slot + size_t(r) * K1R_THREADS * V;
+            if constexpr (V == 4) { float4 q = *reinterpret_cast<const float4*>(src); x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w; }
+            else if constexpr (V == 2) { float2 q = *reinterpret_cast<const float2*>(src); x[r][0] = q.x; x[r][1] = q.y; }
+            else { x[r][0] = *src; }
+        }
         int p = 0;
 #pragma unroll
         for (int i = 0; i < N; ++i) {
@@ -164,24 +189,23 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     // the loop bound is per warp, so that the flush (warp-collective) is uniform
     const int64_t nvec = d / V;
     const int64_t stride = int64_t(gridDim.x) * K1R_THREADS;
-    int64_t wbase = int64_t(blockIdx.x) * K1R_THREADS + warp * 32;
-    float cur[N][V], nxt[N][V];
-    if (wbase < nvec) load_rows(cur, (wbase + lane) * V, wbase + lane < nvec);
+    const int64_t wfirst = int64_t(blockIdx.x) * K1R_THREADS + warp * 32;
+    const int64_t iters = wfirst < nvec ? (nvec - wfirst + stride - 1) / stride : 0;
+#pragma unroll
+    for (int s = 0; s < K1R_STAGES - 1; ++s) {
+        if (s < iters) { const int64_t vi = wfirst + s * stride + lane; request(s, vi, vi < nvec); }
+        cp_async_commit();
+    }
     int since = 0;
-    while (wbase < nvec) {
-        const int64_t nb = wbase + stride;
-        if (nb < nvec) load_rows(nxt, (nb + lane) * V, nb + lane < nvec);
-        accumulate(cur);
-        if (nb < nvec) {
-#pragma unroll
-            for (int r = 0; r < N; ++r) {
-#pragma unroll
-                for (int v = 0; v < V; ++v) cur[r][v] = nxt[r][v];
-            }
-        }
-        wbase = nb;
+    for (int64_t it = 0; it < iters; ++it) {
+        cp_async_wait<K1R_STAGES - 2>();
+        const int64_t nx = it + K1R_STAGES - 1;
+        if (nx < iters) { const int64_t vi = wfirst + nx * stride + lane; request(int(nx % K1R_STAGES), vi, vi < nvec); }
+        cp_async_commit();
+        consume(int(it % K1R_STAGES));
         if (++since == K1R_FLUSH) { flush(); since = 0; }
     }
+    cp_async_wait<0>();
     // ragged tail: the last d % V coordinates, one thread
     if (V > 1 && blockIdx.x == 0 && tid == 0) {
         for (int64_t t = nvec * V; t < d; ++t) {
@@ -224,7 +248,7 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
 template <int NB> struct K1Shape;
 // G = column groups per CTA, KQ = float4 passes of an off-diagonal lane per slab,
 // FLUSH = slabs between fp64 flushes, NSTAGE = depth of the shared-memory ring
-template <> struct K1Shape<3> { static constexpr int G = 3, KQ = 1, FLUSH = 16, NSTAGE = 3; };
+template <> struct K1Shape<3> { static constexpr int G = 2, KQ = 2, FLUSH = 8, NSTAGE = 3; };
 template <> struct K1Shape<4> { static constexpr int G = 2, KQ = 2, FLUSH = 8, NSTAGE = 3; };
 template <> struct K1Shape<5> { static constexpr int G = 1, KQ = 2, FLUSH = 8, NSTAGE = 4; };
 template <> struct K1Shape<6> { static constexpr int G = 1, KQ = 4, FLUSH = 4, NSTAGE = 3; };
@@ -250,6 +274,8 @@ template <int NB> struct K1Dims {
     static constexpr size_t STAGE_BYTES = size_t(R) * TK * 4;
     static constexpr size_t SUM_BYTES   = size_t(G) * TILES * 64 * sizeof(double);
     static constexpr size_t SMEM_BYTES  = NSTAGE * STAGE_BYTES + SUM_BYTES;
+    // two CTAs per SM where registers (<= 128 per thread) and shared memory allow it
+    static constexpr int MIN_CTAS = (THREADS <= 256 && SMEM_BYTES <= 110 * 1024) ? 2 : 1;
 };
 
 __device__ __forceinline__ void off_tile_blocks(int p, int nb, int& I, int& J) {
@@ -284,7 +310,7 @@ __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ 
 }
 
 template <int NB, bool VEC>
-__global__ void __launch_bounds__(K1Dims<NB>::THREADS)
+__global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
 k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
          double* __restrict__ partials, unsigned int* __restrict__ ticket) {
     using D = K1Dims<NB>;
@@ -365,8 +391,8 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
         if (off_warp) {
             const float4* pa = s4 + (I * 8) * D::TK4 + c;
             const float4* pb = s4 + (J * 8) * D::TK4 + c;
-#pragma unroll
-            for (int k = 0; k < D::KQ; ++k) {
+#pragma unroll 1
+            for (int k = 0; k < D::KQ; ++k) {          // rolled: the body is ~530 instructions already
                 float4 a[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) a[i] = pa[i * D::TK4 + k * 16];
@@ -386,7 +412,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
             // two diagonal tiles: pairs i < j of tile I at acc[i*8+j], of tile J at acc[j*8+i]
             const float4* pa = s4 + (I * 8) * D::TK4 + c;
             const float4* pb = s4 + (J * 8) * D::TK4 + c;
-#pragma unroll
+#pragma unroll 1
             for (int k = 0; k < D::KQ; ++k) {
                 float4 a[8];
 #pragma unroll
@@ -469,6 +495,11 @@ cudaError_t persistent_grid(K kern, int threads, size_t smem, int sm_count, int*
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
             if (err != cudaSuccess) return err;
         }
+        if (smem > 0) {   // let several CTAs of shared memory fit on an SM
+            err = cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                       cudaSharedmemCarveoutMaxShared);
+            if (err != cudaSuccess) return err;
+        }
         err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
         if (err != cudaSuccess) return err;
         if (per_sm < 1) per_sm = 1;
@@ -501,10 +532,11 @@ cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, c
     static int per_sm_cache[64] = {0};
     int64_t grid = 1;
     const int64_t nvec = d / V > 0 ? d / V : 1;
-    cudaError_t err = persistent_grid(k1_direct<N, V>, K1R_THREADS, 0, sm_count, per_sm_cache,
+    constexpr size_t smem = K1RDims<N, V>::RING_BYTES;
+    cudaError_t err = persistent_grid(k1_direct<N, V>, K1R_THREADS, smem, sm_count, per_sm_cache,
                                       (nvec + K1R_THREADS - 1) / K1R_THREADS, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, 0, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket());
+    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket());
     return cudaGetLastError();
 }
 

@@ -42,6 +42,9 @@ static cudaError_t run(const float* g, int n, int64_t d, int64_t ld, const gar_s
             err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, 1>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
             if (err != cudaSuccess) return err;
+            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, V>,
+                                       cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+            if (err != cudaSuccess) return err;
             if (dev >= 0 && dev < 64) configured[dev] = true;
         }
     }
