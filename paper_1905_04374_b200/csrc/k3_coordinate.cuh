@@ -19,7 +19,8 @@
 //    that is also loose (twice, the second time from L1).
 // The median is a Batcher odd-even merge network over registers, pruned at
 // compile time to the comparators the middle output depends on; the beta
-// closest values are found by beta passes of arg-min over |a - M|.
+// closest values are found from the beta-th smallest |a - M| (min/max only)
+// and 0/1 masks, with arg-min passes as the general fallback.
 //
 // P is the compiled slot count.  EXACT kernels have theta == P at compile time;
 // the others take theta <= P at run time: slots >= theta are padding that is
@@ -302,26 +303,71 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
                 key[s][v] = (s < theta) ? fabsf(a[s][v] - srt[(P - 1) / 2][v]) : CUDART_INF_F;
         }
 
-        // beta passes of arg-min; equal keys go to the earliest round = highest slot
+        // The beta smallest keys.  beta == 1: the minimum key, then one scan that keeps the
+        // value of the highest slot holding it.  beta == 2, 3: the beta-th smallest key tau is
+        // found with min/max only and the values with key <= tau are summed with a 0/1 mask; if
+        // more values tie at tau than there is room for, or for larger beta, beta passes of
+        // arg-min pick them one by one.  Equal keys go to the earliest round = highest slot.
         float sum[V];
-#pragma unroll
-        for (int v = 0; v < V; ++v) sum[v] = 0.0f;
-        for (int b = 0; b < beta; ++b) {
+        bool need_passes = beta > 3;
+        if (beta == 1) {
 #pragma unroll
             for (int v = 0; v < V; ++v) {
-                float best = key[P - 1][v], ba = a[P - 1][v];
-                int bi = P - 1;
+                float best = key[0][v];
 #pragma unroll
-                for (int s = P - 2; s >= 0; --s) {
-                    const bool take = key[s][v] < best;
-                    best = take ? key[s][v] : best;
-                    ba = take ? a[s][v] : ba;
-                    bi = take ? s : bi;
+                for (int s = 1; s < P; ++s) best = fminf(best, key[s][v]);
+                float ba = a[0][v];
+#pragma unroll
+                for (int s = 1; s < P; ++s) ba = (key[s][v] == best) ? a[s][v] : ba;
+                sum[v] = ba;
+            }
+        } else if (!need_passes) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                float t1 = CUDART_INF_F, t2 = CUDART_INF_F, t3 = CUDART_INF_F;   // three smallest keys so far
+#pragma unroll
+                for (int s = 0; s < P; ++s) {
+                    const float k = key[s][v];
+                    const float x = fmaxf(t1, k);
+                    t1 = fminf(t1, k);
+                    const float y = fmaxf(t2, x);
+                    t2 = fminf(t2, x);
+                    t3 = fminf(t3, y);
                 }
-                sum[v] += ba;
-                if (b + 1 < beta) {
+                const float tau = beta == 2 ? t2 : t3;
+                float s_le = 0.0f, c_le = 0.0f;
 #pragma unroll
-                    for (int s = 0; s < P; ++s) key[s][v] = (s == bi) ? CUDART_INF_F : key[s][v];
+                for (int s = 0; s < P; ++s) {
+                    const float le = key[s][v] <= tau ? 1.0f : 0.0f;
+                    s_le = fmaf(le, a[s][v], s_le);
+                    c_le += le;
+                }
+                sum[v] = s_le;
+                // c_le > beta: several keys tie at tau and not all of them fit
+                // (a non-finite tau or value also lands here)
+                if (!(c_le == float(beta)) || !(fabsf(s_le) <= 3.0e38f)) need_passes = true;
+            }
+        }
+        if (need_passes) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) sum[v] = 0.0f;
+            for (int b = 0; b < beta; ++b) {
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    float best = key[P - 1][v], ba = a[P - 1][v];
+                    int bi = P - 1;
+#pragma unroll
+                    for (int s = P - 2; s >= 0; --s) {
+                        const bool take = key[s][v] < best;
+                        best = take ? key[s][v] : best;
+                        ba = take ? a[s][v] : ba;
+                        bi = take ? s : bi;
+                    }
+                    sum[v] += ba;
+                    if (b + 1 < beta) {
+#pragma unroll
+                        for (int s = 0; s < P; ++s) key[s][v] = (s == bi) ? CUDART_INF_F : key[s][v];
+                    }
                 }
             }
         }

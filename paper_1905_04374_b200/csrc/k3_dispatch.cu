@@ -31,6 +31,7 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
     else if (a % 8 == 0 && ld % 2 == 0) vec = 2;
     // widest width that keeps the kernel's registers in check: large slot counts use narrower vectors
     if (vec == 4 && theta > 8) vec = 2;
+    if (vec == 2 && theta > (preagg ? 12 : 24)) vec = 1;
     static const char* env = std::getenv("GAR_K3_VEC");   // tuning aid: cap the vector width
     if (env) {
         const int cap = std::atoi(env);
