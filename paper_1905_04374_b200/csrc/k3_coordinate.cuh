@@ -65,6 +65,10 @@ template <int V> __device__ __forceinline__ void read_vec(const float* p, float 
     else { float4 t = *reinterpret_cast<const float4*>(p); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
 }
 
+__device__ __forceinline__ void prefetch_l1(const void* p) {
+    asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
+}
+
 __device__ __forceinline__ void cmpswap(float& lo, float& hi) {
     const float a = lo, b = hi;
     lo = fminf(a, b);
@@ -194,6 +198,22 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
             } else {
 #pragma unroll
                 for (int v = 0; v < V; ++v) e[s][v] = 0.0f;
+            }
+        }
+        // few slots: the kernel waits on memory more than it computes, so pull the next
+        // iteration's lines into L1 meanwhile (with many slots the extra instructions cost more)
+        const int64_t vnext = vi + int64_t(gridDim.x) * nthreads;
+        if (P <= 12 && vnext < nvec) {
+            const float* gn = g + t_begin + vnext * V;
+#pragma unroll
+            for (int s = 0; s < P; ++s) {
+                if (s < theta) prefetch_l1(gn + plan.woff[s]);
+            }
+            if constexpr (PREAGG) {
+                for (int k = 0; k < plan.nbase; ++k) prefetch_l1(gn + plan.boff[k]);
+                if (plan.loose_in_smem) {
+                    for (int k = 0; k < plan.nloose; ++k) prefetch_l1(gn + plan.loff[k]);
+                }
             }
         }
 
