@@ -231,8 +231,16 @@ def run_ours(args):
     }
     dom = "k1_distances" if k1_ms >= k3_ms else "k3_coordinate"
     achieved = kernels[dom]["gbs"]
+    # DRAM bytes per coordinate from the committed ncu captures (profiles/), taken on a smaller d of
+    # the same kernel and scaled by d; None where no capture of the current kernel exists
+    ncu_bytes_per_coord = {("k1_distances", 39): 316.5e6 / 2.0e6, ("k3_coordinate", 39): 240.6e6 / 2.0e6,
+                           ("k1_distances", 51): 310.0e6 / 1.5e6, ("k3_coordinate", 51): 302.3e6 / 1.5e6,
+                           ("k1_distances", 15): 244.4e6 / 4.0e6, ("k3_coordinate", 15): 172.0e6 / 4.0e6}
+    per_coord = ncu_bytes_per_coord.get((dom, n))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind, "traffic": None}
+                "frac": achieved / peak, "peak_kind": peak_kind,
+                "traffic": per_coord * d if per_coord else None,
+                "algorithmic_bytes": kernels[dom]["algorithmic_bytes"]}
     # whole-path effective bandwidth against the minimum traffic (n + theta + 1) * 4 d
     path_bytes_northstar = 4.0 * d * (n + theta_b + 1)
     path_bytes_own = 4.0 * d * (n + (rows_k3 if rows_k3 else theta_a) + 1)
