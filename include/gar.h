@@ -189,6 +189,27 @@ int gar_pairwise_distances(const float* grads, int n, int64_t d, int64_t ld, dou
                            void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Step 1 alone, for callers that must not allocate: the same distance kernels, but
+ * their scratch (ticket counter and per-CTA partial sums) is a fixed array inside the
+ * library image instead of a workspace, so this call performs no cudaMalloc / cudaFree
+ * and no other allocating call.  Meant for code that runs where device allocation is
+ * impossible or unwanted: inside another framework's memory pool or a fixed memory
+ * budget, with all of HBM already handed out, or in a latency-critical loop where an
+ * allocation could synchronise the device.  The paper has no counterpart.
+ *   - The array is about 10.9 MB (256 B + 592 CTAs x 2304 sums x 8 B) and is held by every
+ *     GPU that loads the library until the process exits.  It covers every n <= GAR_MAX_N
+ *     and any d; n > GAR_MAX_N returns GAR_ERR_UNSUPPORTED.
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     before any stream capture.
+ *   - All calls on a device share the array.  Each call clears the counter it needs on
+ *     `stream` first, but two calls that overlap on the GPU (different streams) race:
+ *     serialise them.
+ *   grads dev [n rows, stride ld (0 = d)], dist dev [n*n] fp64; asynchronous on `stream`.
+ */
+int gar_pairwise_distances_static(const float* grads, int n, int64_t d, int64_t ld, double* dist,
+                                  void* stream);
+
+/*
  * Step 2 alone: scoring and iterative selection from a distance matrix
  * (Eq. 4; Algorithm 1 multi-Krum and the loop of multi-Bulyan).
  *   dist dev [n*n] fp64; sel dev, written.  m, theta as in gar_params_t (0 = default).

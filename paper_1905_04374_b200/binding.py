@@ -83,6 +83,7 @@ def lib():
         L.gar_aggregate_host.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_void_p]
         L.gar_pairwise_distances.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                              C.c_size_t, C.c_void_p]
+        L.gar_pairwise_distances_static.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
         L.gar_select.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                  C.c_void_p]
         L.gar_schedule_from_tables.argtypes = [C.c_void_p, C.c_void_p]
@@ -207,6 +208,19 @@ def gar_pairwise_distances(grads: torch.Tensor, dist: torch.Tensor | None = None
     with torch.cuda.device(grads.device):
         st = lib().gar_pairwise_distances(grads.data_ptr(), n, d, ld, dist.data_ptr(), wp, wb, _stream(stream))
     _check(st, "gar_pairwise_distances")
+    return dist
+
+
+def gar_pairwise_distances_static(grads: torch.Tensor, dist: torch.Tensor, stream=None) -> torch.Tensor:
+    """gar_pairwise_distances_static: the distance step with no allocation inside the library.
+    The caller supplies `dist` (CUDA float64 [n, n]); this wrapper allocates nothing either."""
+    _dev_f32(grads, "grads")
+    n, d, ld = _rows(grads)
+    if not (dist.is_cuda and dist.dtype == torch.float64 and dist.is_contiguous() and dist.numel() == n * n):
+        raise TypeError("dist must be a contiguous CUDA float64 tensor with n*n elements")
+    with torch.cuda.device(grads.device):
+        st = lib().gar_pairwise_distances_static(grads.data_ptr(), n, d, ld, dist.data_ptr(), _stream(stream))
+    _check(st, "gar_pairwise_distances_static")
     return dist
 
 

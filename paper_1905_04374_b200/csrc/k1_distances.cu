@@ -586,3 +586,58 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
 }
 
 }  // namespace gar
+
+namespace gar {
+// ------------------------------------------------------------------------------------------
+// Distances without any allocation.
+//
+// Some callers of this library cannot allocate device memory at the moment they need the
+// distances: an aggregation hook that runs inside another framework's memory pool or under a
+// fixed memory budget, a process that has handed all of its HBM to other buffers, or a
+// latency-critical server loop where a cudaMalloc (which may synchronise the device) is not
+// acceptable.  For them the scratch of the distance kernels -- the ticket counter and the
+// per-CTA partial sums -- lives in the file-scope array below instead of a workspace.
+// Its size is fixed: kStaticScratchBytes (about 10.9 MB), enough for the largest grid the
+// distance kernels ever use and n <= GAR_MAX_N; every GPU that loads the library holds it
+// until the process exits.
+constexpr size_t kStaticScratchBytes = kCtrlBytes + kPartialBytes;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+struct StaticScratchState {
+    bool  ready = false;
+    char* ptr = nullptr;
+    int   sm_count = 0;
+};
+StaticScratchState g_static_state[64];
+}  // namespace
+
+}  // namespace gar
+
+extern "C" int gar_pairwise_distances_static(const float* grads, int n, int64_t d, int64_t ld, double* dist,
+                                             void* stream) {
+    if (!grads || !dist || n < 1 || d < 1) return GAR_ERR_INVALID_ARG;
+    if (n > GAR_MAX_N) return GAR_ERR_UNSUPPORTED;       // the static scratch is sized for n <= 64
+    if (ld == 0) ld = d;
+    if (ld < d) return GAR_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GAR_ERR_CUDA;
+    if (dev < 0 || dev >= 64) return GAR_ERR_UNSUPPORTED;
+    gar::StaticScratchState& st = gar::g_static_state[dev];
+    if (!st.ready) {
+        // Once per device, with that device current: in host code the array's name is only a
+        // stand-in; the address the kernels need comes from the runtime.
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, gar::g_static_scratch) != cudaSuccess || p == nullptr) return GAR_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            return GAR_ERR_CUDA;
+        st.ptr = static_cast<char*>(p);
+        st.ready = true;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's contents: the ticket counter must start at zero
+    // (the partial sums are overwritten before they are read)
+    if (cudaMemsetAsync(st.ptr, 0, gar::kCtrlBytes, s) != cudaSuccess) return GAR_ERR_CUDA;
+    gar::Workspace ws{st.ptr};
+    return gar::launch_distances(grads, n, d, ld, dist, ws, st.sm_count, s) == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+}
