@@ -158,6 +158,17 @@ def event_time_ms(fn, reps, stream):
     return start.elapsed_time(stop) / reps
 
 
+def max_over_ranks(elapsed_ms: float, world: int, device=None) -> float:
+    """Slowest rank's time (every rank must call it): the job is only as fast as that rank."""
+    if world <= 1:
+        return elapsed_ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -196,11 +207,9 @@ def run_ours(args):
         stop.record(stream)
         torch.cuda.synchronize()
     elapsed_ms = start.elapsed_time(stop)
+    elapsed_ms = max_over_ranks(elapsed_ms, world, dev)
     if world > 1:
-        t = torch.tensor([elapsed_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-        elapsed_ms = float(t.item())
     ms_per_step = elapsed_ms / args.steps
     value = world * args.steps / (elapsed_ms * 1e-3)
 
