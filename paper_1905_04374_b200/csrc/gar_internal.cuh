@@ -41,6 +41,11 @@ struct Workspace {
 cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
                              const Workspace& ws, int sm_count, cudaStream_t stream);
 
+// Tensor-core variant (16 < n <= 64, 16-byte aligned rows), used from kMmaMinDim coordinates on.
+constexpr int64_t kMmaMinDim = 32768;
+cudaError_t launch_distances_mma(const float* grads, int n, int64_t d, int64_t ld, double* dist,
+                                 const Workspace& ws, int sm_count, cudaStream_t stream);
+
 // Scoring + iterative selection (and schedule construction) into *sel.
 cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,
                           int median_of_agr, gar_selection_t* sel, cudaStream_t stream);
