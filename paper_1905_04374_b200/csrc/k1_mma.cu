@@ -27,8 +27,8 @@
 // ring needs no barrier), then reduces the row's
 // maximum with redux.sync, grows the row's exponent if needed (a row has a single
 // owner, so no agreement between warps is required), quantises, transposes the limb
-// bytes with prmt and stores three int8 limb tiles (row stride 36 words:
-// conflict-free fragment loads) into one of two buffers.  Eight consumer warps
+// bytes with prmt and stores three row-major int8 limb tiles (row stride 36 words:
+// conflict-free ldmatrix rows) into one of two buffers.  Eight consumer warps
 // issue the MMAs: warp (r, half) owns row tile r (16 rows) and MT column tiles
 // (8 columns each); tiles on or above the diagonal compute all six products, tiles
 // below it the three non-symmetric ones.  The consumers hold up to 96 int32
@@ -46,7 +46,7 @@ constexpr int K1M_THREADS = 512;
 constexpr int K1M_PRODUCERS = 8;        // warps 0..7
 constexpr int K1M_CONSUMERS = 8;        // warps 8..15
 constexpr int K1M_SLAB = 128;           // columns per slab (one float4 per lane)
-constexpr int K1M_STRIDE = 36;          // words per limb-tile row (32 + 4 padding)
+constexpr int K1M_STRIDE = 36;          // words per limb-tile row (32 + 4 padding: conflict-free ldmatrix rows)
 constexpr int K1M_FLUSH = 32;           // slabs between int32 -> fp64 flushes (|sum| < 2^27)
 constexpr int K1M_MIN_EXP = 21;         // smallest row exponent (keeps the scale a normal float)
 constexpr int K1M_PRODUCER_REGS = 96;    // per thread after setmaxnreg: 256 x 96 + 256 x 160 = 64 K registers
@@ -95,6 +95,11 @@ template <int MT> struct K1MRing {
     static constexpr size_t BYTES = size_t(STAGES) * MT * 16 * 32 * sizeof(float4);
 };
 
+__device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], unsigned smem_addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr));
+}
+
 __device__ __forceinline__ void bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void bar_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
@@ -135,18 +140,23 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
         int row_exp[JR];
 #pragma unroll
         for (int jr = 0; jr < JR; ++jr) row_exp[jr] = K1M_MIN_EXP;
+        const int wpos = lane;                         // this lane's word: columns 4*lane .. 4*lane+3 of the slab
         // cp.async of this lane's float4 of every owned row of a slab into ring stage st
+        const float* rowp[JR];                         // this lane's first float4 of every owned row
+#pragma unroll
+        for (int jr = 0; jr < JR; ++jr) {
+            const int row = warp + jr * K1M_PRODUCERS;
+            rowp[jr] = g + int64_t(row < n ? row : 0) * ld + 4 * lane;
+        }
         auto request = [&](int st, int64_t slab) {
-            const int64_t t = slab * K1M_SLAB + 4 * lane;
-            const int64_t left = d - t;
+            const int64_t t0 = slab * K1M_SLAB;
+            const int64_t left = d - t0 - 4 * lane;
             const int bytes = left >= 4 ? 16 : (left > 0 ? int(left) * 4 : 0);
+            float4* dst = ring + size_t(st) * ROWS * 32 + warp * 32 + lane;
 #pragma unroll
             for (int jr = 0; jr < JR; ++jr) {
                 const int row = warp + jr * K1M_PRODUCERS;
-                if (row < n) {
-                    const float* src = bytes ? g + int64_t(row) * ld + t : g;
-                    cp_async16(&ring[(size_t(st) * ROWS + row) * 32 + lane], src, bytes);
-                }
+                if (row < n) cp_async16(dst + jr * K1M_PRODUCERS * 32, bytes ? rowp[jr] + t0 : g, bytes);
             }
         };
 #pragma unroll
@@ -174,45 +184,56 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
             }
 #pragma unroll
             for (int jr = 0; jr < JR; ++jr) {
-                // |x| as integers: the order of non-negative floats is the order of their bit patterns,
-                // and a NaN (above 0x7f800000) also ends up with exponent 255
-                const unsigned m = max(max(__float_as_uint(v[jr].x) & 0x7fffffffu, __float_as_uint(v[jr].y) & 0x7fffffffu),
-                                       max(__float_as_uint(v[jr].z) & 0x7fffffffu, __float_as_uint(v[jr].w) & 0x7fffffffu));
-                ex[jr] = int(__reduce_max_sync(0xffffffffu, m) >> 23);
+                const float m = fmaxf(fmaxf(fabsf(v[jr].x), fabsf(v[jr].y)), fmaxf(fabsf(v[jr].z), fabsf(v[jr].w)));
+                // x - x is 0 for finite x and NaN otherwise: one flag for "some value is Inf or NaN"
+                const float nf = ((v[jr].x - v[jr].x) + (v[jr].y - v[jr].y)) + ((v[jr].z - v[jr].z) + (v[jr].w - v[jr].w));
+                const unsigned mb = (nf != nf) ? 0x7f800000u : __float_as_uint(m);
+                ex[jr] = int(__reduce_max_sync(0xffffffffu, mb) >> 23);
             }
-            // phase 2: exponents, quantisation, limb tiles
-            bool grew = false;
+            // phase 2: exponents (branch-free), then quantisation, limb split and stores stage by
+            // stage over all owned rows, so that the rows' dependent chains overlap
+            bool grew = false, any_bad = false;
+            float scale[JR];
 #pragma unroll
             for (int jr = 0; jr < JR; ++jr) {
-                const int row = warp + jr * K1M_PRODUCERS;
-                if (row < n) {
-                    const bool bad = ex[jr] == 255;
-                    if (bad) {
-                        if (lane == 0) {
+                const bool bad = ex[jr] == 255;
+                const bool up = !bad && ex[jr] > row_exp[jr];
+                row_exp[jr] = up ? ex[jr] + 1 : row_exp[jr];               // one binade of headroom
+                grew |= up;
+                any_bad |= bad;
+                scale[jr] = __uint_as_float(unsigned(275 - row_exp[jr]) << 23);   // 2^(148-E)
+            }
+            if (any_bad) {                                                   // rare: a row holds Inf or NaN
+#pragma unroll
+                for (int jr = 0; jr < JR; ++jr) {
+                    const int row = warp + jr * K1M_PRODUCERS;
+                    if (ex[jr] == 255) {
+                        v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);            // quantised as zeros, flagged
+                        if (lane == 0 && row < n) {
                             if (row < 32) atomicOr(&sm.nonfinite_lo, 1u << row); else atomicOr(&sm.nonfinite_hi, 1u << (row - 32));
                         }
-                    } else if (ex[jr] > row_exp[jr]) {
-                        row_exp[jr] = ex[jr] + 1;                           // one binade of headroom
-                        grew = true;
                     }
-                    const int E = row_exp[jr];
-                    const float scale = bad ? 0.0f : __uint_as_float(unsigned(275 - E) << 23);   // 2^(148-E)
-                    const float xs[4] = {bad ? 0.0f : v[jr].x, bad ? 0.0f : v[jr].y, bad ? 0.0f : v[jr].z, bad ? 0.0f : v[jr].w};
-                    unsigned w[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        // round to nearest integer through the 1.5 * 2^23 trick; the low three bytes of
-                        // (q + 0x808080) ^ 0x808080 are the signed limbs l3, l2, l1
-                        const float t = fmaf(xs[k], scale, 12582912.0f);
-                        w[k] = (__float_as_uint(t) + (0x00808080u - 0x4B400000u)) ^ 0x00808080u;
-                    }
-                    const unsigned p01 = prmt(w[0], w[1], 0x5140u), p23 = prmt(w[2], w[3], 0x5140u);
-                    const unsigned h01 = prmt(w[0], w[1], 0x0062u), h23 = prmt(w[2], w[3], 0x0062u);
-                    sm.limb[buf][2][row][lane] = prmt(p01, p23, 0x5410u);   // l3
-                    sm.limb[buf][1][row][lane] = prmt(p01, p23, 0x7632u);   // l2
-                    sm.limb[buf][0][row][lane] = prmt(h01, h23, 0x5410u);   // l1
-                    if (lane == 0) sm.slab_exp[buf][row] = E;
                 }
+            }
+            unsigned w[JR][4];
+#pragma unroll
+            for (int jr = 0; jr < JR; ++jr) {
+                // round to nearest integer through the 1.5 * 2^23 trick; the low three bytes of
+                // (q + 0x808080), each xor 0x80, are the signed limbs l3, l2, l1
+                w[jr][0] = __float_as_uint(fmaf(v[jr].x, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                w[jr][1] = __float_as_uint(fmaf(v[jr].y, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                w[jr][2] = __float_as_uint(fmaf(v[jr].z, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                w[jr][3] = __float_as_uint(fmaf(v[jr].w, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+            }
+#pragma unroll
+            for (int jr = 0; jr < JR; ++jr) {
+                const int row = warp + jr * K1M_PRODUCERS;                  // rows >= n hold zeros: harmless stores
+                const unsigned p01 = prmt(w[jr][0], w[jr][1], 0x5140u), p23 = prmt(w[jr][2], w[jr][3], 0x5140u);
+                const unsigned h01 = prmt(w[jr][0], w[jr][1], 0x0062u), h23 = prmt(w[jr][2], w[jr][3], 0x0062u);
+                sm.limb[buf][2][row][wpos] = prmt(p01, p23, 0x5410u) ^ 0x80808080u;   // l3
+                sm.limb[buf][1][row][wpos] = prmt(p01, p23, 0x7632u) ^ 0x80808080u;   // l2
+                sm.limb[buf][0][row][wpos] = prmt(h01, h23, 0x5410u) ^ 0x80808080u;   // l1
+                if (lane == 0) sm.slab_exp[buf][row] = row_exp[jr];
             }
             if (grew && lane == 0) sm.grow[buf] = 1;
             __threadfence_block();
@@ -275,28 +296,44 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
                 bar_sync(BAR_CONS, K1M_CONSUMERS * 32);
             }
             if (mma_warp) {
+                // ldmatrix addresses: lane l supplies the 16-byte row (l % 8) of matrix l / 8.
+                // A (16 rows x 32 bytes): matrices (rows 0-7, bytes 0-15), (rows 8-15, 0-15), (rows 0-7, 16-31),
+                // (rows 8-15, 16-31) = a0..a3.  B for two column tiles: (tile, bytes 0-15), (tile, 16-31),
+                // (tile+1, 0-15), (tile+1, 16-31) = b0, b1 of the first tile, b0, b1 of the second.
+                const int lrow = lane & 7, lmat = lane >> 3;
+                const unsigned a_off = unsigned(((rt * 16 + lrow + (lmat & 1) * 8) * K1M_STRIDE + (lmat >> 1) * 4) * 4);
+                const unsigned b_off = unsigned((((half * MT + (lmat >> 1)) * 8 + lrow) * K1M_STRIDE + (lmat & 1) * 4) * 4);
+                const unsigned tile0 = static_cast<unsigned>(__cvta_generic_to_shared(&sm.limb[buf][0][0][0]));
+                constexpr unsigned LIMB_BYTES = 64 * K1M_STRIDE * 4;
 #pragma unroll 1
                 for (int ks = 0; ks < 4; ++ks) {
-                    unsigned a1[4], a2[4], a3[4];
-                    const int ar = rt * 16 + gq, kw = ks * 8 + cq;
-                    a1[0] = sm.limb[buf][0][ar][kw]; a1[1] = sm.limb[buf][0][ar + 8][kw]; a1[2] = sm.limb[buf][0][ar][kw + 4]; a1[3] = sm.limb[buf][0][ar + 8][kw + 4];
-                    a2[0] = sm.limb[buf][1][ar][kw]; a2[1] = sm.limb[buf][1][ar + 8][kw]; a2[2] = sm.limb[buf][1][ar][kw + 4]; a2[3] = sm.limb[buf][1][ar + 8][kw + 4];
-                    a3[0] = sm.limb[buf][2][ar][kw]; a3[1] = sm.limb[buf][2][ar + 8][kw]; a3[2] = sm.limb[buf][2][ar][kw + 4]; a3[3] = sm.limb[buf][2][ar + 8][kw + 4];
+                    const unsigned kb = ks * 32;                              // 32 bytes of every row per k-step
+                    unsigned af[3][4];
 #pragma unroll
-                    for (int a = 0; a < MT; ++a) {
-                        const int ct = half * MT + a;
-                        const int br = ct * 8 + gq;
-                        unsigned b1[2], b2[2], b3[2];
-                        b1[0] = sm.limb[buf][0][br][kw]; b1[1] = sm.limb[buf][0][br][kw + 4];
-                        b2[0] = sm.limb[buf][1][br][kw]; b2[1] = sm.limb[buf][1][br][kw + 4];
-                        mma_s8(acc[a][1], a2, b1);               // L2 L1^T
-                        mma_s8(acc[a][2], a3, b1);               // L3 L1^T
-                        mma_s8(acc[a][4], a3, b2);               // L3 L2^T
-                        if (ct >= 2 * rt) {                      // on or above the diagonal (warp-uniform)
-                            b3[0] = sm.limb[buf][2][br][kw]; b3[1] = sm.limb[buf][2][br][kw + 4];
-                            mma_s8(acc[a][0], a1, b1);           // L1 L1^T
-                            mma_s8(acc[a][3], a2, b2);           // L2 L2^T
-                            mma_s8(acc[a][5], a3, b3);           // L3 L3^T
+                    for (int l = 0; l < 3; ++l) ldmatrix_x4(af[l], tile0 + l * LIMB_BYTES + a_off + kb);
+#pragma unroll
+                    for (int a2 = 0; a2 < MT; a2 += 2) {
+                        unsigned bf[3][4];                                    // [limb][b0, b1 of tile a2; b0, b1 of tile a2+1]
+#pragma unroll
+                        for (int l = 0; l < 3; ++l)
+                            ldmatrix_x4(bf[l], tile0 + l * LIMB_BYTES + b_off + unsigned(a2 * 8 * K1M_STRIDE * 4) + kb);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int a = a2 + h;
+                            if (a < MT) {
+                                const int ct = half * MT + a;
+                                const unsigned (&b1)[2] = *reinterpret_cast<const unsigned (*)[2]>(&bf[0][2 * h]);
+                                const unsigned (&b2)[2] = *reinterpret_cast<const unsigned (*)[2]>(&bf[1][2 * h]);
+                                const unsigned (&b3)[2] = *reinterpret_cast<const unsigned (*)[2]>(&bf[2][2 * h]);
+                                mma_s8(acc[a][1], af[1], b1);            // L2 L1^T
+                                mma_s8(acc[a][2], af[2], b1);            // L3 L1^T
+                                mma_s8(acc[a][4], af[2], b2);            // L3 L2^T
+                                if (ct >= 2 * rt) {                      // on or above the diagonal (warp-uniform)
+                                    mma_s8(acc[a][0], af[0], b1);        // L1 L1^T
+                                    mma_s8(acc[a][3], af[1], b2);        // L2 L2^T
+                                    mma_s8(acc[a][5], af[2], b3);        // L3 L3^T
+                                }
+                            }
                         }
                     }
                 }
