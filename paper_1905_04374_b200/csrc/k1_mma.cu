@@ -51,6 +51,7 @@ constexpr int K1M_FLUSH = 32;           // slabs between int32 -> fp64 flushes (
 constexpr int K1M_MIN_EXP = 21;         // smallest row exponent (keeps the scale a normal float)
 constexpr int K1M_PRODUCER_REGS = 96;    // per thread after setmaxnreg: 256 x 96 + 256 x 160 = 64 K registers
 constexpr int K1M_CONSUMER_REGS = 160;
+constexpr int K1M_LAUNCH_REGS = 128;     // 64 K registers / 512 threads
 constexpr int K1M_TRI = 2080;           // entries (i <= j) of a 64 x 64 matrix
 
 // named barriers (0 is __syncthreads)
@@ -61,7 +62,7 @@ constexpr int BAR_CONS = 5;             // consumers only
 // followed in shared memory by the raw ring: float4 [stages][rows][32 lanes]
 struct K1MSmem {
     unsigned limb[2][3][64][K1M_STRIDE]; // [buffer][limb: 0 = l1 (most significant)][row][4 columns per word]
-    double   px[K1M_TRI];                // 2^32 L1L1^T + 2^16 L2L2^T + L3L3^T       (row <= col, triangular index)
+    double   px[64][64];                 // 2^32 L1L1^T + 2^16 L2L2^T + L3L3^T       (tiles on or above the diagonal)
     double   py[64][64];                 // 2^24 L2L1^T + 2^16 L3L1^T + 2^8 L3L2^T   (all entries)
     int      slab_exp[2][64];            // exponent E each row of the buffer was quantised with
     int      cons_exp[64];               // exponents of the consumers' running int32 sums
@@ -100,8 +101,16 @@ __device__ __forceinline__ void ldmatrix_x4(unsigned (&r)[4], unsigned smem_addr
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_addr));
 }
 
-__device__ __forceinline__ void bar_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-__device__ __forceinline__ void bar_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+// The aligned barrier, ldmatrix and mma forms need the whole warp at the instruction together:
+// reconverge after any lane-dependent branch before a barrier.
+__device__ __forceinline__ void bar_sync(int id, int count) {
+    __syncwarp();
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive(int id, int count) {
+    __syncwarp();
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 
 __device__ __forceinline__ double pow2(int e) {      // 2^e as a double, -1022 <= e <= 1023
     return __hiloint2double((1023 + e) << 20, 0);
@@ -123,7 +132,7 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
     float4* ring = reinterpret_cast<float4*>(smem_raw + sizeof(K1MSmem));   // [NST][ROWS][32]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    for (int i = tid; i < K1M_TRI; i += K1M_THREADS) sm.px[i] = 0.0;
+    for (int i = tid; i < 64 * 64; i += K1M_THREADS) (&sm.px[0][0])[i] = 0.0;
     for (int i = tid; i < 64 * 64; i += K1M_THREADS) (&sm.py[0][0])[i] = 0.0;
     for (int i = tid; i < 2 * 3 * 64 * K1M_STRIDE; i += K1M_THREADS) (&sm.limb[0][0][0][0])[i] = 0u;
     if (tid < 64) { sm.cons_exp[tid] = K1M_MIN_EXP; sm.slab_exp[0][tid] = K1M_MIN_EXP; sm.slab_exp[1][tid] = K1M_MIN_EXP; }
@@ -240,12 +249,15 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
             bar_arrive(BAR_FULL + buf, K1M_THREADS);
         }
         cp_async_wait<0>();
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(K1M_LAUNCH_REGS));   // waits for the consumers' release
     } else {
         // ================================================================ consumers
         const int cw = warp - K1M_PRODUCERS;                  // 0..7
         const int ctid = tid - K1M_PRODUCERS * 32;            // 0..255
         const bool mma_warp = cw < 2 * MT;
-        const int rt = cw % MT, half = cw / MT;
+        constexpr unsigned kRoles = MT == 2 ? 0x00003210u : (MT == 3 ? 0x00243150u : 0x72645310u);
+        const int role = int((kRoles >> (4 * cw)) & 15u);
+        const int rt = role >> 1, half = role & 1;
         const int gq = lane >> 2, cq = lane & 3;
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(K1M_CONSUMER_REGS));
         int acc[MT][6][4];                                    // [column tile][11, 21, 31, 22, 32, 33][fragment]
@@ -271,10 +283,10 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
                         // exact: |sums| < 2^27, so every bracket fits a double's 53 bits
                         const double y = ((double(acc[a][1][k]) * 256.0 + double(acc[a][2][k])) * 256.0 + double(acc[a][4][k])) * pow2(e + 8);
                         sm.py[i][j] += y;
-                        if (upper && i <= j) {
-                            const double x = double(acc[a][0][k]) * pow2(e + 32) +
+                        if (upper) {                                       // warp-uniform; entries below the diagonal of a
+                            const double x = double(acc[a][0][k]) * pow2(e + 32) +   // diagonal tile are kept but never read
                                              (double(acc[a][3][k]) * 65536.0 + double(acc[a][5][k])) * pow2(e);
-                            sm.px[tri_slot(i, j)] += x;
+                            sm.px[i][j] += x;
                         }
 #pragma unroll
                         for (int p = 0; p < 6; ++p) acc[a][p][k] = 0;
@@ -287,9 +299,12 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
         for (int64_t it = 0; it < mine; ++it) {
             const int buf = int(it & 1);
             bar_sync(BAR_FULL + buf, K1M_THREADS);                         // the buffer's limb tiles are written
-            if (sm.grow[buf]) {                                            // uniform: the scales change
+            const bool grow = sm.grow[buf] != 0;                           // uniform: the scales change
+            if (grow || since_flush == K1M_FLUSH) {                        // the one flush site of the loop
                 flush();
                 since_flush = 0;
+            }
+            if (grow) {
                 bar_sync(BAR_CONS, K1M_CONSUMERS * 32);
                 if (ctid < 64) sm.cons_exp[ctid] = sm.slab_exp[buf][ctid];
                 if (ctid == 0) sm.grow[buf] = 0;
@@ -339,9 +354,10 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
                 }
             }
             if (it + 2 < mine) bar_arrive(BAR_EMPTY + buf, K1M_THREADS);   // hand the buffer back
-            if (++since_flush == K1M_FLUSH) { flush(); since_flush = 0; }
+            ++since_flush;
         }
         flush();
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(K1M_LAUNCH_REGS));   // back to the launch allocation
     }
     __syncthreads();
 
@@ -350,7 +366,7 @@ k1_mma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __rest
     double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
     for (int idx = tid; idx < 64 * 64; idx += K1M_THREADS) {
         const int i = idx >> 6, j = idx & 63;
-        if (i <= j) my_partial[tri_slot(i, j)] = sm.px[tri_slot(i, j)] + (sm.py[i][j] + sm.py[j][i]);
+        if (i <= j) my_partial[tri_slot(i, j)] = sm.px[i][j] + (sm.py[i][j] + sm.py[j][i]);
     }
     if (tid == 0) { my_partial[2300] = double(sm.nonfinite_lo); my_partial[2301] = double(sm.nonfinite_hi); }
 

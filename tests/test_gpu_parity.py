@@ -81,6 +81,75 @@ def test_distances_nonfinite_rows(pkg):
     assert_outputs_match(out, want)
 
 
+# The distance kernel for 16 < n <= 64, 16-byte-aligned rows and d >= 32768 forms the Gram matrix
+# from exact integer limbs; the cases below reach it (the ones above mostly stop short of it).
+@pytest.mark.parametrize("n", [17, 24, 25, 31, 32, 33, 40, 41, 47, 48, 49, 56, 57, 63, 64])
+def test_distances_large_d_every_row_count(pkg, n):
+    d = 33_000 + 4 * n
+    G = pkg.workloads.make_uniform(n, d, device=DEV, seed=100 + n)
+    G -= 0.5
+    D = pkg.gar_pairwise_distances(G).cpu().numpy()
+    want = O.pairwise_sq_distances(G.cpu().numpy())
+    np.testing.assert_allclose(D, want, rtol=1e-6, atol=0)
+    assert np.array_equal(D, D.T) and np.all(np.diag(D) == 0)
+
+
+@pytest.mark.parametrize("n", [23, 39, 51])
+@pytest.mark.parametrize("where", ["first", "middle", "late", "everywhere"])
+def test_distances_exact_on_small_integers(pkg, n, where):
+    """Rows of small integers, non-zero only in one band of columns: the squared distances are
+    integers below 2^53 and every summation order gives them exactly, so any contribution that is
+    dropped, doubled or filed under the wrong pair shows."""
+    d = 148 * 128 * 70 + 8
+    cols = torch.arange(d, device=DEV)
+    band = {"first": cols < 148 * 128, "middle": (cols >= 148 * 128 * 20) & (cols < 148 * 128 * 21),
+            "late": cols >= 148 * 128 * 69, "everywhere": cols >= 0}[where]
+    c = torch.arange(1, n + 1, dtype=torch.float32, device=DEV)[:, None]
+    sign = torch.where(cols % 3 == 0, -1.0, 1.0)[None, :]
+    G = (c * sign) * band[None, :].to(torch.float32)
+    G[n // 2] *= -1.0
+    D = pkg.gar_pairwise_distances(G).cpu().numpy()
+    want = O.pairwise_sq_distances(G.cpu().numpy())
+    assert want.max() < 2.0 ** 53
+    assert np.array_equal(D, want)
+
+
+@pytest.mark.parametrize("n", [23, 39, 51])
+def test_distances_growing_magnitudes(pkg, n):
+    """The magnitude of every row doubles a dozen times along the columns, at a different place
+    for every row: running sums are rescaled again and again while they are non-zero."""
+    d = 1_200_004
+    G = pkg.workloads.make_uniform(n, d, device=DEV, seed=7 * n) - 0.5
+    cols = torch.arange(d, device=DEV)
+    for i in range(n):
+        G[i] *= torch.exp2(torch.floor(cols * (12.0 + (i % 5)) / d) - 6.0)
+    G[3] = G[n - 1]                                    # two identical rows: exactly 0 between them
+    D = pkg.gar_pairwise_distances(G).cpu().numpy()
+    want = O.pairwise_sq_distances(G.cpu().numpy())
+    np.testing.assert_allclose(D, want, rtol=1e-6, atol=0)
+    assert D[3, n - 1] == 0 and np.array_equal(D, D.T)
+
+
+def test_distances_large_d_strided_nonfinite_reproducible(pkg):
+    n, d = 39, 50_000
+    big = pkg.workloads.make_uniform(n, d + 12, device=DEV, seed=9) - 0.5
+    for view in (big[:, :d], big[:, 4:d + 4], big[:, 8:d]):          # 16-byte-aligned starts, ld != d
+        D = pkg.gar_pairwise_distances(view).cpu().numpy()
+        want = O.pairwise_sq_distances(view.cpu().numpy())
+        np.testing.assert_allclose(D, want, rtol=1e-6, atol=0)
+    G = big[:, :d].contiguous()
+    assert torch.equal(pkg.gar_pairwise_distances(G).clone(), pkg.gar_pairwise_distances(G).clone())
+    G[5, 17] = float("nan")
+    G[20, d - 1] = float("inf")
+    G[38, 40_000] = float("-inf")
+    D = pkg.gar_pairwise_distances(G).cpu().numpy()
+    want = O.pairwise_sq_distances(G.cpu().numpy())
+    bad = np.isinf(want)
+    assert bad[5].sum() == n - 1 and bad[20].sum() == n - 1 and bad[38].sum() == n - 1
+    assert np.array_equal(np.isinf(D), bad)
+    np.testing.assert_allclose(D[~bad], want[~bad], rtol=1e-6, atol=0)
+
+
 # ------------------------------------------------ selection from the oracle's D
 @pytest.mark.parametrize("rule", ["krum", "multi_krum", "bulyan", "multi_bulyan"])
 @pytest.mark.parametrize("cfg,n,f", CONFIGS)
