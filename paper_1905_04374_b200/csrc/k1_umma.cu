@@ -1,0 +1,541 @@
+// Pairwise squared distances (the D_ij that the scores of Eq. 4 sum) for 16 < n <= 64 with the
+// Gram matrix on the fifth-generation tensor cores: tcgen05.mma, kind::i8, accumulators in
+// tensor memory.
+//
+// Arithmetic (the same exact scheme as the mma.sync kernel in k1_mma.cu).  Every row keeps a
+// running exponent E; a value x is rounded to the integer q = rint(x * 2^(148-E)), |q| < 2^22, and
+// q is split into three signed bytes q = l1 * 2^16 + l2 * 2^8 + l3.  With the byte matrices L1, L2,
+// L3 (rows x columns) the Gram matrix of the rounded rows is
+//     sum_ab 2^(8(3-a)) 2^(8(3-b)) La Lb^T        (a, b = 1..3),
+// int8 x int8 products summed exactly in int32.  The six products with a <= b are formed, kept as
+//     px = 2^32 L1L1^T + 2^16 L2L2^T + L3L3^T      (symmetric)
+//     pz = 2^24 L1L2^T + 2^16 L1L3^T + 2^8 L2L3^T
+// so that P = px + pz + pz^T, and D_ij = P_ii + P_jj - 2 P_ij.  Identical rows give identical
+// entries P_ii = P_ij = P_jj and a distance of exactly 0.
+//
+// One CTA per SM, persistent over slabs of 128 columns, four kinds of warps:
+//   producers (3 rows each)  cp.async ring -> quantise -> byte tiles in shared memory, laid out as
+//                            the K-major, unswizzled operand of tcgen05.mma: 16-byte chunks of a
+//                            row, rows in groups of eight (128 bytes), chunk stride LBO
+//   one MMA warp             per slab 4 k-steps x 2 instructions from one lane:
+//                            [L1; L2] x [L1; L2; L3]^T (128 x 192) and [L3; 0] x L3^T (128 x 64),
+//                            int32 accumulators in one of two sets of 256 tensor-memory columns
+//   four flush warps         when a row's exponent grows (or after 256 slabs) the MMA warp moves to
+//                            the other set; these warps read the closed set (tcgen05.ld, one warp
+//                            per 32 lanes), scale by the exponents it was built under and add it,
+//                            in fp64, into the CTA's px / pz arrays in global memory (L2)
+// Hand-offs are mbarriers (producer -> MMA, tcgen05.commit -> producer / flush, flush -> MMA);
+// every wait is bounded: a wait that gives up raises an error flag, all roles leave their loops,
+// the distance matrix is filled with NaN and the control block's error word is set.
+#include <cstdlib>
+
+#include "gar_internal.cuh"
+
+namespace gar {
+namespace {
+
+constexpr int KU_SLAB = 128;                 // columns per slab (one float4 per lane and row)
+constexpr int KU_JR = 3;                     // rows per producer warp
+constexpr int KU_NBUF = 3;                   // byte-tile buffers
+constexpr int KU_LBO = 256 * 16 + 16;        // bytes between 16-byte column chunks (256 rows + padding: conflict-free stores)
+constexpr int KU_SBO = 128;                  // bytes between groups of eight rows
+constexpr int KU_BUF_BYTES = 8 * KU_LBO;     // one slab: 8 chunks of 16 columns
+constexpr int KU_PERIOD = 256;               // slabs per accumulator set at most: |sum| <= 256 * 128 * 2^14 = 2^29
+constexpr int KU_MIN_EXP = 21;               // smallest row exponent (keeps the scale a normal float)
+constexpr int KU_SET_COLS = 256;             // tensor-memory columns per accumulator set (192 + 64)
+constexpr int KU_FLUSH_WARPS = 4;            // warps 0..3: tensor-memory lanes 32 w .. 32 w + 31
+constexpr int KU_MMA_WARP = 4;
+constexpr int KU_FIRST_PRODUCER = 5;
+constexpr unsigned KU_SPIN_LIMIT = 1u << 22; // polls of a barrier before a wait gives up (a few tenths of a second)
+constexpr int KU_BAR_FLUSH = 1;              // named barrier of the flush warps
+constexpr int KU_TRI = 2080;
+
+struct KUSmem {
+    unsigned long long full[KU_NBUF];        // producers -> MMA warp: the buffer's tiles are written
+    unsigned long long empty[KU_NBUF];       // tcgen05.commit -> producers: the MMAs that read the buffer are done
+    unsigned long long accfull[2];           // tcgen05.commit -> flush warps: the set is closed and complete
+    unsigned long long accfree[2];           // flush warps -> MMA warp: the set has been read
+    unsigned tmem_base;
+    int      error;
+    int      grow[KU_NBUF];                  // some row of the buffer uses a larger exponent than before
+    int      set_last[2];                    // the set is the CTA's last one
+    int      slab_exp[KU_NBUF][64];          // exponent each row of the buffer was quantised with
+    int      set_exp[2][64];                 // exponents of the rows while the set was accumulated
+    unsigned nonfinite_lo, nonfinite_hi;
+    int      is_last;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait for the phase with the given parity, the same answer in every lane of the warp.
+// False: the wait gave up (error flag raised) or another role raised the flag.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* error,
+                                          unsigned sleep_ns = 40, unsigned limit = KU_SPIN_LIMIT) {
+    bool ok = false;
+    for (unsigned spin = 0; spin < limit; ++spin) {
+        if (mbar_test(bar, parity)) { ok = true; break; }
+        if (*error) break;
+        if (spin > 32) __nanosleep(sleep_ns);
+        if (spin + 1 == limit) *error = 1;
+    }
+    return __all_sync(0xffffffffu, ok);
+}
+
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(unsigned* smem_dst, unsigned ncols) {      // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned ncols) {         // whole warp
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// Shared-memory operand descriptor: K-major, no swizzle.  Bits [0,14) address / 16, [16,30) chunk
+// stride / 16, [32,46) eight-row-group stride / 16, [46,48) = 1 (descriptor version), layout type 0.
+__device__ __forceinline__ unsigned long long umma_desc(unsigned saddr) {
+    return static_cast<unsigned long long>((saddr >> 4) & 0x3fffu) |
+           (static_cast<unsigned long long>(KU_LBO >> 4) << 16) |
+           (static_cast<unsigned long long>(KU_SBO >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor, kind::i8: int32 accumulators (2 at bit 4), signed 8-bit A and B (1 at bits
+// 7 and 10), both K-major (bits 15, 16 clear), N / 8 at bit 17, M / 16 at bit 24.
+__host__ __device__ constexpr unsigned umma_idesc(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | (unsigned(n >> 3) << 17) | (unsigned(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_i8(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc, unsigned idesc,
+                                        unsigned accumulate) {                            // one thread
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned long long* bar) {                    // one thread
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// this thread's lane of tensor memory, 8 consecutive columns
+__device__ __forceinline__ void tmem_ld8(unsigned taddr, int (&r)[8]) {                   // whole warp
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel) {
+    unsigned r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ double pow2(int e) { return __hiloint2double((1023 + e) << 20, 0); }   // -1022 <= e <= 1023
+__device__ __forceinline__ int tri_slot(int i, int j) { return i * 64 - (i * (i - 1)) / 2 + (j - i); }   // i <= j < 64
+
+// Shared memory: KUSmem, the byte-tile buffers, the raw ring float4 [NST][3 * producer warps][32].
+// scratch: per CTA 2 x 64 x 64 doubles (px and pz, stored transposed: [j][i]).
+template <int NST, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1)
+k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
+        double* __restrict__ partials, double* __restrict__ scratch, unsigned int* __restrict__ ticket,
+        unsigned int* __restrict__ error_word) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    KUSmem& sm = *reinterpret_cast<KUSmem*>(smem_raw);
+    constexpr int HEAD = (int(sizeof(KUSmem)) + 127) & ~127;
+    unsigned char* limb = smem_raw + HEAD;                                     // [KU_NBUF][KU_BUF_BYTES]
+    float4* ring = reinterpret_cast<float4*>(limb + KU_NBUF * KU_BUF_BYTES);    // [NST][3 pw][32]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nthreads = blockDim.x;
+    const int pw = (nthreads >> 5) - KU_FIRST_PRODUCER;                        // producer warps
+    const int ring_rows = KU_JR * pw;
+    volatile int* error = &sm.error;
+
+    for (int i = tid; i < KU_NBUF * KU_BUF_BYTES / 4; i += nthreads) reinterpret_cast<unsigned*>(limb)[i] = 0u;
+    if (tid < 64) {
+#pragma unroll
+        for (int b = 0; b < KU_NBUF; ++b) sm.slab_exp[b][tid] = KU_MIN_EXP;
+        sm.set_exp[0][tid] = KU_MIN_EXP;
+        sm.set_exp[1][tid] = KU_MIN_EXP;
+    }
+    if (tid == 0) {
+#pragma unroll
+        for (int b = 0; b < KU_NBUF; ++b) {
+            mbar_init(&sm.full[b], unsigned(pw));
+            mbar_init(&sm.empty[b], 1u);
+            sm.grow[b] = 0;
+        }
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sm.accfull[s], 1u);
+            mbar_init(&sm.accfree[s], unsigned(KU_FLUSH_WARPS));
+            sm.set_last[s] = 0;
+        }
+        sm.error = 0; sm.nonfinite_lo = 0u; sm.nonfinite_hi = 0u; sm.is_last = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == KU_MMA_WARP) tmem_alloc(&sm.tmem_base, 2 * KU_SET_COLS);
+    fence_async_smem();                  // the zeroed tiles are read by the tensor core (async proxy)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = sm.tmem_base;
+
+    const int64_t nslabs = (d + KU_SLAB - 1) / KU_SLAB;
+    const int64_t first = blockIdx.x, step = gridDim.x;
+    const int64_t mine = first < nslabs ? (nslabs - first + step - 1) / step : 0;
+    double* px_t = scratch + size_t(blockIdx.x) * 8192;
+    double* pz_t = px_t + 4096;
+
+    if (warp >= KU_FIRST_PRODUCER) {
+        // ================================================================ producers
+        const int p = warp - KU_FIRST_PRODUCER;
+        int row_exp[KU_JR];
+        const float* rowp[KU_JR];
+#pragma unroll
+        for (int jr = 0; jr < KU_JR; ++jr) {
+            const int row = p + jr * pw;
+            row_exp[jr] = KU_MIN_EXP;
+            rowp[jr] = g + int64_t(row < n ? row : 0) * ld + 4 * lane;
+        }
+        auto request = [&](int st, int64_t slab) {
+            const int64_t t0 = slab * KU_SLAB;
+            const int64_t left = d - t0 - 4 * lane;
+            const int bytes = left >= 4 ? 16 : (left > 0 ? int(left) * 4 : 0);
+            float4* dst = ring + (size_t(st) * ring_rows + p) * 32 + lane;
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr)
+                if (p + jr * pw < n) cp_async16(dst + size_t(jr) * pw * 32, bytes ? rowp[jr] + t0 : g, bytes);
+        };
+#pragma unroll
+        for (int s0 = 0; s0 < NST - 1; ++s0) {
+            if (s0 < mine) request(s0, first + s0 * step);
+            cp_async_commit();
+        }
+        const unsigned lane_off = unsigned(lane >> 2) * KU_LBO + unsigned(lane & 3) * 4;   // this lane's 4 columns
+        int buf = 0, st = 0;
+        unsigned empty_parity = 1;          // parity of the phase before the first one: the first KU_NBUF waits pass
+        for (int64_t it = 0; it < mine; ++it) {
+            cp_async_wait<NST - 2>();                                     // this lane's copies of slab `it` have landed
+            {
+                const int64_t nx = it + NST - 1;
+                int nst = st + NST - 1; if (nst >= NST) nst -= NST;
+                if (nx < mine) request(nst, first + nx * step);            // the stage read one iteration ago
+                cp_async_commit();
+            }
+            float4 v[KU_JR];
+            int ex[KU_JR];
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr) {
+                const int row = p + jr * pw;
+                v[jr] = row < n ? ring[(size_t(st) * ring_rows + row) * 32 + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr) {
+                // largest |value| as an integer: Inf and NaN come out with exponent 255
+                const unsigned a0 = __float_as_uint(v[jr].x) & 0x7fffffffu, a1 = __float_as_uint(v[jr].y) & 0x7fffffffu;
+                const unsigned a2 = __float_as_uint(v[jr].z) & 0x7fffffffu, a3 = __float_as_uint(v[jr].w) & 0x7fffffffu;
+                ex[jr] = int(__reduce_max_sync(0xffffffffu, max(max(a0, a1), max(a2, a3))) >> 23);
+            }
+            bool grew = false, any_bad = false;
+            float scale[KU_JR];
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr) {
+                const bool bad = ex[jr] == 255;
+                const bool up = !bad && ex[jr] > row_exp[jr];
+                row_exp[jr] = up ? ex[jr] + 1 : row_exp[jr];               // one binade of headroom
+                grew |= up;
+                any_bad |= bad;
+                scale[jr] = __uint_as_float(unsigned(275 - row_exp[jr]) << 23);   // 2^(148-E)
+            }
+            if (any_bad) {                                                   // rare: a row holds Inf or NaN
+#pragma unroll
+                for (int jr = 0; jr < KU_JR; ++jr) {
+                    const int row = p + jr * pw;
+                    if (ex[jr] == 255) {
+                        v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);            // quantised as zeros, flagged
+                        if (lane == 0 && row < n) {
+                            if (row < 32) atomicOr(&sm.nonfinite_lo, 1u << row); else atomicOr(&sm.nonfinite_hi, 1u << (row - 32));
+                        }
+                    }
+                }
+            }
+            unsigned w[KU_JR][4];
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr) {
+                // round to nearest through the 1.5 * 2^23 trick; the low three bytes of (q + 0x808080),
+                // each xor 0x80, are the signed bytes l1, l2, l3
+                w[jr][0] = __float_as_uint(fmaf(v[jr].x, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                w[jr][1] = __float_as_uint(fmaf(v[jr].y, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                w[jr][2] = __float_as_uint(fmaf(v[jr].z, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                w[jr][3] = __float_as_uint(fmaf(v[jr].w, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+            }
+            // the MMAs that read this buffer three slabs ago are done
+            if (!mbar_wait(&sm.empty[buf], empty_parity, error)) break;
+            unsigned char* tile = limb + buf * KU_BUF_BYTES + lane_off;
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr) {
+                const int row = p + jr * pw;
+                if (row < n) {
+                    const unsigned p01 = prmt(w[jr][0], w[jr][1], 0x5140u), p23 = prmt(w[jr][2], w[jr][3], 0x5140u);
+                    const unsigned h01 = prmt(w[jr][0], w[jr][1], 0x0062u), h23 = prmt(w[jr][2], w[jr][3], 0x0062u);
+                    *reinterpret_cast<unsigned*>(tile + (row) * 16)       = prmt(h01, h23, 0x5410u) ^ 0x80808080u;   // l1
+                    *reinterpret_cast<unsigned*>(tile + (64 + row) * 16)  = prmt(p01, p23, 0x7632u) ^ 0x80808080u;   // l2
+                    *reinterpret_cast<unsigned*>(tile + (128 + row) * 16) = prmt(p01, p23, 0x5410u) ^ 0x80808080u;   // l3
+                    if (lane == 0) sm.slab_exp[buf][row] = row_exp[jr];
+                }
+            }
+            if (grew && lane == 0) sm.grow[buf] = 1;
+            fence_async_smem();                      // generic-proxy stores -> visible to the tensor core's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.full[buf]);
+            if (++buf == KU_NBUF) { buf = 0; empty_parity ^= 1u; }
+            if (++st == NST) st = 0;
+        }
+        cp_async_wait<0>();
+    } else if (warp == KU_MMA_WARP) {
+        // ================================================================ MMA issue
+        constexpr unsigned IDESC_A = umma_idesc(128, 192), IDESC_B = umma_idesc(128, 64);
+        const unsigned limb_addr = smem_u32(limb);
+        int set = 0, since = 0;
+        int opened0 = 0, opened1 = 0;
+        bool have_open = false, fresh = true;
+        int buf = 0;
+        unsigned full_parity = 0;
+        for (int64_t it = 0; it < mine; ++it) {
+            if (!mbar_wait(&sm.full[buf], full_parity, error)) break;
+            tc_fence_after();
+            const bool grow = *reinterpret_cast<volatile int*>(&sm.grow[buf]) != 0;
+            if (!have_open || grow || since == KU_PERIOD) {
+                if (have_open) {                                            // close the running set
+                    __syncwarp();
+                    if (lane == 0) umma_commit(&sm.accfull[set]);
+                    set ^= 1;
+                }
+                const int opened = set ? opened1 : opened0;
+                if (opened > 0 && !mbar_wait(&sm.accfree[set], unsigned(opened - 1) & 1u, error)) break;
+                tc_fence_after();
+                sm.set_exp[set][lane] = sm.slab_exp[buf][lane];
+                sm.set_exp[set][lane + 32] = sm.slab_exp[buf][lane + 32];
+                if (lane == 0) { sm.grow[buf] = 0; sm.set_last[set] = 0; }
+                __threadfence_block();
+                __syncwarp();
+                if (set) ++opened1; else ++opened0;
+                have_open = true; fresh = true; since = 0;
+            }
+            if (lane == 0) {
+                const unsigned d1 = tmem_base + unsigned(set * KU_SET_COLS), d2 = d1 + 192u;
+                const unsigned base = limb_addr + unsigned(buf) * KU_BUF_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const unsigned long long t1 = umma_desc(base + unsigned(ks) * 2u * KU_LBO);            // rows 0..: L1, L2, L3
+                    const unsigned long long t3 = umma_desc(base + unsigned(ks) * 2u * KU_LBO + 128u * 16u);   // rows 128..: L3, zeros
+                    const unsigned acc = (fresh && ks == 0) ? 0u : 1u;
+                    umma_i8(d1, t1, t1, IDESC_A, acc);          // [L1; L2] x [L1; L2; L3]^T
+                    umma_i8(d2, t3, t3, IDESC_B, acc);          // [L3; 0] x L3^T
+                }
+                umma_commit(&sm.empty[buf]);                    // arrives when these MMAs have read the buffer
+            }
+            __syncwarp();
+            fresh = false;
+            ++since;
+            if (++buf == KU_NBUF) { buf = 0; full_parity ^= 1u; }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            if (have_open) {
+                sm.set_last[set] = 1;
+                __threadfence_block();
+                umma_commit(&sm.accfull[set]);
+            } else {
+                sm.error = 1;                                   // nothing was opened: a wait gave up at once
+            }
+        }
+    } else {
+        // ================================================================ flush: tensor memory -> fp64
+        const int q = warp;                                     // lanes 32 q .. 32 q + 31 of tensor memory
+        const int L = q * 32 + lane;
+        const int i = L & 63;
+        const bool lower = L >= 64;                             // rows of L2 (L1 otherwise)
+        const int ftid = tid;                                   // 0..127
+        for (int k = ftid; k < 8192; k += KU_FLUSH_WARPS * 32) __stcg(px_t + k, 0.0);
+        asm volatile("bar.sync %0, %1;" ::"r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
+        for (int k = 0;; ++k) {
+            const int set = k & 1;
+            // a set closes rarely: poll slowly; then agree over the four warps (they meet at named barriers below)
+            const bool ok = mbar_wait(&sm.accfull[set], unsigned(k >> 1) & 1u, error, 1000u, 1u << 20);
+            unsigned all_ok;
+            asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                         : "=r"(all_ok) : "r"(unsigned(ok)), "r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
+            if (!all_ok) { if (lane == 0) sm.error = 1; break; }
+            tc_fence_after();
+            const int last = *reinterpret_cast<volatile int*>(&sm.set_last[set]);
+            const int ei = sm.set_exp[set][i] - 296;
+            const unsigned tbase = tmem_base + (unsigned(q * 32) << 16) + unsigned(set * KU_SET_COLS);
+#pragma unroll 1
+            for (int phase = 0; phase < 2; ++phase) {
+                if ((phase == 1) == lower) {                    // warp-uniform: L1 rows first, then L2 rows
+#pragma unroll 1
+                    for (int j0 = 0; j0 < n; j0 += 8) {
+                        int r0[8], r1[8], r2[8], r3[8];
+                        if (!lower) {
+                            tmem_ld8(tbase + unsigned(j0), r0);             // L1 L1^T
+                            tmem_ld8(tbase + unsigned(64 + j0), r1);        // L1 L2^T
+                            tmem_ld8(tbase + unsigned(128 + j0), r2);       // L1 L3^T
+                            tmem_ld8(tbase + unsigned(192 + j0), r3);       // L3 L3^T
+                        } else {
+                            tmem_ld8(tbase + unsigned(64 + j0), r0);        // L2 L2^T
+                            tmem_ld8(tbase + unsigned(128 + j0), r1);       // L2 L3^T
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) { r2[t] = 0; r3[t] = 0; }
+                        }
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) {
+                            const int j = j0 + t;
+                            const int e = ei + sm.set_exp[set][j & 63];       // s_i s_j = 2^e
+                            double x, y;                                      // exact: |sums| < 2^30
+                            if (!lower) {
+                                x = double(r0[t]) * pow2(e + 32) + double(r3[t]) * pow2(e);
+                                y = (double(r1[t]) * 256.0 + double(r2[t])) * pow2(e + 16);
+                            } else {
+                                x = double(r0[t]) * pow2(e + 16);
+                                y = double(r1[t]) * pow2(e + 8);
+                            }
+                            if (i < n && j < n) {
+                                __stcg(px_t + j * 64 + i, __ldcg(px_t + j * 64 + i) + x);
+                                __stcg(pz_t + j * 64 + i, __ldcg(pz_t + j * 64 + i) + y);
+                            }
+                        }
+                    }
+                }
+                asm volatile("bar.sync %0, %1;" ::"r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.accfree[set]);
+            if (last) break;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == KU_MMA_WARP) tmem_dealloc(tmem_base, 2 * KU_SET_COLS);
+
+    // CTA partial: P_ij = px_ij + (pz_ij + pz_ji) for i <= j (the same expression on the diagonal, so
+    // identical rows give bit-identical P_ii, P_ij, P_jj); slots 2300/2301: non-finite row masks,
+    // 2302: error flag
+    double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
+    for (int idx = tid; idx < 64 * 64; idx += nthreads) {
+        const int i = idx >> 6, j = idx & 63;
+        if (i <= j) {
+            double v = 0.0;
+            if (j < n) v = __ldcg(px_t + j * 64 + i) + (__ldcg(pz_t + j * 64 + i) + __ldcg(pz_t + i * 64 + j));
+            my_partial[tri_slot(i, j)] = v;
+        }
+    }
+    if (tid == 0) {
+        my_partial[2300] = double(sm.nonfinite_lo);
+        my_partial[2301] = double(sm.nonfinite_hi);
+        my_partial[2302] = double(sm.error);
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sm.is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!sm.is_last) return;
+    __threadfence();
+
+    // last CTA: add the partials in CTA order, then D_ij = P_ii + P_jj - 2 P_ij
+    double* ptot = reinterpret_cast<double*>(limb);              // reuse: 2080 totals
+    for (int s = tid; s < KU_TRI; s += nthreads) {
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+        unsigned b = 0;
+        for (; b + 4 <= gridDim.x; b += 4) {
+            s0 += __ldcg(partials + size_t(b) * kPairSlots + s);
+            s1 += __ldcg(partials + size_t(b + 1) * kPairSlots + s);
+            s2 += __ldcg(partials + size_t(b + 2) * kPairSlots + s);
+            s3 += __ldcg(partials + size_t(b + 3) * kPairSlots + s);
+        }
+        for (; b < gridDim.x; ++b) s0 += __ldcg(partials + size_t(b) * kPairSlots + s);
+        ptot[s] = (s0 + s1) + (s2 + s3);
+    }
+    if (tid == 0) {
+        unsigned lo = 0u, hi = 0u, err = 0u;
+        for (unsigned b = 0; b < gridDim.x; ++b) {
+            lo |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2300));
+            hi |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2301));
+            err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2302));
+        }
+        sm.nonfinite_lo = lo; sm.nonfinite_hi = hi; sm.error = int(err);
+        if (err) *error_word = 1u;
+    }
+    __syncthreads();
+    const unsigned long long bad = (static_cast<unsigned long long>(sm.nonfinite_hi) << 32) | sm.nonfinite_lo;
+    const bool failed = sm.error != 0;
+    for (int idx = tid; idx < n * n; idx += nthreads) {
+        const int i = idx / n, j = idx - i * n;
+        double v = 0.0;
+        if (i != j) {
+            const int lo = i < j ? i : j, hi = i < j ? j : i;
+            v = ptot[tri_slot(lo, lo)] + ptot[tri_slot(hi, hi)] - 2.0 * ptot[tri_slot(lo, hi)];
+            if (v < 0.0) v = 0.0;
+            if (((bad >> i) | (bad >> j)) & 1ull) v = INFINITY;
+        }
+        dist[idx] = failed ? __longlong_as_double(0x7ff8000000000000ll) : v;
+    }
+    if (tid == 0) *ticket = 0u;               // ready for the next call
+}
+
+template <int NST, int MAXT>
+cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
+                      int pw, cudaStream_t stream) {
+    static size_t configured[64] = {0};                        // dynamic shared memory the kernel is allowed, per device
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    const size_t head = (sizeof(KUSmem) + 127) & ~size_t(127);
+    const size_t smem = head + size_t(KU_NBUF) * KU_BUF_BYTES + size_t(NST) * KU_JR * pw * 32 * sizeof(float4);
+    if (dev < 0 || dev >= 64 || configured[dev] < smem) {
+        err = cudaFuncSetAttribute(k1_umma<NST, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (err != cudaSuccess) return err;
+        if (dev >= 0 && dev < 64) configured[dev] = smem;
+    }
+    // one CTA per SM: every CTA owns all 512 tensor-memory columns of its SM (the shared memory it
+    // asks for, more than half an SM's, keeps a second CTA away)
+    const int64_t nslabs = (d + KU_SLAB - 1) / KU_SLAB;
+    int64_t grid = sm_count;
+    if (grid > kMaxCtasUmma) grid = kMaxCtasUmma;
+    if (grid > nslabs) grid = nslabs;
+    k1_umma<NST, MAXT><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
+        g, n, d, ld, dist, ws.partials(), ws.scratch(), ws.ticket(), ws.k1_error());
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+// 16 < n <= 64, grads 16-byte aligned, ld % 4 == 0.
+cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
+                                  int sm_count, cudaStream_t stream) {
+    const int pw = (n + KU_JR - 1) / KU_JR;                    // producer warps: three rows each
+    if (pw <= 14) return launch_ku<4, 32 * (KU_FIRST_PRODUCER + 14)>(grads, n, d, ld, dist, ws, sm_count, pw, stream);
+    if (pw <= 17) return launch_ku<4, 32 * (KU_FIRST_PRODUCER + 22)>(grads, n, d, ld, dist, ws, sm_count, pw, stream);
+    return launch_ku<3, 32 * (KU_FIRST_PRODUCER + 22)>(grads, n, d, ld, dist, ws, sm_count, pw, stream);
+}
+
+}  // namespace gar
