@@ -139,9 +139,6 @@ __device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
     return r;
 }
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc, int src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(src_bytes) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
@@ -204,61 +201,85 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 
     if (warp >= KU_FIRST_PRODUCER) {
         // ================================================================ producers
+        // All shared-memory addresses are 32-bit window offsets and every per-slab quantity is kept
+        // incrementally: this loop's instruction count bounds the kernel.
         const int p = warp - KU_FIRST_PRODUCER;
         int row_exp[KU_JR];
-        const float* rowp[KU_JR];
+        const float* nextp[KU_JR];                     // this lane's float4 of the next slab to request
+        bool valid[KU_JR];
+        unsigned tile_off[KU_JR];                      // byte offset of (row, this lane's 4 columns) in a tile buffer
 #pragma unroll
         for (int jr = 0; jr < KU_JR; ++jr) {
             const int row = p + jr * pw;
+            valid[jr] = row < n;
             row_exp[jr] = KU_MIN_EXP;
-            rowp[jr] = g + int64_t(row < n ? row : 0) * ld + 4 * lane;
+            nextp[jr] = g + int64_t(valid[jr] ? row : 0) * ld + first * KU_SLAB + 4 * lane;
+            tile_off[jr] = unsigned(lane >> 2) * KU_LBO + unsigned(lane & 3) * 4 + unsigned(row) * 16;
         }
-        auto request = [&](int st, int64_t slab) {
-            const int64_t t0 = slab * KU_SLAB;
-            const int64_t left = d - t0 - 4 * lane;
-            const int bytes = left >= 4 ? 16 : (left > 0 ? int(left) * 4 : 0);
-            float4* dst = ring + (size_t(st) * ring_rows + p) * 32 + lane;
+        const int64_t advance = step * KU_SLAB;                                    // floats between this CTA's slabs
+        const unsigned stage_bytes = unsigned(ring_rows) * 512u, row_stride = unsigned(pw) * 512u;
+        const unsigned my_ring = smem_u32(ring) + unsigned(p * 32 + lane) * 16u;   // (stage 0, row p, this lane)
+        const unsigned limb_u32 = smem_u32(limb);
+        // the last slab of the matrix may be ragged: bytes of this lane's float4 that exist there
+        const int64_t last_left = d - (nslabs - 1) * KU_SLAB - 4 * lane;
+        const int last_bytes = last_left >= 4 ? 16 : (last_left > 0 ? int(last_left) * 4 : 0);
+        const int last_it = (first + (mine - 1) * step == nslabs - 1) ? int(mine - 1) : -1;   // this CTA's iteration of it
+        auto request = [&](unsigned stage_off, int it_req) {
+            const int bytes = it_req == last_it ? last_bytes : 16;
 #pragma unroll
-            for (int jr = 0; jr < KU_JR; ++jr)
-                if (p + jr * pw < n) cp_async16(dst + size_t(jr) * pw * 32, bytes ? rowp[jr] + t0 : g, bytes);
+            for (int jr = 0; jr < KU_JR; ++jr) {
+                if (valid[jr]) {
+                    const float* src = bytes ? nextp[jr] : g;                        // nothing is read when bytes == 0
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n"
+                                 ::"r"(my_ring + stage_off + unsigned(jr) * row_stride), "l"(src), "r"(bytes) : "memory");
+                    nextp[jr] += advance;
+                }
+            }
         };
+        const int nmine = int(mine);
+        unsigned req_off = 0;                           // stage of the next request
 #pragma unroll
         for (int s0 = 0; s0 < NST - 1; ++s0) {
-            if (s0 < mine) request(s0, first + s0 * step);
+            if (s0 < nmine) request(req_off, s0);
             cp_async_commit();
+            req_off += stage_bytes;
         }
-        const unsigned lane_off = unsigned(lane >> 2) * KU_LBO + unsigned(lane & 3) * 4;   // this lane's 4 columns
-        int buf = 0, st = 0;
+        unsigned cur_off = 0, buf_off = 0;              // stage being read, tile buffer being written
+        int buf = 0;
         unsigned empty_parity = 1;          // parity of the phase before the first one: the first KU_NBUF waits pass
-        for (int64_t it = 0; it < mine; ++it) {
+        for (int it = 0; it < nmine; ++it) {
             cp_async_wait<NST - 2>();                                     // this lane's copies of slab `it` have landed
-            {
-                const int64_t nx = it + NST - 1;
-                int nst = st + NST - 1; if (nst >= NST) nst -= NST;
-                if (nx < mine) request(nst, first + nx * step);            // the stage read one iteration ago
-                cp_async_commit();
-            }
+            if (it + NST - 1 < nmine) request(req_off, it + NST - 1);     // into the stage read one iteration ago
+            cp_async_commit();
+            req_off += stage_bytes;
+            if (req_off == unsigned(NST) * stage_bytes) req_off = 0;
             float4 v[KU_JR];
             int ex[KU_JR];
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
-                const int row = p + jr * pw;
-                v[jr] = row < n ? ring[(size_t(st) * ring_rows + row) * 32 + lane] : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (valid[jr])
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                 : "=f"(v[jr].x), "=f"(v[jr].y), "=f"(v[jr].z), "=f"(v[jr].w)
+                                 : "r"(my_ring + cur_off + unsigned(jr) * row_stride) : "memory");
             }
+            cur_off += stage_bytes;
+            if (cur_off == unsigned(NST) * stage_bytes) cur_off = 0;
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
-                // largest |value| as an integer: Inf and NaN come out with exponent 255
-                const unsigned a0 = __float_as_uint(v[jr].x) & 0x7fffffffu, a1 = __float_as_uint(v[jr].y) & 0x7fffffffu;
-                const unsigned a2 = __float_as_uint(v[jr].z) & 0x7fffffffu, a3 = __float_as_uint(v[jr].w) & 0x7fffffffu;
-                ex[jr] = int(__reduce_max_sync(0xffffffffu, max(max(a0, a1), max(a2, a3))) >> 23);
+                // largest |value| of the slab row; x * 0 is 0 for finite x and NaN otherwise, so the sum
+                // below is the maximum, or NaN (exponent field 255) when a value is Inf or NaN
+                const float m = fmaxf(fmaxf(fabsf(v[jr].x), fabsf(v[jr].y)), fmaxf(fabsf(v[jr].z), fabsf(v[jr].w)));
+                const float nf = fmaf(v[jr].x, 0.f, fmaf(v[jr].y, 0.f, fmaf(v[jr].z, 0.f, v[jr].w * 0.f)));
+                ex[jr] = int(__reduce_max_sync(0xffffffffu, __float_as_uint(m + nf)) >> 23);   // >= 255: not finite
             }
             bool grew = false, any_bad = false;
             float scale[KU_JR];
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
-                const bool bad = ex[jr] == 255;
+                const bool bad = ex[jr] >= 255;
                 const bool up = !bad && ex[jr] > row_exp[jr];
-                row_exp[jr] = up ? ex[jr] + 1 : row_exp[jr];               // one binade of headroom
+                if (up) row_exp[jr] = ex[jr] + 1;                            // one binade of headroom
                 grew |= up;
                 any_bad |= bad;
                 scale[jr] = __uint_as_float(unsigned(275 - row_exp[jr]) << 23);   // 2^(148-E)
@@ -267,9 +288,9 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 #pragma unroll
                 for (int jr = 0; jr < KU_JR; ++jr) {
                     const int row = p + jr * pw;
-                    if (ex[jr] == 255) {
+                    if (ex[jr] >= 255) {
                         v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);            // quantised as zeros, flagged
-                        if (lane == 0 && row < n) {
+                        if (lane == 0 && valid[jr]) {
                             if (row < 32) atomicOr(&sm.nonfinite_lo, 1u << row); else atomicOr(&sm.nonfinite_hi, 1u << (row - 32));
                         }
                     }
@@ -287,25 +308,24 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             }
             // the MMAs that read this buffer three slabs ago are done
             if (!mbar_wait(&sm.empty[buf], empty_parity, error)) break;
-            unsigned char* tile = limb + buf * KU_BUF_BYTES + lane_off;
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
-                const int row = p + jr * pw;
-                if (row < n) {
+                if (valid[jr]) {
                     const unsigned p01 = prmt(w[jr][0], w[jr][1], 0x5140u), p23 = prmt(w[jr][2], w[jr][3], 0x5140u);
                     const unsigned h01 = prmt(w[jr][0], w[jr][1], 0x0062u), h23 = prmt(w[jr][2], w[jr][3], 0x0062u);
-                    *reinterpret_cast<unsigned*>(tile + (row) * 16)       = prmt(h01, h23, 0x5410u) ^ 0x80808080u;   // l1
-                    *reinterpret_cast<unsigned*>(tile + (64 + row) * 16)  = prmt(p01, p23, 0x7632u) ^ 0x80808080u;   // l2
-                    *reinterpret_cast<unsigned*>(tile + (128 + row) * 16) = prmt(p01, p23, 0x5410u) ^ 0x80808080u;   // l3
-                    if (lane == 0) sm.slab_exp[buf][row] = row_exp[jr];
+                    const unsigned at = limb_u32 + buf_off + tile_off[jr];
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(at), "r"(prmt(h01, h23, 0x5410u) ^ 0x80808080u) : "memory");             // l1
+                    asm volatile("st.shared.b32 [%0+1024], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x7632u) ^ 0x80808080u) : "memory");        // l2: rows 64..
+                    asm volatile("st.shared.b32 [%0+2048], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x5410u) ^ 0x80808080u) : "memory");        // l3: rows 128..
+                    if (lane == 0) sm.slab_exp[buf][p + jr * pw] = row_exp[jr];
                 }
             }
             if (grew && lane == 0) sm.grow[buf] = 1;
             fence_async_smem();                      // generic-proxy stores -> visible to the tensor core's reads
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.full[buf]);
-            if (++buf == KU_NBUF) { buf = 0; empty_parity ^= 1u; }
-            if (++st == NST) st = 0;
+            buf_off += KU_BUF_BYTES;
+            if (++buf == KU_NBUF) { buf = 0; buf_off = 0; empty_parity ^= 1u; }
         }
         cp_async_wait<0>();
     } else if (warp == KU_MMA_WARP) {
