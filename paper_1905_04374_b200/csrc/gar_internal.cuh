@@ -10,7 +10,6 @@ namespace gar {
 // ---- workspace layout (device) -------------------------------------------
 // [0, 256)                control block (ticket counter of the distance kernel)
 // [256, +partials)        per-CTA partial distance sums, fp64
-// [.., +scratch)          per-CTA fp64 running sums of the tcgen05 distance kernel
 // [.., +n*n doubles)      distance matrix
 // [.., +sizeof(selection)) selection result / coordinate-phase schedule
 constexpr int    kMaxCtasK1      = 592;                 // upper bound on the distance kernel's grid
@@ -18,15 +17,12 @@ constexpr int    kMaxTiles       = 36;                  // 8x8 row-block pairs a
 constexpr int    kPairSlots      = kMaxTiles * 64;      // fp64 slots per CTA partial
 constexpr size_t kCtrlBytes      = 256;
 constexpr size_t kPartialBytes   = size_t(kMaxCtasK1) * kPairSlots * sizeof(double);
-constexpr int    kMaxCtasUmma    = 160;                 // grid bound of the tcgen05 distance kernel (one CTA per SM)
-constexpr size_t kUmmaScratchBytes = size_t(kMaxCtasUmma) * 2 * 64 * 64 * sizeof(double);
 constexpr size_t kDistBytes      = size_t(GAR_MAX_N) * GAR_MAX_N * sizeof(double);
 
 constexpr size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 
 constexpr size_t kOffPartials  = kCtrlBytes;
-constexpr size_t kOffScratch   = kOffPartials + align256(kPartialBytes);
-constexpr size_t kOffDist      = kOffScratch + align256(kUmmaScratchBytes);
+constexpr size_t kOffDist      = kOffPartials + align256(kPartialBytes);
 constexpr size_t kOffSelection = kOffDist + align256(kDistBytes);
 constexpr size_t kWorkspaceBytes = kOffSelection + align256(sizeof(gar_selection_t));
 
@@ -34,7 +30,6 @@ struct Workspace {
     char* base;
     unsigned int*    ticket()    const { return reinterpret_cast<unsigned int*>(base); }
     unsigned int*    k1_error()  const { return reinterpret_cast<unsigned int*>(base) + 2; }   // a bounded device wait gave up
-    double*          scratch()   const { return reinterpret_cast<double*>(base + kOffScratch); }
     double*          partials()  const { return reinterpret_cast<double*>(base + kOffPartials); }
     double*          dist()      const { return reinterpret_cast<double*>(base + kOffDist); }
     gar_selection_t* selection() const { return reinterpret_cast<gar_selection_t*>(base + kOffSelection); }

@@ -607,7 +607,7 @@ namespace gar {
 // Its size is fixed: kStaticScratchBytes (about 10.9 MB), enough for the largest grid the
 // distance kernels ever use and n <= GAR_MAX_N; every GPU that loads the library holds it
 // until the process exits.
-constexpr size_t kStaticScratchBytes = kOffScratch + kUmmaScratchBytes;
+constexpr size_t kStaticScratchBytes = kCtrlBytes + kPartialBytes;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {

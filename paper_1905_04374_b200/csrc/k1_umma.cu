@@ -18,12 +18,13 @@
 //                            the K-major, unswizzled operand of tcgen05.mma: 16-byte chunks of a
 //                            row, rows in groups of eight (128 bytes), chunk stride LBO
 //   one MMA warp             per slab 4 k-steps x 2 instructions from one lane:
-//                            [L1; L2] x [L1; L2; L3]^T (128 x 192) and [L3; 0] x L3^T (128 x 64),
+//                            [L1; L2] x [L1; L2; L3]^T (128 x 192) and [L3; *] x L3^T (128 x 64; the lower 64
+//                            rows of the second A run on into the next chunk and their products are never read),
 //                            int32 accumulators in one of two sets of 256 tensor-memory columns
 //   four flush warps         when a row's exponent grows (or after 256 slabs) the MMA warp moves to
 //                            the other set; these warps read the closed set (tcgen05.ld, one warp
 //                            per 32 lanes), scale by the exponents it was built under and add it,
-//                            in fp64, into the CTA's px / pz arrays in global memory (L2)
+//                            in fp64, into the CTA's px / pz arrays in shared memory
 // Hand-offs are mbarriers (producer -> MMA, tcgen05.commit -> producer / flush, flush -> MMA);
 // every wait is bounded: a wait that gives up raises an error flag, all roles leave their loops,
 // the distance matrix is filled with NaN and the control block's error word is set.
@@ -37,7 +38,7 @@ namespace {
 constexpr int KU_SLAB = 128;                 // columns per slab (one float4 per lane and row)
 constexpr int KU_JR = 3;                     // rows per producer warp
 constexpr int KU_NBUF = 3;                   // byte-tile buffers
-constexpr int KU_LBO = 256 * 16 + 16;        // bytes between 16-byte column chunks (256 rows + padding: conflict-free stores)
+constexpr int KU_LBO = 192 * 16 + 16;        // bytes between 16-byte column chunks (192 rows + padding: conflict-free stores)
 constexpr int KU_SBO = 128;                  // bytes between groups of eight rows
 constexpr int KU_BUF_BYTES = 8 * KU_LBO;     // one slab: 8 chunks of 16 columns
 constexpr int KU_PERIOD = 256;               // slabs per accumulator set at most: |sum| <= 256 * 128 * 2^14 = 2^29
@@ -145,25 +146,27 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 __device__ __forceinline__ double pow2(int e) { return __hiloint2double((1023 + e) << 20, 0); }   // -1022 <= e <= 1023
 __device__ __forceinline__ int tri_slot(int i, int j) { return i * 64 - (i * (i - 1)) / 2 + (j - i); }   // i <= j < 64
 
-// Shared memory: KUSmem, the byte-tile buffers, the raw ring float4 [NST][3 * producer warps][32].
-// scratch: per CTA 2 x 64 x 64 doubles (px and pz, stored transposed: [j][i]).
+// Shared memory: KUSmem, the byte-tile buffers, px and pz (2 x 64 x 64 doubles, stored transposed:
+// [j][i]), the raw ring float4 [NST][3 * producer warps][32].
 template <int NST, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1)
 k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
-        double* __restrict__ partials, double* __restrict__ scratch, unsigned int* __restrict__ ticket,
+        double* __restrict__ partials, unsigned int* __restrict__ ticket,
         unsigned int* __restrict__ error_word) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     KUSmem& sm = *reinterpret_cast<KUSmem*>(smem_raw);
     constexpr int HEAD = (int(sizeof(KUSmem)) + 127) & ~127;
     unsigned char* limb = smem_raw + HEAD;                                     // [KU_NBUF][KU_BUF_BYTES]
-    float4* ring = reinterpret_cast<float4*>(limb + KU_NBUF * KU_BUF_BYTES);    // [NST][3 pw][32]
+    double* px_t = reinterpret_cast<double*>(limb + KU_NBUF * KU_BUF_BYTES);    // [64][64]: px_t[j * 64 + i] = px_ij
+    double* pz_t = px_t + 4096;
+    float4* ring = reinterpret_cast<float4*>(pz_t + 4096);                      // [NST][3 pw][32]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nthreads = blockDim.x;
     const int pw = (nthreads >> 5) - KU_FIRST_PRODUCER;                        // producer warps
     const int ring_rows = KU_JR * pw;
     volatile int* error = &sm.error;
 
-    for (int i = tid; i < KU_NBUF * KU_BUF_BYTES / 4; i += nthreads) reinterpret_cast<unsigned*>(limb)[i] = 0u;
+    for (int i = tid; i < (KU_NBUF * KU_BUF_BYTES + 2 * 4096 * 8) / 4; i += nthreads) reinterpret_cast<unsigned*>(limb)[i] = 0u;
     if (tid < 64) {
 #pragma unroll
         for (int b = 0; b < KU_NBUF; ++b) sm.slab_exp[b][tid] = KU_MIN_EXP;
@@ -196,8 +199,6 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     const int64_t nslabs = (d + KU_SLAB - 1) / KU_SLAB;
     const int64_t first = blockIdx.x, step = gridDim.x;
     const int64_t mine = first < nslabs ? (nslabs - first + step - 1) / step : 0;
-    double* px_t = scratch + size_t(blockIdx.x) * 8192;
-    double* pz_t = px_t + 4096;
 
     if (warp >= KU_FIRST_PRODUCER) {
         // ================================================================ producers
@@ -364,10 +365,10 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     const unsigned long long t1 = umma_desc(base + unsigned(ks) * 2u * KU_LBO);            // rows 0..: L1, L2, L3
-                    const unsigned long long t3 = umma_desc(base + unsigned(ks) * 2u * KU_LBO + 128u * 16u);   // rows 128..: L3, zeros
+                    const unsigned long long t3 = umma_desc(base + unsigned(ks) * 2u * KU_LBO + 128u * 16u);   // rows 128..: L3, then unread rows
                     const unsigned acc = (fresh && ks == 0) ? 0u : 1u;
                     umma_i8(d1, t1, t1, IDESC_A, acc);          // [L1; L2] x [L1; L2; L3]^T
-                    umma_i8(d2, t3, t3, IDESC_B, acc);          // [L3; 0] x L3^T
+                    umma_i8(d2, t3, t3, IDESC_B, acc);          // [L3; *] x L3^T
                 }
                 umma_commit(&sm.empty[buf]);                    // arrives when these MMAs have read the buffer
             }
@@ -392,9 +393,6 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         const int L = q * 32 + lane;
         const int i = L & 63;
         const bool lower = L >= 64;                             // rows of L2 (L1 otherwise)
-        const int ftid = tid;                                   // 0..127
-        for (int k = ftid; k < 8192; k += KU_FLUSH_WARPS * 32) __stcg(px_t + k, 0.0);
-        asm volatile("bar.sync %0, %1;" ::"r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
         for (int k = 0;; ++k) {
             const int set = k & 1;
             // a set closes rarely: poll slowly; then agree over the four warps (they meet at named barriers below)
@@ -438,8 +436,8 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
                                 y = double(r1[t]) * pow2(e + 8);
                             }
                             if (i < n && j < n) {
-                                __stcg(px_t + j * 64 + i, __ldcg(px_t + j * 64 + i) + x);
-                                __stcg(pz_t + j * 64 + i, __ldcg(pz_t + j * 64 + i) + y);
+                                px_t[j * 64 + i] += x;
+                                pz_t[j * 64 + i] += y;
                             }
                         }
                     }
@@ -465,7 +463,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         const int i = idx >> 6, j = idx & 63;
         if (i <= j) {
             double v = 0.0;
-            if (j < n) v = __ldcg(px_t + j * 64 + i) + (__ldcg(pz_t + j * 64 + i) + __ldcg(pz_t + i * 64 + j));
+            if (j < n) v = px_t[j * 64 + i] + (pz_t[j * 64 + i] + pz_t[i * 64 + j]);
             my_partial[tri_slot(i, j)] = v;
         }
     }
@@ -524,13 +522,11 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 
 template <int NST, int MAXT>
 cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
-                      int pw, cudaStream_t stream) {
+                      int pw, size_t smem, cudaStream_t stream) {
     static size_t configured[64] = {0};                        // dynamic shared memory the kernel is allowed, per device
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
-    const size_t head = (sizeof(KUSmem) + 127) & ~size_t(127);
-    const size_t smem = head + size_t(KU_NBUF) * KU_BUF_BYTES + size_t(NST) * KU_JR * pw * 32 * sizeof(float4);
     if (dev < 0 || dev >= 64 || configured[dev] < smem) {
         err = cudaFuncSetAttribute(k1_umma<NST, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (err != cudaSuccess) return err;
@@ -540,10 +536,10 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     // asks for, more than half an SM's, keeps a second CTA away)
     const int64_t nslabs = (d + KU_SLAB - 1) / KU_SLAB;
     int64_t grid = sm_count;
-    if (grid > kMaxCtasUmma) grid = kMaxCtasUmma;
+    if (grid > kMaxCtasK1) grid = kMaxCtasK1;
     if (grid > nslabs) grid = nslabs;
     k1_umma<NST, MAXT><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
-        g, n, d, ld, dist, ws.partials(), ws.scratch(), ws.ticket(), ws.k1_error());
+        g, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error());
     return cudaGetLastError();
 }
 
@@ -553,9 +549,19 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
 cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
                                   int sm_count, cudaStream_t stream) {
     const int pw = (n + KU_JR - 1) / KU_JR;                    // producer warps: three rows each
-    if (pw <= 14) return launch_ku<4, 32 * (KU_FIRST_PRODUCER + 14)>(grads, n, d, ld, dist, ws, sm_count, pw, stream);
-    if (pw <= 17) return launch_ku<4, 32 * (KU_FIRST_PRODUCER + 22)>(grads, n, d, ld, dist, ws, sm_count, pw, stream);
-    return launch_ku<3, 32 * (KU_FIRST_PRODUCER + 22)>(grads, n, d, ld, dist, ws, sm_count, pw, stream);
+    const size_t fixed = ((sizeof(KUSmem) + 127) & ~size_t(127)) + size_t(KU_NBUF) * KU_BUF_BYTES + 2 * 4096 * sizeof(double);
+    const size_t stage = size_t(KU_JR) * pw * 32 * sizeof(float4);
+    constexpr size_t kSmemMax = 227 * 1024;                    // per-CTA limit of the SM
+    constexpr int kSmall = 32 * (KU_FIRST_PRODUCER + 14), kLarge = 32 * (KU_FIRST_PRODUCER + 22);
+    int nst = 4;
+    while (nst > 2 && fixed + nst * stage > kSmemMax) --nst;   // deepest raw ring that fits
+    const size_t smem = fixed + nst * stage;
+#define GAR_KU(NSTV, MAXTV) return launch_ku<NSTV, MAXTV>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream)
+    if (pw <= 14) { if (nst == 4) GAR_KU(4, kSmall); if (nst == 3) GAR_KU(3, kSmall); GAR_KU(2, kSmall); }
+    if (nst == 4) GAR_KU(4, kLarge);
+    if (nst == 3) GAR_KU(3, kLarge);
+    GAR_KU(2, kLarge);
+#undef GAR_KU
 }
 
 }  // namespace gar
