@@ -26,16 +26,17 @@ K3_P_LIST(K3_DECL)
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, const gar_selection_t* sel,
                               int theta, int preagg, float* out, int sm_count, cudaStream_t stream) {
     const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out);
-    int vec = 1;
-    if (a % 16 == 0 && ld % 4 == 0) vec = 4;
-    else if (a % 8 == 0 && ld % 2 == 0) vec = 2;
+    int vec_max = 1;                                      // what the alignment allows
+    if (a % 16 == 0 && ld % 4 == 0) vec_max = 4;
+    else if (a % 8 == 0 && ld % 2 == 0) vec_max = 2;
     // widest width that keeps the kernel's registers in check: large slot counts use narrower vectors
+    int vec = vec_max;
     if (vec == 4 && theta > 8) vec = 2;
     if (vec == 2 && theta > (preagg ? 12 : 24)) vec = 1;
-    static const char* env = std::getenv("GAR_K3_VEC");   // tuning aid: cap the vector width
+    static const char* env = std::getenv("GAR_K3_VEC");   // tuning aid: vector width, if the alignment allows it
     if (env) {
-        const int cap = std::atoi(env);
-        if (cap == 1 || cap == 2 || cap == 4) vec = vec < cap ? vec : cap;
+        const int want = std::atoi(env);
+        if (want == 1 || want == 2 || want == 4) vec = want < vec_max ? want : vec_max;
     }
 #define K3_TRY(P) \
     if (theta <= P) return launch_k3_p<P>(grads, n, d, ld, sel, preagg, vec, out, sm_count, stream);
