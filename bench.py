@@ -242,7 +242,7 @@ def run_ours(args):
     achieved = kernels[dom]["gbs"]
     # DRAM bytes per coordinate from the committed ncu captures (profiles/), taken on a smaller d of
     # the same kernel and scaled by d; None where no capture of the current kernel exists
-    ncu_bytes_per_coord = {("k1_distances", 39): 316.3e6 / 2.0e6, ("k3_coordinate", 39): 240.6e6 / 2.0e6, ("k3_coordinate", 51): 302.3e6 / 1.5e6,
+    ncu_bytes_per_coord = {("k1_distances", 39): 317.0e6 / 2.0e6, ("k3_coordinate", 39): 240.6e6 / 2.0e6, ("k3_coordinate", 51): 302.3e6 / 1.5e6,
                            ("k1_distances", 15): 244.4e6 / 4.0e6, ("k3_coordinate", 15): 172.0e6 / 4.0e6}
     per_coord = ncu_bytes_per_coord.get((dom, n))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",

@@ -29,7 +29,6 @@ def _nvcc() -> str:
 
 def _units():
     units = [("k1_distances.cu", "k1_distances.o", []),
-             ("k1_mma.cu", "k1_mma.o", []),
              ("k1_umma.cu", "k1_umma.o", []),
              ("k2_select.cu", "k2_select.o", []),
              ("k3_dispatch.cu", "k3_dispatch.o", []),

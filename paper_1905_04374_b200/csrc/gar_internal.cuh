@@ -42,11 +42,9 @@ struct Workspace {
 cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
                              const Workspace& ws, int sm_count, cudaStream_t stream);
 
-// Tensor-core variant (16 < n <= 64, 16-byte aligned rows), used from kMmaMinDim coordinates on.
+// Tensor-core variant (tcgen05, accumulators in tensor memory) for 16 < n <= 64 and 16-byte
+// aligned rows, used from kMmaMinDim coordinates on.
 constexpr int64_t kMmaMinDim = 32768;
-cudaError_t launch_distances_mma(const float* grads, int n, int64_t d, int64_t ld, double* dist,
-                                 const Workspace& ws, int sm_count, cudaStream_t stream);
-// tcgen05 variant of the same arithmetic (accumulators in tensor memory), same conditions.
 cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist,
                                   const Workspace& ws, int sm_count, cudaStream_t stream);
 

@@ -567,11 +567,9 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
     if (n == 1) return cudaMemsetAsync(dist, 0, sizeof(double), stream);
     // many rows and a long dimension: exact integer Gram product on the tensor cores (HBM-bound);
     // short dimensions keep the FP32 difference form, whose per-term error does not rely on averaging
-    static const bool no_mma = std::getenv("GAR_K1_NO_MMA") != nullptr;   // tuning aid
-    static const bool no_umma = std::getenv("GAR_K1_NO_UMMA") != nullptr;  // tuning aid: mma.sync kernel instead of tcgen05
+    static const bool no_mma = std::getenv("GAR_K1_NO_MMA") != nullptr;   // tuning aid: CUDA-core kernel instead
     if (n > 16 && vec == 4 && d >= kMmaMinDim && !no_mma)
-        return no_umma ? launch_distances_mma(grads, n, d, ld, dist, ws, sm_count, stream)
-                       : launch_distances_umma(grads, n, d, ld, dist, ws, sm_count, stream);
+        return launch_distances_umma(grads, n, d, ld, dist, ws, sm_count, stream);
 #define GAR_K1_DIRECT(NV) case NV: return launch_direct_n<NV>(grads, d, ld, dist, ws, sm_count, stream, vec);
 #define GAR_K1_TILED(NBV)                                                                          \
     case NBV:                                                                                      \

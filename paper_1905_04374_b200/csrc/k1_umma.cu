@@ -2,9 +2,8 @@
 // Gram matrix on the fifth-generation tensor cores: tcgen05.mma, kind::i8, accumulators in
 // tensor memory.
 //
-// Arithmetic (the same exact scheme as the mma.sync kernel in k1_mma.cu).  Every row keeps a
-// running exponent E; a value x is rounded to the integer q = rint(x * 2^(148-E)), |q| < 2^22, and
-// q is split into three signed bytes q = l1 * 2^16 + l2 * 2^8 + l3.  With the byte matrices L1, L2,
+// Arithmetic.  Every row keeps a running exponent E; a value x is rounded to the integer
+// q = rint(x * 2^(148-E)), |q| <= 2^22 (a relative step of 2^-21 of the row's largest binade), and q is split into three signed bytes q = l1 * 2^16 + l2 * 2^8 + l3.  With the byte matrices L1, L2,
 // L3 (rows x columns) the Gram matrix of the rounded rows is
 //     sum_ab 2^(8(3-a)) 2^(8(3-b)) La Lb^T        (a, b = 1..3),
 // int8 x int8 products summed exactly in int32.  The six products with a <= b are formed, kept as
