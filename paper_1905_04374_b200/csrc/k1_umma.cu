@@ -139,6 +139,19 @@ __device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
     return r;
 }
+// Rounds the four values times `scale` to integers q through the 1.5 * 2^23 trick; w = q + 0x808080,
+// whose low three bytes, each xor 0x80, are the signed bytes l1, l2, l3 of q.  `outside` collects the
+// bits in which a result's sign and exponent field differ from those of [2^23, 2^24).
+__device__ __forceinline__ void quantise4(const float4& v, float scale, unsigned (&w)[4], unsigned& outside) {
+    const unsigned u0 = __float_as_uint(fmaf(v.x, scale, 12582912.0f)), u1 = __float_as_uint(fmaf(v.y, scale, 12582912.0f));
+    const unsigned u2 = __float_as_uint(fmaf(v.z, scale, 12582912.0f)), u3 = __float_as_uint(fmaf(v.w, scale, 12582912.0f));
+    outside |= (u0 ^ 0x4B000000u) | (u1 ^ 0x4B000000u);
+    outside |= (u2 ^ 0x4B000000u) | (u3 ^ 0x4B000000u);
+    w[0] = u0 + (0x00808080u - 0x4B400000u);
+    w[1] = u1 + (0x00808080u - 0x4B400000u);
+    w[2] = u2 + (0x00808080u - 0x4B400000u);
+    w[3] = u3 + (0x00808080u - 0x4B400000u);
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
 
@@ -205,6 +218,8 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         // incrementally: this loop's instruction count bounds the kernel.
         const int p = warp - KU_FIRST_PRODUCER;
         int row_exp[KU_JR];
+        float scale[KU_JR];                            // 2^(148 - row_exp)
+        int exp_stores = 0;                            // tile buffers that still lack the rows' current exponents
         const float* nextp[KU_JR];                     // this lane's float4 of the next slab to request
         bool valid[KU_JR];
         unsigned tile_off[KU_JR];                      // byte offset of (row, this lane's 4 columns) in a tile buffer
@@ -213,6 +228,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             const int row = p + jr * pw;
             valid[jr] = row < n;
             row_exp[jr] = KU_MIN_EXP;
+            scale[jr] = __uint_as_float(unsigned(275 - KU_MIN_EXP) << 23);
             nextp[jr] = g + int64_t(valid[jr] ? row : 0) * ld + first * KU_SLAB + 4 * lane;
             tile_off[jr] = unsigned(lane >> 2) * KU_LBO + unsigned(lane & 3) * 4 + unsigned(row) * 16;
         }
@@ -254,7 +270,6 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             req_off += stage_bytes;
             if (req_off == unsigned(NST) * stage_bytes) req_off = 0;
             float4 v[KU_JR];
-            int ex[KU_JR];
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
                 v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -265,46 +280,43 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             }
             cur_off += stage_bytes;
             if (cur_off == unsigned(NST) * stage_bytes) cur_off = 0;
+            // Common case: quantise with the rows' current scales.  x * scale + 1.5 * 2^23 lies in
+            // [2^23, 2^24) (exponent field 150) exactly when |x * scale| stays inside the 2^22 range
+            // of the three bytes; any other exponent field (a larger value, Inf, NaN) sends the warp
+            // to the path below, which finds the rows' new exponents.
+            unsigned w[KU_JR][4];
+            unsigned outside = 0u;
 #pragma unroll
-            for (int jr = 0; jr < KU_JR; ++jr) {
-                // largest |value| of the slab row; x * 0 is 0 for finite x and NaN otherwise, so the sum
-                // below is the maximum, or NaN (exponent field 255) when a value is Inf or NaN
-                const float m = fmaxf(fmaxf(fabsf(v[jr].x), fabsf(v[jr].y)), fmaxf(fabsf(v[jr].z), fabsf(v[jr].w)));
-                const float nf = fmaf(v[jr].x, 0.f, fmaf(v[jr].y, 0.f, fmaf(v[jr].z, 0.f, v[jr].w * 0.f)));
-                ex[jr] = int(__reduce_max_sync(0xffffffffu, __float_as_uint(m + nf)) >> 23);   // >= 255: not finite
-            }
-            bool grew = false, any_bad = false;
-            float scale[KU_JR];
-#pragma unroll
-            for (int jr = 0; jr < KU_JR; ++jr) {
-                const bool bad = ex[jr] >= 255;
-                const bool up = !bad && ex[jr] > row_exp[jr];
-                if (up) row_exp[jr] = ex[jr] + 1;                            // one binade of headroom
-                grew |= up;
-                any_bad |= bad;
-                scale[jr] = __uint_as_float(unsigned(275 - row_exp[jr]) << 23);   // 2^(148-E)
-            }
-            if (any_bad) {                                                   // rare: a row holds Inf or NaN
+            for (int jr = 0; jr < KU_JR; ++jr) quantise4(v[jr], scale[jr], w[jr], outside);
+            bool grew = false;
+            if (__any_sync(0xffffffffu, outside >= 0x00800000u)) {
+                int ex[KU_JR];
 #pragma unroll
                 for (int jr = 0; jr < KU_JR; ++jr) {
-                    const int row = p + jr * pw;
-                    if (ex[jr] >= 255) {
-                        v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);            // quantised as zeros, flagged
+                    // largest |value| of the slab row; x * 0 is 0 for finite x and NaN otherwise, so the sum
+                    // below is the maximum, or NaN (exponent field 255) when a value is Inf or NaN
+                    const float m = fmaxf(fmaxf(fabsf(v[jr].x), fabsf(v[jr].y)), fmaxf(fabsf(v[jr].z), fabsf(v[jr].w)));
+                    const float nf = fmaf(v[jr].x, 0.f, fmaf(v[jr].y, 0.f, fmaf(v[jr].z, 0.f, v[jr].w * 0.f)));
+                    ex[jr] = int(__reduce_max_sync(0xffffffffu, __float_as_uint(m + nf)) >> 23);   // >= 255: not finite
+                }
+#pragma unroll
+                for (int jr = 0; jr < KU_JR; ++jr) {
+                    const bool bad = ex[jr] >= 255;
+                    const bool up = !bad && ex[jr] > row_exp[jr];
+                    if (up) row_exp[jr] = ex[jr] + 1;                            // one binade of headroom
+                    grew |= up;
+                    scale[jr] = __uint_as_float(unsigned(275 - row_exp[jr]) << 23);   // 2^(148-E)
+                    if (bad) {                                                   // a row holds Inf or NaN:
+                        v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);                // quantised as zeros, flagged
+                        const int row = p + jr * pw;
                         if (lane == 0 && valid[jr]) {
                             if (row < 32) atomicOr(&sm.nonfinite_lo, 1u << row); else atomicOr(&sm.nonfinite_hi, 1u << (row - 32));
                         }
                     }
+                    unsigned unused = 0u;
+                    quantise4(v[jr], scale[jr], w[jr], unused);
                 }
-            }
-            unsigned w[KU_JR][4];
-#pragma unroll
-            for (int jr = 0; jr < KU_JR; ++jr) {
-                // round to nearest through the 1.5 * 2^23 trick; the low three bytes of (q + 0x808080),
-                // each xor 0x80, are the signed bytes l1, l2, l3
-                w[jr][0] = __float_as_uint(fmaf(v[jr].x, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
-                w[jr][1] = __float_as_uint(fmaf(v[jr].y, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
-                w[jr][2] = __float_as_uint(fmaf(v[jr].z, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
-                w[jr][3] = __float_as_uint(fmaf(v[jr].w, scale[jr], 12582912.0f)) + (0x00808080u - 0x4B400000u);
+                exp_stores = KU_NBUF;                // every tile buffer gets the new exponents once
             }
             // the MMAs that read this buffer three slabs ago are done
             if (!mbar_wait(&sm.empty[buf], empty_parity, error)) break;
@@ -317,7 +329,14 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
                     asm volatile("st.shared.b32 [%0], %1;" ::"r"(at), "r"(prmt(h01, h23, 0x5410u) ^ 0x80808080u) : "memory");             // l1
                     asm volatile("st.shared.b32 [%0+1024], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x7632u) ^ 0x80808080u) : "memory");        // l2: rows 64..
                     asm volatile("st.shared.b32 [%0+2048], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x5410u) ^ 0x80808080u) : "memory");        // l3: rows 128..
-                    if (lane == 0) sm.slab_exp[buf][p + jr * pw] = row_exp[jr];
+                }
+            }
+            if (exp_stores > 0) {                    // warp-uniform
+                --exp_stores;
+                if (lane == 0) {
+#pragma unroll
+                    for (int jr = 0; jr < KU_JR; ++jr)
+                        if (valid[jr]) sm.slab_exp[buf][p + jr * pw] = row_exp[jr];
                 }
             }
             if (grew && lane == 0) sm.grow[buf] = 1;
