@@ -1,0 +1,257 @@
+// Coordinate phase (Algorithm 1, multi-Bulyan: Median, Argpartition, Average), staged through
+// shared memory by bulk copies.
+//
+// A tile is KB_TC consecutive coordinates of every gradient the phase reads (the winners, and for
+// the pre-aggregating rules every gradient of some set: "staged rows").  One lane of a producer
+// warp fetches a tile with one bulk copy per staged row (KB_TC * 4 contiguous bytes each) into a
+// ring of stages; a stage's mbarrier counts the bytes in.  The compute threads own one coordinate
+// of the tile each: all values they need sit in shared memory at offsets that are fixed at compile
+// time for the winners (staged row s = slot s), so no address arithmetic, no load instruction per
+// gradient and no exposed global-memory latency is left in their loop.  Every gradient is read
+// from global memory exactly once.
+//
+// Pre-aggregation (G^agr[s] = mean over the set of slot s) follows the selection kernel's
+// summation plan (layout in gar.h), restated branch-free:
+//     T_s = T_{s-1} + cw_s * e_s        cw_s = 1 for a chained winner, else 0      (T_-1 = sum of base rows)
+//     a_s = (T_s + C[col_s]) / m_s
+// The corrections C (sums over the "loose" gradients) are evaluated first, once per correction slot
+// in slot order, into a private shared-memory column per thread; col_s names the latest one at or
+// before slot s (column 0 holds zero).
+#pragma once
+#include "k3_coordinate.cuh"
+
+namespace gar {
+
+constexpr int KB_TC = 256;                    // coordinates per tile = compute threads per CTA
+constexpr int KB_THREADS = KB_TC + 32;        // + the producer warp
+constexpr int KB_MAX_STAGES = 4;
+constexpr unsigned KB_SPIN_LIMIT = 1u << 22;  // polls of a barrier before a wait gives up
+constexpr int KB_BAR_COMPUTE = 1;             // named barrier of the compute warps
+constexpr int KB_ROW_BYTES = KB_TC * 4;
+
+struct alignas(16) KBSlot {
+    float cw;        // 1: the slot's winner joins the running sum here
+    float im;        // 1 / |set|
+    int   coff;      // byte offset of the slot's correction column
+    int   pad;
+};
+
+struct KBPlan {
+    unsigned long long full[KB_MAX_STAGES];   // bulk copies -> compute threads: the stage's bytes have landed
+    unsigned long long empty[KB_MAX_STAGES];  // compute warps -> producer: the stage has been read
+    KBSlot   slot[GAR_MAX_N];
+    int64_t  roff[GAR_MAX_N];                 // staged row -> element offset of its gradient
+    int      theta, beta, median_of_agr, lo_pads;
+    int      nrows, nbase, ncorr, nstages;
+    int      error;
+    int      loose_row[GAR_MAX_N];            // loose gradient -> staged row
+    int      saved_col[GAR_MAX_SAVED];
+    uint8_t  corr_src[GAR_MAX_N];             // GAR_SRC_ZERO, GAR_SRC_CONT or the column to start from
+    uint8_t  corr_nadd[GAR_MAX_N];
+};
+
+__device__ __forceinline__ unsigned kb_smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ bool kb_test(unsigned bar, unsigned parity) {
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait for the phase with the given parity (about a second at most); the thread sleeps
+// between polls so that a waiting warp leaves the issue slots to the computing ones.  False: the
+// wait gave up (error flag raised) or, unless `ignore_flag`, somebody else raised the flag.
+__device__ __forceinline__ bool kb_wait(unsigned bar, unsigned parity, volatile int* error, bool ignore_flag = false) {
+    for (unsigned spin = 0; spin < KB_SPIN_LIMIT; ++spin) {
+        if (kb_test(bar, parity)) return true;
+        if (!ignore_flag && *error) return false;
+        __nanosleep(100);
+    }
+    *error = 1;
+    return false;
+}
+
+// Dynamic shared memory: [staged-row indices of the plan's additions, 16-byte padded]
+// [correction columns (ncorr + 1) x KB_TC floats] [stages: nrows x KB_TC floats each].
+template <int P, bool EXACT, bool PREAGG>
+__global__ void __launch_bounds__(KB_THREADS)
+k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t* __restrict__ sel,
+        float* __restrict__ out, int pool_bytes) {
+    __shared__ KBPlan plan;
+    extern __shared__ __align__(128) unsigned char kb_dyn[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int theta = EXACT ? P : sel->theta;
+
+    // ---- plan -----------------------------------------------------------------------------
+    const int nbase = PREAGG ? sel->nbase : 0;
+    const int nloose = PREAGG ? sel->nloose : 0;
+    const int nadds = PREAGG ? sel->total_adds : 0;
+    for (int s = tid; s < GAR_MAX_N; s += KB_THREADS) {
+        KBSlot sl;
+        sl.cw = 0.0f; sl.im = 0.0f; sl.coff = 0; sl.pad = 0;
+        if (s < theta) {
+            const int r = theta - 1 - s;
+            plan.roff[s] = int64_t(sel->winners[r]) * ld;
+            sl.cw = ((sel->chain_mask >> s) & 1ull) ? 1.0f : 0.0f;
+            sl.im = 1.0f / float(sel->m[r]);
+        }
+        plan.slot[s] = sl;
+    }
+    for (int k = tid; k < nbase; k += KB_THREADS) plan.roff[theta + k] = int64_t(sel->base_rows[k]) * ld;
+    for (int u = tid; u < nloose; u += KB_THREADS) {        // a loose gradient that is also a winner shares its row
+        const int row = sel->loose_rows[u];
+        int match = -1;
+        for (int s = 0; s < theta; ++s)
+            if (sel->winners[theta - 1 - s] == row) match = s;
+        plan.loose_row[u] = match;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int nrows = theta + nbase;
+        for (int u = 0; u < nloose; ++u) {
+            if (plan.loose_row[u] < 0) {
+                plan.roff[nrows] = int64_t(sel->loose_rows[u]) * ld;
+                plan.loose_row[u] = nrows++;
+            }
+        }
+        plan.nrows = nrows;
+        plan.nbase = nbase;
+        plan.theta = theta;
+        plan.beta = sel->beta;
+        plan.median_of_agr = sel->median_of_agr;
+        plan.lo_pads = (P - 1) / 2 - (theta - 1) / 2;
+        plan.error = 0;
+        // corrections in slot order: column j + 1 holds the j-th one, column 0 is zero
+        int ncorr = 0, col = 0;
+        if (PREAGG) {
+            for (int s = 0; s < theta; ++s) {
+                if ((sel->corr_mask >> s) & 1ull) {
+                    const int src = sel->slot_src[s];
+                    plan.corr_src[ncorr] = uint8_t((src == GAR_SRC_ZERO || src == GAR_SRC_CONT) ? src : plan.saved_col[src]);
+                    plan.corr_nadd[ncorr] = sel->slot_nadd[s];
+                    ++ncorr;
+                    col = ncorr;
+                    const int sv = sel->slot_save[s];
+                    if (sv != GAR_SAVE_NONE) plan.saved_col[sv] = col;
+                }
+                plan.slot[s].coff = col * KB_ROW_BYTES;
+            }
+        }
+        plan.ncorr = ncorr;
+        const int fixed = ((nadds + 15) & ~15) + (ncorr + 1) * KB_ROW_BYTES;
+        int nst = (pool_bytes - fixed) / (nrows * KB_ROW_BYTES);
+        if (nst > KB_MAX_STAGES) nst = KB_MAX_STAGES;
+        plan.nstages = nst;
+        if (nst < 1) plan.error = 1;                   // cannot happen with the launcher's pool size
+        for (int st = 0; st < KB_MAX_STAGES; ++st) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(kb_smem_u32(&plan.full[st])), "r"(1u) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(kb_smem_u32(&plan.empty[st])), "r"(unsigned(KB_TC / 32)) : "memory");
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    uint8_t* const add_row = kb_dyn;
+    for (int k = tid; k < nadds; k += KB_THREADS) add_row[k] = uint8_t(plan.loose_row[sel->add_pos[k]]);
+    const int ncorr = plan.ncorr, nrows = plan.nrows, nstages = plan.nstages;
+    float* const ccol = reinterpret_cast<float*>(kb_dyn + ((nadds + 15) & ~15));
+    unsigned char* const stages = reinterpret_cast<unsigned char*>(ccol) + (ncorr + 1) * KB_ROW_BYTES;
+    const unsigned stage_bytes = unsigned(nrows) * KB_ROW_BYTES;
+    if (tid < KB_TC) ccol[tid] = 0.0f;
+    __syncthreads();
+    volatile int* error = &plan.error;
+
+    const int64_t first = blockIdx.x, step = gridDim.x;
+    const int64_t mine = first < ntiles ? (ntiles - first + step - 1) / step : 0;
+
+    if (warp == KB_TC / 32) {
+        // ================================================================ producer
+        // every lane fetches the staged rows lane, lane + 32, ...: a tile's copies leave together
+        if (!*error) {
+            int st = 0;
+            unsigned parity = 1;                     // the phase before the first one: the first nstages waits pass
+            int64_t i = 0;
+            for (; i < mine; ++i) {
+                if (!__all_sync(0xffffffffu, kb_wait(kb_smem_u32(&plan.empty[st]), parity, error))) break;
+                const unsigned bar = kb_smem_u32(&plan.full[st]);
+                if (lane == 0)
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(stage_bytes) : "memory");
+                __syncwarp();
+                const float* src = g + (first + i * step) * KB_TC;
+                const unsigned dst = kb_smem_u32(stages) + unsigned(st) * stage_bytes;
+                for (int r = lane; r < nrows; r += 32)
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(dst + unsigned(r) * KB_ROW_BYTES), "l"(src + plan.roff[r]), "r"(unsigned(KB_ROW_BYTES)), "r"(bar) : "memory");
+                if (++st == nstages) { st = 0; parity ^= 1u; }
+            }
+            // no copy may be in flight when the CTA leaves: wait (bounded) for the last tiles issued,
+            // also when a wait above gave up
+            for (int64_t j = i > nstages ? i - nstages : 0; j < i; ++j)
+                kb_wait(kb_smem_u32(&plan.full[j % nstages]), unsigned(j / nstages) & 1u, error, true);
+        }
+    } else {
+        // ================================================================ compute: one coordinate per thread
+        const int beta = plan.beta;
+        const float inv_beta = 1.0f / float(beta);
+        const int lo_pads = EXACT ? 0 : plan.lo_pads;
+        const bool med_agr = PREAGG && plan.median_of_agr != 0;
+        float* const mycol = ccol + tid;
+        int st = 0;
+        unsigned parity = 0;
+        bool ok = !*error;
+        for (int64_t i = 0; ok && i < mine; ++i) {
+            // one warp polls the stage's barrier, the others sleep in a hardware barrier meanwhile
+            if (warp == 0) kb_wait(kb_smem_u32(&plan.full[st]), parity, error);
+            unsigned failed;                      // the same answer in every compute thread
+            asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                         : "=r"(failed) : "r"(*error), "r"(KB_BAR_COMPUTE), "r"(KB_TC) : "memory");
+            if (failed) break;
+            const float* sv = reinterpret_cast<const float*>(stages + size_t(st) * stage_bytes) + tid;
+            float e[P][1], a[P][1];
+#pragma unroll
+            for (int s = 0; s < P; ++s) e[s][0] = (s < theta) ? sv[s * KB_TC] : 0.0f;
+            if constexpr (PREAGG) {
+                float T = 0.0f;
+                const float* bp = sv + theta * KB_TC;
+                int k = 0;
+                for (; k + 4 <= nbase; k += 4) {
+                    const float x0 = bp[0], x1 = bp[KB_TC], x2 = bp[2 * KB_TC], x3 = bp[3 * KB_TC];
+                    T += x0; T += x1; T += x2; T += x3;
+                    bp += 4 * KB_TC;
+                }
+                for (; k < nbase; ++k) { T += bp[0]; bp += KB_TC; }
+                float C = 0.0f;
+                int kadd = 0;
+                for (int j = 0; j < ncorr; ++j) {
+                    const int src = plan.corr_src[j];
+                    if (src == GAR_SRC_ZERO) C = 0.0f;
+                    else if (src != GAR_SRC_CONT) C = mycol[src * KB_TC];
+                    const int kend = kadd + plan.corr_nadd[j];
+                    for (; kadd < kend; ++kadd) C += sv[int(add_row[kadd]) * KB_TC];
+                    mycol[(j + 1) * KB_TC] = C;
+                }
+#pragma unroll
+                for (int s = 0; s < P; ++s) {
+                    const KBSlot sl = plan.slot[s];
+                    T = fmaf(e[s][0], sl.cw, T);
+                    const float c = *reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(mycol) + sl.coff);
+                    a[s][0] = (T + c) * sl.im;
+                }
+            } else {
+#pragma unroll
+                for (int s = 0; s < P; ++s) a[s][0] = e[s][0];
+            }
+            // the stage's values are in registers (or folded into T and C): hand it back
+            __syncwarp();
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(kb_smem_u32(&plan.empty[st])) : "memory");
+            float res[1];
+            k3_finish<P, 1>(e, a, theta, beta, inv_beta, lo_pads, med_agr, res);
+            out[(first + i * step) * KB_TC + tid] = res[0];
+            if (++st == nstages) { st = 0; parity ^= 1u; }
+        }
+    }
+    __syncthreads();
+    if (tid == 0 && plan.error) sel->status = GAR_ERR_TIMEOUT;
+}
+
+}  // namespace gar

@@ -132,6 +132,105 @@ template <int N, int V> __device__ __forceinline__ void median_network(float (&x
     median_network_apply<N, V>(x, std::make_index_sequence<MedianNet<N>::data.count>{});
 }
 
+// Last part of a coordinate's work, on V coordinates at once: M = lower median of the theta real
+// values of e (of a when median_of_a), then the average of the beta values of a closest to M
+// (Algorithm 1, multi-Bulyan: Median, Argpartition, Average).  e and a hold P slots of which the
+// first theta are real; e is destroyed.
+template <int P, int V>
+__device__ __forceinline__ void k3_finish(float (&e)[P][V], float (&a)[P][V], int theta, int beta, float inv_beta,
+                                          int lo_pads, bool median_of_a, float (&res)[V]) {
+    // median of the theta real values (lower middle), padding split around them
+    float srt[P][V];
+#pragma unroll
+    for (int s = 0; s < P; ++s) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const float real = median_of_a ? a[s][v] : e[s][v];
+            const float pad = (s - theta < lo_pads) ? -CUDART_INF_F : CUDART_INF_F;
+            srt[s][v] = (s < theta) ? real : pad;
+        }
+    }
+    median_network<P, V>(srt);
+    float key[P][V];
+#pragma unroll
+    for (int s = 0; s < P; ++s) {
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            key[s][v] = (s < theta) ? fabsf(a[s][v] - srt[(P - 1) / 2][v]) : CUDART_INF_F;
+    }
+
+    // The beta smallest keys.  beta == 1: the minimum key, then one scan that keeps the
+    // value of the highest slot holding it.  beta == 2, 3: the beta-th smallest key tau is
+    // found with min/max only and the values with key <= tau are summed with a 0/1 mask; if
+    // more values tie at tau than there is room for, or for larger beta, beta passes of
+    // arg-min pick them one by one.  Equal keys go to the earliest round = highest slot.
+    float sum[V];
+    bool need_passes = beta > 3;
+    if (beta == 1) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            float best = key[0][v];
+#pragma unroll
+            for (int s = 1; s < P; ++s) best = fminf(best, key[s][v]);
+            float ba = a[0][v];
+#pragma unroll
+            for (int s = 1; s < P; ++s) ba = (key[s][v] == best) ? a[s][v] : ba;
+            sum[v] = ba;
+        }
+    } else if (!need_passes) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            float t1 = CUDART_INF_F, t2 = CUDART_INF_F, t3 = CUDART_INF_F;   // three smallest keys so far
+#pragma unroll
+            for (int s = 0; s < P; ++s) {
+                const float k = key[s][v];
+                const float x = fmaxf(t1, k);
+                t1 = fminf(t1, k);
+                const float y = fmaxf(t2, x);
+                t2 = fminf(t2, x);
+                t3 = fminf(t3, y);
+            }
+            const float tau = beta == 2 ? t2 : t3;
+            float s_le = 0.0f, c_le = 0.0f;
+#pragma unroll
+            for (int s = 0; s < P; ++s) {
+                const float le = key[s][v] <= tau ? 1.0f : 0.0f;
+                s_le = fmaf(le, a[s][v], s_le);
+                c_le += le;
+            }
+            sum[v] = s_le;
+            // c_le > beta: several keys tie at tau and not all of them fit
+            // (a non-finite tau or value also lands here)
+            if (!(c_le == float(beta)) || !(fabsf(s_le) <= 3.0e38f)) need_passes = true;
+        }
+    }
+    if (need_passes) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) sum[v] = 0.0f;
+        for (int b = 0; b < beta; ++b) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                float best = key[P - 1][v], ba = a[P - 1][v];
+                int bi = P - 1;
+#pragma unroll
+                for (int s = P - 2; s >= 0; --s) {
+                    const bool take = key[s][v] < best;
+                    best = take ? key[s][v] : best;
+                    ba = take ? a[s][v] : ba;
+                    bi = take ? s : bi;
+                }
+                sum[v] += ba;
+                if (b + 1 < beta) {
+#pragma unroll
+                    for (int s = 0; s < P; ++s) key[s][v] = (s == bi) ? CUDART_INF_F : key[s][v];
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) res[v] = sum[v] * inv_beta;
+}
+
 __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* __restrict__ sel, int64_t ld, int P,
                                           bool preagg, int loose_cap) {
     const int tid = threadIdx.x;
@@ -303,103 +402,15 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
             }
         }
 
-        // median of the theta real values (lower middle), padding split around them
-        float srt[P][V];
-#pragma unroll
-        for (int s = 0; s < P; ++s) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const float real = (PREAGG && med_agr) ? a[s][v] : e[s][v];
-                const float pad = (s - theta < lo_pads) ? -CUDART_INF_F : CUDART_INF_F;
-                srt[s][v] = (s < theta) ? real : pad;
-            }
-        }
-        median_network<P, V>(srt);
-        float key[P][V];
-#pragma unroll
-        for (int s = 0; s < P; ++s) {
-#pragma unroll
-            for (int v = 0; v < V; ++v)
-                key[s][v] = (s < theta) ? fabsf(a[s][v] - srt[(P - 1) / 2][v]) : CUDART_INF_F;
-        }
-
-        // The beta smallest keys.  beta == 1: the minimum key, then one scan that keeps the
-        // value of the highest slot holding it.  beta == 2, 3: the beta-th smallest key tau is
-        // found with min/max only and the values with key <= tau are summed with a 0/1 mask; if
-        // more values tie at tau than there is room for, or for larger beta, beta passes of
-        // arg-min pick them one by one.  Equal keys go to the earliest round = highest slot.
-        float sum[V];
-        bool need_passes = beta > 3;
-        if (beta == 1) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                float best = key[0][v];
-#pragma unroll
-                for (int s = 1; s < P; ++s) best = fminf(best, key[s][v]);
-                float ba = a[0][v];
-#pragma unroll
-                for (int s = 1; s < P; ++s) ba = (key[s][v] == best) ? a[s][v] : ba;
-                sum[v] = ba;
-            }
-        } else if (!need_passes) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                float t1 = CUDART_INF_F, t2 = CUDART_INF_F, t3 = CUDART_INF_F;   // three smallest keys so far
-#pragma unroll
-                for (int s = 0; s < P; ++s) {
-                    const float k = key[s][v];
-                    const float x = fmaxf(t1, k);
-                    t1 = fminf(t1, k);
-                    const float y = fmaxf(t2, x);
-                    t2 = fminf(t2, x);
-                    t3 = fminf(t3, y);
-                }
-                const float tau = beta == 2 ? t2 : t3;
-                float s_le = 0.0f, c_le = 0.0f;
-#pragma unroll
-                for (int s = 0; s < P; ++s) {
-                    const float le = key[s][v] <= tau ? 1.0f : 0.0f;
-                    s_le = fmaf(le, a[s][v], s_le);
-                    c_le += le;
-                }
-                sum[v] = s_le;
-                // c_le > beta: several keys tie at tau and not all of them fit
-                // (a non-finite tau or value also lands here)
-                if (!(c_le == float(beta)) || !(fabsf(s_le) <= 3.0e38f)) need_passes = true;
-            }
-        }
-        if (need_passes) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) sum[v] = 0.0f;
-            for (int b = 0; b < beta; ++b) {
-#pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    float best = key[P - 1][v], ba = a[P - 1][v];
-                    int bi = P - 1;
-#pragma unroll
-                    for (int s = P - 2; s >= 0; --s) {
-                        const bool take = key[s][v] < best;
-                        best = take ? key[s][v] : best;
-                        ba = take ? a[s][v] : ba;
-                        bi = take ? s : bi;
-                    }
-                    sum[v] += ba;
-                    if (b + 1 < beta) {
-#pragma unroll
-                        for (int s = 0; s < P; ++s) key[s][v] = (s == bi) ? CUDART_INF_F : key[s][v];
-                    }
-                }
-            }
-        }
         float res[V];
-#pragma unroll
-        for (int v = 0; v < V; ++v) res[v] = sum[v] * inv_beta;
+        k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, PREAGG && med_agr, res);
         store_vec<V>(out + t, res);
     }
 }
 
 template <int P>
-cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
-                        int vec, float* out, int sm_count, cudaStream_t stream);
+cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
+                        int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
+template <int P> int bulk_ctas_for(int n, int theta);
 
 }  // namespace gar

@@ -1,7 +1,7 @@
 // One instantiation of the coordinate kernel per compiled slot count K3_P
 // (this file is compiled once for every entry of K3_P_LIST in k3_dispatch.cu;
 // K3_EXACT = 1 when the kernel is only used with theta == K3_P).
-#include "k3_coordinate.cuh"
+#include "k3_bulk.cuh"
 
 #if !defined(K3_P) || !defined(K3_EXACT)
 #error "compile with -DK3_P=<slot count> -DK3_EXACT=<0|1>"
@@ -21,8 +21,45 @@ static inline void preagg_shape(int loose_cap, int V, int* threads, size_t* smem
     *smem = per_thread * t;
 }
 
+// Shared memory the staged kernel needs for one stage in the worst case (every gradient staged,
+// a correction in every slot, theta * n additions in the plan).
+static inline size_t bulk_pool_min(int n, int theta) {
+    return size_t((theta * n + 15) & ~15) + size_t(theta + 1) * KB_ROW_BYTES + size_t(n) * KB_ROW_BYTES;
+}
+
+// Full tiles [0, ntiles * KB_TC) through the staged kernel, `ctas` CTAs per SM.
+template <int P, bool PREAGG>
+static cudaError_t run_bulk(const float* g, int n, int64_t ntiles, int64_t ld, const gar_selection_t* sel, int theta,
+                            int ctas, float* out, int sm_count, cudaStream_t stream) {
+    constexpr bool EXACT = (K3_EXACT != 0);
+    constexpr size_t kPerSm = 225 * 1024, kPerCta = 3584;      // static shared memory + the system's share, rounded up
+    const size_t pool_min = bulk_pool_min(n, theta);
+    size_t pool = (kPerSm / size_t(ctas) - kPerCta) & ~size_t(127);
+    const size_t pool_max = pool_min + size_t(KB_MAX_STAGES - 1) * n * KB_ROW_BYTES;
+    if (pool > pool_max) pool = pool_max;
+    if (pool < pool_min) return cudaErrorInvalidValue;
+    static size_t configured[64] = {0};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (dev < 0 || dev >= 64 || configured[dev] < pool) {
+        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(pool));
+        if (err != cudaSuccess) return err;
+        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                   cudaSharedmemCarveoutMaxShared);
+        if (err != cudaSuccess) return err;
+        if (dev >= 0 && dev < 64) configured[dev] = pool;
+    }
+    int64_t grid = int64_t(sm_count) * ctas;
+    if (grid > ntiles) grid = ntiles;
+    k3_bulk<P, EXACT, PREAGG><<<unsigned(grid), KB_THREADS, pool, stream>>>(g, ntiles, ld, const_cast<gar_selection_t*>(sel),
+                                                                             out, int(pool));
+    return cudaGetLastError();
+}
+
+// Coordinates [t0, d): t0 is a multiple of 4.
 template <int P, bool PREAGG, int V>
-static cudaError_t run(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, float* out,
+static cudaError_t run(const float* g, int n, int64_t t0, int64_t d, int64_t ld, const gar_selection_t* sel, float* out,
                        int sm_count, cudaStream_t stream) {
     constexpr bool EXACT = (K3_EXACT != 0);
     int threads = K3_THREADS, threads1 = K3_THREADS;
@@ -48,13 +85,13 @@ static cudaError_t run(const float* g, int n, int64_t d, int64_t ld, const gar_s
             if (dev >= 0 && dev < 64) configured[dev] = true;
         }
     }
-    const int64_t d_vec = d - d % V;
-    if (d_vec > 0) {
-        const int64_t nvec = d_vec / V;
+    const int64_t d_vec = d - (d - t0) % V;
+    if (d_vec > t0) {
+        const int64_t nvec = (d_vec - t0) / V;
         int64_t blocks = (nvec + threads - 1) / threads;
         const int64_t cap = int64_t(sm_count) * 8;
         if (blocks > cap) blocks = cap;
-        k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, 0, d_vec, ld, sel, out,
+        k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, t0, d_vec, ld, sel, out,
                                                                                          loose_cap);
     }
     if (d_vec < d) {   // ragged tail (only when ld > d): scalar kernel on the last d % V coordinates
@@ -64,19 +101,37 @@ static cudaError_t run(const float* g, int n, int64_t d, int64_t ld, const gar_s
 }
 
 template <>
-cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int preagg,
-                              int vec, float* out, int sm_count, cudaStream_t stream) {
+cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
+                              int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream) {
+    int64_t t0 = 0;
+    if (bulk_ctas > 0 && d >= KB_TC) {           // whole tiles staged through shared memory, the rest below
+        const int64_t ntiles = d / KB_TC;
+        const cudaError_t err = preagg ? run_bulk<K3_P, true>(g, n, ntiles, ld, sel, theta, bulk_ctas, out, sm_count, stream)
+                                       : run_bulk<K3_P, false>(g, n, ntiles, ld, sel, theta, bulk_ctas, out, sm_count, stream);
+        if (err != cudaSuccess) return err;
+        t0 = ntiles * KB_TC;
+        if (t0 == d) return cudaSuccess;
+    }
     // 4-wide vectors are only compiled for small slot counts (register budget)
     constexpr bool kWide = (K3_P <= 8);
     if (vec == 4 && !kWide) vec = 2;
     if (preagg) {
-        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, d, ld, sel, out, sm_count, stream);
-        if (vec == 2) return run<K3_P, true, 2>(g, n, d, ld, sel, out, sm_count, stream);
-        return run<K3_P, true, 1>(g, n, d, ld, sel, out, sm_count, stream);
+        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, t0, d, ld, sel, out, sm_count, stream);
+        if (vec == 2) return run<K3_P, true, 2>(g, n, t0, d, ld, sel, out, sm_count, stream);
+        return run<K3_P, true, 1>(g, n, t0, d, ld, sel, out, sm_count, stream);
     }
-    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, d, ld, sel, out, sm_count, stream);
-    if (vec == 2) return run<K3_P, false, 2>(g, n, d, ld, sel, out, sm_count, stream);
-    return run<K3_P, false, 1>(g, n, d, ld, sel, out, sm_count, stream);
+    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, t0, d, ld, sel, out, sm_count, stream);
+    if (vec == 2) return run<K3_P, false, 2>(g, n, t0, d, ld, sel, out, sm_count, stream);
+    return run<K3_P, false, 1>(g, n, t0, d, ld, sel, out, sm_count, stream);
+}
+
+// CTAs per SM the staged kernel would get for n gradients and theta slots (0: it cannot run).
+template <>
+int bulk_ctas_for<K3_P>(int n, int theta) {
+    const size_t per_cta = bulk_pool_min(n, theta) + 3584;
+    int ctas = int((225 * 1024) / per_cta);
+    const int by_threads = 2048 / KB_THREADS;
+    return ctas < by_threads ? ctas : by_threads;
 }
 
 }  // namespace gar
