@@ -46,7 +46,7 @@ constexpr int KU_SET_COLS = 256;             // tensor-memory columns per accumu
 constexpr int KU_FLUSH_WARPS = 4;            // warps 0..3: tensor-memory lanes 32 w .. 32 w + 31
 constexpr int KU_MMA_WARP = 4;
 constexpr int KU_FIRST_PRODUCER = 5;
-constexpr unsigned KU_SPIN_LIMIT = 1u << 22; // polls of a barrier before a wait gives up (a few tenths of a second)
+constexpr unsigned KU_SPIN_LIMIT = 1u << 20; // suspended waits of a barrier before a wait gives up
 constexpr int KU_BAR_FLUSH = 1;              // named barrier of the flush warps
 constexpr int KU_TRI = 2080;
 
@@ -73,21 +73,23 @@ __device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned coun
 __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
+// One wait for the phase with the given parity: the thread is suspended in the barrier unit until the
+// phase completes or a hardware time limit passes, whichever comes first; true if it completed.
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
     unsigned done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                  : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return done != 0;
 }
-// Bounded wait for the phase with the given parity, the same answer in every lane of the warp.
+// Bounded wait for the phase with the given parity, the same answer in every lane of the warp.  A
+// waiting warp sleeps in the barrier unit and leaves the issue slots to the working ones.
 // False: the wait gave up (error flag raised) or another role raised the flag.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* error,
-                                          unsigned sleep_ns = 40, unsigned limit = KU_SPIN_LIMIT) {
+                                          unsigned limit = KU_SPIN_LIMIT) {
     bool ok = false;
     for (unsigned spin = 0; spin < limit; ++spin) {
-        if (mbar_test(bar, parity)) { ok = true; break; }
+        if (mbar_try_wait(bar, parity)) { ok = true; break; }
         if (*error) break;
-        if (spin > 32) __nanosleep(sleep_ns);
         if (spin + 1 == limit) *error = 1;
     }
     return __all_sync(0xffffffffu, ok);
@@ -414,7 +416,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         for (int k = 0;; ++k) {
             const int set = k & 1;
             // a set closes rarely: poll slowly; then agree over the four warps (they meet at named barriers below)
-            const bool ok = mbar_wait(&sm.accfull[set], unsigned(k >> 1) & 1u, error, 1000u, 1u << 20);
+            const bool ok = mbar_wait(&sm.accfull[set], unsigned(k >> 1) & 1u, error);
             unsigned all_ok;
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(all_ok) : "r"(unsigned(ok)), "r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");

@@ -25,7 +25,7 @@ namespace gar {
 constexpr int KB_TC = 256;                    // coordinates per tile = compute threads per CTA
 constexpr int KB_THREADS = KB_TC + 32;        // + the producer warp
 constexpr int KB_MAX_STAGES = 4;
-constexpr unsigned KB_SPIN_LIMIT = 1u << 22;  // polls of a barrier before a wait gives up
+constexpr unsigned KB_SPIN_LIMIT = 1u << 20;  // suspended waits of a barrier before a wait gives up
 constexpr int KB_BAR_COMPUTE = 1;             // named barrier of the compute warps
 constexpr int KB_ROW_BYTES = KB_TC * 4;
 
@@ -46,26 +46,27 @@ struct KBPlan {
     int      error;
     int      loose_row[GAR_MAX_N];            // loose gradient -> staged row
     int      saved_col[GAR_MAX_SAVED];
-    uint8_t  corr_src[GAR_MAX_N];             // GAR_SRC_ZERO, GAR_SRC_CONT or the column to start from
+    uint8_t  corr_src[GAR_MAX_N];             // column the correction starts from
     uint8_t  corr_nadd[GAR_MAX_N];
 };
 
 __device__ __forceinline__ unsigned kb_smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
 
-__device__ __forceinline__ bool kb_test(unsigned bar, unsigned parity) {
+// One wait for the phase with the given parity: the thread is suspended in the barrier unit until the
+// phase completes or a hardware time limit passes, whichever comes first; true if it completed.
+__device__ __forceinline__ bool kb_try_wait(unsigned bar, unsigned parity) {
     unsigned done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                  : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     return done != 0;
 }
-// Bounded wait for the phase with the given parity (about a second at most); the thread sleeps
-// between polls so that a waiting warp leaves the issue slots to the computing ones.  False: the
-// wait gave up (error flag raised) or, unless `ignore_flag`, somebody else raised the flag.
+// Bounded wait for the phase with the given parity; a waiting warp sleeps in the barrier unit and
+// leaves the issue slots to the computing ones.  False: the wait gave up (error flag raised) or,
+// unless `ignore_flag`, somebody else raised the flag.
 __device__ __forceinline__ bool kb_wait(unsigned bar, unsigned parity, volatile int* error, bool ignore_flag = false) {
     for (unsigned spin = 0; spin < KB_SPIN_LIMIT; ++spin) {
-        if (kb_test(bar, parity)) return true;
+        if (kb_try_wait(bar, parity)) return true;
         if (!ignore_flag && *error) return false;
-        __nanosleep(100);
     }
     *error = 1;
     return false;
@@ -121,16 +122,23 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
         plan.median_of_agr = sel->median_of_agr;
         plan.lo_pads = (P - 1) / 2 - (theta - 1) / 2;
         plan.error = 0;
-        // corrections in slot order: column j + 1 holds the j-th one, column 0 is zero
+        // Corrections: column 0 holds zero, column j + 1 the j-th sum that has to be formed (a slot
+        // that adds loose gradients).  A slot that only restarts from zero, continues, or takes up
+        // a saved sum just names the column that already holds its value.
         int ncorr = 0, col = 0;
         if (PREAGG) {
             for (int s = 0; s < theta; ++s) {
                 if ((sel->corr_mask >> s) & 1ull) {
                     const int src = sel->slot_src[s];
-                    plan.corr_src[ncorr] = uint8_t((src == GAR_SRC_ZERO || src == GAR_SRC_CONT) ? src : plan.saved_col[src]);
-                    plan.corr_nadd[ncorr] = sel->slot_nadd[s];
-                    ++ncorr;
-                    col = ncorr;
+                    const int from = src == GAR_SRC_ZERO ? 0 : (src == GAR_SRC_CONT ? col : plan.saved_col[src]);
+                    const int nadd = sel->slot_nadd[s];
+                    if (nadd == 0) {
+                        col = from;
+                    } else {
+                        plan.corr_src[ncorr] = uint8_t(from);
+                        plan.corr_nadd[ncorr] = uint8_t(nadd);
+                        col = ++ncorr;
+                    }
                     const int sv = sel->slot_save[s];
                     if (sv != GAR_SAVE_NONE) plan.saved_col[sv] = col;
                 }
@@ -219,22 +227,19 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
                     bp += 4 * KB_TC;
                 }
                 for (; k < nbase; ++k) { T += bp[0]; bp += KB_TC; }
-                float C = 0.0f;
                 int kadd = 0;
                 for (int j = 0; j < ncorr; ++j) {
-                    const int src = plan.corr_src[j];
-                    if (src == GAR_SRC_ZERO) C = 0.0f;
-                    else if (src != GAR_SRC_CONT) C = mycol[src * KB_TC];
+                    float C = mycol[int(plan.corr_src[j]) * KB_TC];
                     const int kend = kadd + plan.corr_nadd[j];
                     for (; kadd < kend; ++kadd) C += sv[int(add_row[kadd]) * KB_TC];
                     mycol[(j + 1) * KB_TC] = C;
                 }
 #pragma unroll
                 for (int s = 0; s < P; ++s) {
-                    const KBSlot sl = plan.slot[s];
-                    T = fmaf(e[s][0], sl.cw, T);
-                    const float c = *reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(mycol) + sl.coff);
-                    a[s][0] = (T + c) * sl.im;
+                    const float4 sl = *reinterpret_cast<const float4*>(&plan.slot[s]);      // cw, im, coff
+                    T = fmaf(e[s][0], sl.x, T);
+                    const float c = *reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(mycol) + __float_as_int(sl.z));
+                    a[s][0] = (T + c) * sl.y;
                 }
             } else {
 #pragma unroll

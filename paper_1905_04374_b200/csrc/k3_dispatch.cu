@@ -40,11 +40,12 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
         const int want = std::atoi(env);
         if (want == 1 || want == 2 || want == 4) vec = want < vec_max ? want : vec_max;
     }
-    // Staging through shared memory by bulk copies needs 16-byte aligned row segments; it pays from
-    // a handful of slots on (below, the register kernel with 4-wide loads is at least as fast).
+    // Staging through shared memory by bulk copies needs 16-byte aligned row segments.  It pays where
+    // the register kernel has to fall back to narrow loads: from 13 slots on with pre-aggregation,
+    // from 25 on without (below, the register kernel with 2- or 4-wide loads is at least as fast).
     static const char* env_bulk = std::getenv("GAR_K3_BULK");          // tuning aids: 0 = off, else the slot count it starts at
     static const char* env_ctas = std::getenv("GAR_K3_BULK_CTAS");     // CTAs per SM
-    int bulk_from = 10;
+    int bulk_from = preagg ? 13 : 25;
     if (env_bulk) bulk_from = std::atoi(env_bulk) > 0 ? std::atoi(env_bulk) : 1 << 30;
     const bool bulk = vec_max == 4 && theta >= bulk_from;
 #define K3_TRY(P)                                                                                              \
