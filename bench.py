@@ -24,6 +24,9 @@ if ROOT not in sys.path:
 METRIC = "multi_bulyan_aggregations_per_sec"
 UNIT = "aggregations/s"
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) per coordinate of the dominant kernels, from the ncu captures under
+# profiles/ (kernel, n) -> bytes; a kernel that changed since its capture has no entry.
+NCU_DRAM_BYTES_PER_COORD = {}
 
 
 def measured_hbm_peak():
@@ -242,8 +245,7 @@ def run_ours(args):
     achieved = kernels[dom]["gbs"]
     # DRAM bytes per coordinate from the committed ncu captures (profiles/), taken on a smaller d of
     # the same kernel and scaled by d; None where no capture of the current kernel exists
-    ncu_bytes_per_coord = {("k1_distances", 39): 317.0e6 / 2.0e6, ("k3_coordinate", 39): 240.6e6 / 2.0e6, ("k3_coordinate", 51): 302.3e6 / 1.5e6,
-                           ("k1_distances", 15): 244.4e6 / 4.0e6, ("k3_coordinate", 15): 172.0e6 / 4.0e6}
+    ncu_bytes_per_coord = NCU_DRAM_BYTES_PER_COORD
     per_coord = ncu_bytes_per_coord.get((dom, n))
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_kind": peak_kind,
@@ -260,6 +262,18 @@ def run_ours(args):
     }
     path["frac_of_nominal_8TBs"] = path["effective_gbs"] / NOMINAL_HBM_GBS
     path["frac_of_measured_peak"] = path["effective_gbs"] / peak
+
+    # ---- the same workload under the rule the benchmark spec's summary describes (theta = n - 2f
+    # iterated Krum winners, beta = theta - 2f, no pre-aggregation): GAR_BULYAN
+    k3b_sel = pkg.new_selection(dev)
+    pkg.gar_select("bulyan", dmat, n, f, sel=k3b_sel)
+    k3b_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, k3b_sel, theta_b, 0, out=out), reps, stream)
+    bulyan_ms = event_time_ms(lambda: pkg.gar_aggregate("bulyan", G, f, out=out), reps, stream)
+    variant = {"rule": "bulyan", "theta": theta_b, "beta": pkg.gar_beta("bulyan", n, f), "ms_per_aggregation": bulyan_ms,
+               "aggregations_per_sec": 1e3 / bulyan_ms, "k3_coordinate_ms": k3b_ms,
+               "effective_gbs": path_bytes_northstar / (bulyan_ms * 1e-3) / 1e9,
+               "frac_of_measured_peak": path_bytes_northstar / (bulyan_ms * 1e-3) / 1e9 / peak,
+               "frac_of_nominal_8TBs": path_bytes_northstar / (bulyan_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS}
 
     # ---- end to end through the host entry point (pinned host buffers, copies timed)
     e2e = None
@@ -289,8 +303,9 @@ def run_ours(args):
                    "beta": pkg.gar_beta("multi_bulyan", n, f), "parallelism": f"replicas x{world}",
                    "l2": "input (%.2f GB) larger than L2; no flush" % (4e-9 * n * d) if 4 * n * d > 2.6e8
                    else "input fits L2; not flushed between steps"},
-        "roofline": roofline, "path": path, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e,
-        "gpu_launches": 3 * args.steps, "clocks": clocks.summary(),
+        "roofline": roofline, "path": path, "kernels": kernels, "variant_bulyan": variant, "cpu_baseline": cpu, "e2e": e2e,
+        # distances, selection, coordinate phase (+ one more coordinate kernel for a ragged tail)
+        "gpu_launches": (3 + (1 if d % 256 else 0)) * args.steps, "clocks": clocks.summary(),
     }
     print(json.dumps(line), flush=True)
     if world > 1:

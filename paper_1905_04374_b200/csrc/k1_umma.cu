@@ -162,7 +162,8 @@ __device__ __forceinline__ int tri_slot(int i, int j) { return i * 64 - (i * (i 
 
 // Shared memory: KUSmem, the byte-tile buffers, px and pz (2 x 64 x 64 doubles, stored transposed:
 // [j][i]), the raw ring float4 [NST][3 * producer warps][32].
-template <int NST, int MAXT>
+// FULL: n is a multiple of KU_JR, every producer warp owns KU_JR real rows (no per-row tests).
+template <int NST, int MAXT, bool FULL>
 __global__ void __launch_bounds__(MAXT, 1)
 k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
         double* __restrict__ partials, unsigned int* __restrict__ ticket,
@@ -228,7 +229,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 #pragma unroll
         for (int jr = 0; jr < KU_JR; ++jr) {
             const int row = p + jr * pw;
-            valid[jr] = row < n;
+            valid[jr] = FULL || row < n;
             row_exp[jr] = KU_MIN_EXP;
             scale[jr] = __uint_as_float(unsigned(275 - KU_MIN_EXP) << 23);
             nextp[jr] = g + int64_t(valid[jr] ? row : 0) * ld + first * KU_SLAB + 4 * lane;
@@ -540,7 +541,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     if (tid == 0) *ticket = 0u;               // ready for the next call
 }
 
-template <int NST, int MAXT>
+template <int NST, int MAXT, bool FULL>
 cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                       int pw, size_t smem, cudaStream_t stream) {
     static size_t configured[64] = {0};                        // dynamic shared memory the kernel is allowed, per device
@@ -548,7 +549,7 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64 || configured[dev] < smem) {
-        err = cudaFuncSetAttribute(k1_umma<NST, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        err = cudaFuncSetAttribute(k1_umma<NST, MAXT, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = smem;
     }
@@ -558,7 +559,7 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     int64_t grid = sm_count;
     if (grid > kMaxCtasK1) grid = kMaxCtasK1;
     if (grid > nslabs) grid = nslabs;
-    k1_umma<NST, MAXT><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
+    k1_umma<NST, MAXT, FULL><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
         g, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error());
     return cudaGetLastError();
 }
@@ -576,7 +577,11 @@ cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t 
     int nst = 4;
     while (nst > 2 && fixed + nst * stage > kSmemMax) --nst;   // deepest raw ring that fits
     const size_t smem = fixed + nst * stage;
-#define GAR_KU(NSTV, MAXTV) return launch_ku<NSTV, MAXTV>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream)
+#define GAR_KU(NSTV, MAXTV)                                                                                 \
+    do {                                                                                                    \
+        if (n == KU_JR * pw) return launch_ku<NSTV, MAXTV, true>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream); \
+        return launch_ku<NSTV, MAXTV, false>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream);           \
+    } while (0)
     if (pw <= 14) { if (nst == 4) GAR_KU(4, kSmall); if (nst == 3) GAR_KU(3, kSmall); GAR_KU(2, kSmall); }
     if (nst == 4) GAR_KU(4, kLarge);
     if (nst == 3) GAR_KU(3, kLarge);
