@@ -1,11 +1,11 @@
 // Coordinate phase (Algorithm 1, multi-Bulyan: Median, Argpartition, Average), staged through
 // shared memory by bulk copies.
 //
-// A tile is KB_TC consecutive coordinates of every gradient the phase reads (the winners, and for
+// A tile is TC consecutive coordinates of every gradient the phase reads (the winners, and for
 // the pre-aggregating rules every gradient of some set: "staged rows").  One lane of a producer
-// warp fetches a tile with one bulk copy per staged row (KB_TC * 4 contiguous bytes each) into a
-// ring of stages; a stage's mbarrier counts the bytes in.  The compute threads own one coordinate
-// of the tile each: all values they need sit in shared memory at offsets that are fixed at compile
+// warp fetches a tile with one bulk copy per staged row (TC * 4 contiguous bytes each) into a
+// ring of stages; a stage's mbarrier counts the bytes in.  The compute threads own V adjacent
+// coordinates of the tile each (V = 4, 2, 1 as the slot count grows and registers get scarce): all values they need sit in shared memory at offsets that are fixed at compile
 // time for the winners (staged row s = slot s), so no address arithmetic, no load instruction per
 // gradient and no exposed global-memory latency is left in their loop.  Every gradient is read
 // from global memory exactly once.
@@ -22,12 +22,16 @@
 
 namespace gar {
 
-constexpr int KB_TC = 256;                    // coordinates per tile = compute threads per CTA
-constexpr int KB_THREADS = KB_TC + 32;        // + the producer warp
+// Shape of a CTA that gives every compute thread V adjacent coordinates of a tile.
+template <int V> struct KBShape {
+    static constexpr int CT = V == 1 ? 256 : 128;       // compute threads
+    static constexpr int TC = CT * V;                   // coordinates per tile
+    static constexpr int THREADS = CT + 32;             // + the producer warp
+    static constexpr int ROW_BYTES = TC * 4;            // one staged row of a tile (one bulk copy)
+};
 constexpr int KB_MAX_STAGES = 4;
 constexpr unsigned KB_SPIN_LIMIT = 1u << 20;  // suspended waits of a barrier before a wait gives up
 constexpr int KB_BAR_COMPUTE = 1;             // named barrier of the compute warps
-constexpr int KB_ROW_BYTES = KB_TC * 4;
 
 struct alignas(16) KBSlot {
     float cw;        // 1: the slot's winner joins the running sum here
@@ -73,11 +77,13 @@ __device__ __forceinline__ bool kb_wait(unsigned bar, unsigned parity, volatile 
 }
 
 // Dynamic shared memory: [staged-row indices of the plan's additions, 16-byte padded]
-// [correction columns (ncorr + 1) x KB_TC floats] [stages: nrows x KB_TC floats each].
-template <int P, bool EXACT, bool PREAGG>
-__global__ void __launch_bounds__(KB_THREADS)
+// [correction columns (ncorr + 1) x TC floats] [stages: nrows x TC floats each].
+template <int P, bool EXACT, bool PREAGG, int V>
+__global__ void __launch_bounds__(KBShape<V>::THREADS)
 k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t* __restrict__ sel,
         float* __restrict__ out, int pool_bytes) {
+    constexpr int KB_TC = KBShape<V>::TC, KB_CT = KBShape<V>::CT, KB_THREADS = KBShape<V>::THREADS;
+    constexpr int KB_ROW_BYTES = KBShape<V>::ROW_BYTES;
     __shared__ KBPlan plan;
     extern __shared__ __align__(128) unsigned char kb_dyn[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -153,7 +159,7 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
         if (nst < 1) plan.error = 1;                   // cannot happen with the launcher's pool size
         for (int st = 0; st < KB_MAX_STAGES; ++st) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(kb_smem_u32(&plan.full[st])), "r"(1u) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(kb_smem_u32(&plan.empty[st])), "r"(unsigned(KB_TC / 32)) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(kb_smem_u32(&plan.empty[st])), "r"(unsigned(KB_CT / 32)) : "memory");
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -164,14 +170,14 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
     float* const ccol = reinterpret_cast<float*>(kb_dyn + ((nadds + 15) & ~15));
     unsigned char* const stages = reinterpret_cast<unsigned char*>(ccol) + (ncorr + 1) * KB_ROW_BYTES;
     const unsigned stage_bytes = unsigned(nrows) * KB_ROW_BYTES;
-    if (tid < KB_TC) ccol[tid] = 0.0f;
+    for (int c = tid; c < KB_TC; c += KB_THREADS) ccol[c] = 0.0f;
     __syncthreads();
     volatile int* error = &plan.error;
 
     const int64_t first = blockIdx.x, step = gridDim.x;
     const int64_t mine = first < ntiles ? (ntiles - first + step - 1) / step : 0;
 
-    if (warp == KB_TC / 32) {
+    if (warp == KB_CT / 32) {
         // ================================================================ producer
         // every lane fetches the staged rows lane, lane + 32, ...: a tile's copies leave together
         if (!*error) {
@@ -197,12 +203,12 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
                 kb_wait(kb_smem_u32(&plan.full[j % nstages]), unsigned(j / nstages) & 1u, error, true);
         }
     } else {
-        // ================================================================ compute: one coordinate per thread
+        // ================================================================ compute: V coordinates per thread
         const int beta = plan.beta;
         const float inv_beta = 1.0f / float(beta);
         const int lo_pads = EXACT ? 0 : plan.lo_pads;
         const bool med_agr = PREAGG && plan.median_of_agr != 0;
-        float* const mycol = ccol + tid;
+        float* const mycol = ccol + tid * V;
         int st = 0;
         unsigned parity = 0;
         bool ok = !*error;
@@ -211,47 +217,77 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
             if (warp == 0) kb_wait(kb_smem_u32(&plan.full[st]), parity, error);
             unsigned failed;                      // the same answer in every compute thread
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                         : "=r"(failed) : "r"(*error), "r"(KB_BAR_COMPUTE), "r"(KB_TC) : "memory");
+                         : "=r"(failed) : "r"(*error), "r"(KB_BAR_COMPUTE), "r"(KB_CT) : "memory");
             if (failed) break;
-            const float* sv = reinterpret_cast<const float*>(stages + size_t(st) * stage_bytes) + tid;
-            float e[P][1], a[P][1];
+            const float* sv = reinterpret_cast<const float*>(stages + size_t(st) * stage_bytes) + tid * V;
+            float e[P][V], a[P][V];
 #pragma unroll
-            for (int s = 0; s < P; ++s) e[s][0] = (s < theta) ? sv[s * KB_TC] : 0.0f;
+            for (int s = 0; s < P; ++s) {
+                if (s < theta) {
+                    read_vec<V>(sv + s * KB_TC, e[s]);
+                } else {
+#pragma unroll
+                    for (int v = 0; v < V; ++v) e[s][v] = 0.0f;
+                }
+            }
             if constexpr (PREAGG) {
-                float T = 0.0f;
+                float T[V];
+#pragma unroll
+                for (int v = 0; v < V; ++v) T[v] = 0.0f;
                 const float* bp = sv + theta * KB_TC;
                 int k = 0;
                 for (; k + 4 <= nbase; k += 4) {
-                    const float x0 = bp[0], x1 = bp[KB_TC], x2 = bp[2 * KB_TC], x3 = bp[3 * KB_TC];
-                    T += x0; T += x1; T += x2; T += x3;
+                    float x0[V], x1[V], x2[V], x3[V];
+                    read_vec<V>(bp, x0); read_vec<V>(bp + KB_TC, x1); read_vec<V>(bp + 2 * KB_TC, x2); read_vec<V>(bp + 3 * KB_TC, x3);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) { T[v] += x0[v]; T[v] += x1[v]; T[v] += x2[v]; T[v] += x3[v]; }
                     bp += 4 * KB_TC;
                 }
-                for (; k < nbase; ++k) { T += bp[0]; bp += KB_TC; }
+                for (; k < nbase; ++k) {
+                    float x0[V];
+                    read_vec<V>(bp, x0);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) T[v] += x0[v];
+                    bp += KB_TC;
+                }
                 int kadd = 0;
                 for (int j = 0; j < ncorr; ++j) {
-                    float C = mycol[int(plan.corr_src[j]) * KB_TC];
+                    float C[V];
+                    read_vec<V>(mycol + int(plan.corr_src[j]) * KB_TC, C);
                     const int kend = kadd + plan.corr_nadd[j];
-                    for (; kadd < kend; ++kadd) C += sv[int(add_row[kadd]) * KB_TC];
-                    mycol[(j + 1) * KB_TC] = C;
+                    for (; kadd < kend; ++kadd) {
+                        float x[V];
+                        read_vec<V>(sv + int(add_row[kadd]) * KB_TC, x);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) C[v] += x[v];
+                    }
+                    store_vec<V>(mycol + (j + 1) * KB_TC, C);
                 }
 #pragma unroll
                 for (int s = 0; s < P; ++s) {
                     const float4 sl = *reinterpret_cast<const float4*>(&plan.slot[s]);      // cw, im, coff
-                    T = fmaf(e[s][0], sl.x, T);
-                    const float c = *reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(mycol) + __float_as_int(sl.z));
-                    a[s][0] = (T + c) * sl.y;
+                    float c[V];
+                    read_vec<V>(reinterpret_cast<const float*>(reinterpret_cast<const unsigned char*>(mycol) + __float_as_int(sl.z)), c);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        T[v] = fmaf(e[s][v], sl.x, T[v]);
+                        a[s][v] = (T[v] + c[v]) * sl.y;
+                    }
                 }
             } else {
 #pragma unroll
-                for (int s = 0; s < P; ++s) a[s][0] = e[s][0];
+                for (int s = 0; s < P; ++s) {
+#pragma unroll
+                    for (int v = 0; v < V; ++v) a[s][v] = e[s][v];
+                }
             }
             // the stage's values are in registers (or folded into T and C): hand it back
             __syncwarp();
             if (lane == 0)
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(kb_smem_u32(&plan.empty[st])) : "memory");
-            float res[1];
-            k3_finish<P, 1>(e, a, theta, beta, inv_beta, lo_pads, med_agr, res);
-            out[(first + i * step) * KB_TC + tid] = res[0];
+            float res[V];
+            k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, med_agr, res);
+            store_vec<V>(out + (first + i * step) * KB_TC + tid * V, res);
             if (++st == nstages) { st = 0; parity ^= 1u; }
         }
     }

@@ -411,6 +411,6 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
 template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
                         int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
-template <int P> int bulk_ctas_for(int n, int theta);
+template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 
 }  // namespace gar

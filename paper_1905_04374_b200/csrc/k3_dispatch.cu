@@ -16,12 +16,12 @@ namespace gar {
 template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
                         int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
-template <int P> int bulk_ctas_for(int n, int theta);
+template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 #define K3_DECL(P)                                                                                              \
     template <>                                                                                                 \
     cudaError_t launch_k3_p<P>(const float*, int, int64_t, int64_t, const gar_selection_t*, int, int, int, int, \
                                float*, int, cudaStream_t);                                                      \
-    template <> int bulk_ctas_for<P>(int, int);
+    template <> int bulk_ctas_for<P>(int, int, int);
 K3_P_LIST(K3_DECL)
 #undef K3_DECL
 
@@ -40,17 +40,18 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
         const int want = std::atoi(env);
         if (want == 1 || want == 2 || want == 4) vec = want < vec_max ? want : vec_max;
     }
-    // Staging through shared memory by bulk copies needs 16-byte aligned row segments.  It pays where
-    // the register kernel has to fall back to narrow loads: from 13 slots on with pre-aggregation,
-    // from 25 on without (below, the register kernel with 2- or 4-wide loads is at least as fast).
+    // Staging through shared memory by bulk copies needs 16-byte aligned row segments.  With
+    // pre-aggregation it is the faster kernel at every slot count; without (Bulyan, median, Krum:
+    // the winners are all that is read) the register kernel with 2- or 4-wide loads keeps up with
+    // memory and wins until it has to fall back to scalar loads, from 25 slots on.
     static const char* env_bulk = std::getenv("GAR_K3_BULK");          // tuning aids: 0 = off, else the slot count it starts at
     static const char* env_ctas = std::getenv("GAR_K3_BULK_CTAS");     // CTAs per SM
-    int bulk_from = preagg ? 13 : 25;
+    int bulk_from = preagg ? 1 : 25;
     if (env_bulk) bulk_from = std::atoi(env_bulk) > 0 ? std::atoi(env_bulk) : 1 << 30;
     const bool bulk = vec_max == 4 && theta >= bulk_from;
 #define K3_TRY(P)                                                                                              \
     if (theta <= P) {                                                                                          \
-        int ctas = bulk ? bulk_ctas_for<P>(n, theta) : 0;                                                      \
+        int ctas = bulk ? bulk_ctas_for<P>(n, theta, preagg) : 0;                                                      \
         if (ctas > 0 && env_ctas && std::atoi(env_ctas) > 0 && std::atoi(env_ctas) < ctas) ctas = std::atoi(env_ctas); \
         return launch_k3_p<P>(grads, n, d, ld, sel, theta, preagg, vec, ctas, out, sm_count, stream);          \
     }

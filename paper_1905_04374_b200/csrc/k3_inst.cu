@@ -21,21 +21,37 @@ static inline void preagg_shape(int loose_cap, int V, int* threads, size_t* smem
     *smem = per_thread * t;
 }
 
+// Coordinates per thread of the staged kernel for this slot count (registers: 2 K3_P V values).
+template <bool PREAGG> struct BulkV { static constexpr int V = K3_P <= 8 ? 4 : (K3_P <= (PREAGG ? 12 : 24) ? 2 : 1); };
+
 // Shared memory the staged kernel needs for one stage in the worst case (every gradient staged,
 // a correction in every slot, theta * n additions in the plan).
-static inline size_t bulk_pool_min(int n, int theta) {
-    return size_t((theta * n + 15) & ~15) + size_t(theta + 1) * KB_ROW_BYTES + size_t(n) * KB_ROW_BYTES;
+static inline size_t bulk_pool_min(int n, int theta, int row_bytes) {
+    return size_t((theta * n + 15) & ~15) + size_t(theta + 1) * row_bytes + size_t(n) * row_bytes;
+}
+constexpr size_t kBulkPerSm = 225 * 1024, kBulkPerCta = 3584;   // usable per SM; static shared memory + the system's share per CTA
+
+template <bool PREAGG>
+static int bulk_ctas(int n, int theta) {
+    using S = KBShape<BulkV<PREAGG>::V>;
+    int ctas = int(kBulkPerSm / (bulk_pool_min(n, theta, S::ROW_BYTES) + kBulkPerCta));
+    const int by_threads = 2048 / S::THREADS;
+    return ctas < by_threads ? ctas : by_threads;
 }
 
-// Full tiles [0, ntiles * KB_TC) through the staged kernel, `ctas` CTAs per SM.
+// Full tiles [0, *covered) through the staged kernel, `ctas` CTAs per SM.
 template <int P, bool PREAGG>
-static cudaError_t run_bulk(const float* g, int n, int64_t ntiles, int64_t ld, const gar_selection_t* sel, int theta,
-                            int ctas, float* out, int sm_count, cudaStream_t stream) {
+static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta,
+                            int ctas, float* out, int sm_count, cudaStream_t stream, int64_t* covered) {
     constexpr bool EXACT = (K3_EXACT != 0);
-    constexpr size_t kPerSm = 225 * 1024, kPerCta = 3584;      // static shared memory + the system's share, rounded up
-    const size_t pool_min = bulk_pool_min(n, theta);
-    size_t pool = (kPerSm / size_t(ctas) - kPerCta) & ~size_t(127);
-    const size_t pool_max = pool_min + size_t(KB_MAX_STAGES - 1) * n * KB_ROW_BYTES;
+    constexpr int V = BulkV<PREAGG>::V;
+    using S = KBShape<V>;
+    *covered = 0;
+    const int64_t ntiles = d / S::TC;
+    if (ntiles == 0) return cudaSuccess;
+    const size_t pool_min = bulk_pool_min(n, theta, S::ROW_BYTES);
+    size_t pool = (kBulkPerSm / size_t(ctas) - kBulkPerCta) & ~size_t(127);
+    const size_t pool_max = pool_min + size_t(KB_MAX_STAGES - 1) * n * S::ROW_BYTES;
     if (pool > pool_max) pool = pool_max;
     if (pool < pool_min) return cudaErrorInvalidValue;
     static size_t configured[64] = {0};
@@ -43,17 +59,18 @@ static cudaError_t run_bulk(const float* g, int n, int64_t ntiles, int64_t ld, c
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64 || configured[dev] < pool) {
-        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(pool));
+        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(pool));
         if (err != cudaSuccess) return err;
-        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG, V>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                    cudaSharedmemCarveoutMaxShared);
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = pool;
     }
     int64_t grid = int64_t(sm_count) * ctas;
     if (grid > ntiles) grid = ntiles;
-    k3_bulk<P, EXACT, PREAGG><<<unsigned(grid), KB_THREADS, pool, stream>>>(g, ntiles, ld, const_cast<gar_selection_t*>(sel),
-                                                                             out, int(pool));
+    k3_bulk<P, EXACT, PREAGG, V><<<unsigned(grid), S::THREADS, pool, stream>>>(g, ntiles, ld, const_cast<gar_selection_t*>(sel),
+                                                                                out, int(pool));
+    *covered = ntiles * S::TC;
     return cudaGetLastError();
 }
 
@@ -104,12 +121,10 @@ template <>
 cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
                               int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream) {
     int64_t t0 = 0;
-    if (bulk_ctas > 0 && d >= KB_TC) {           // whole tiles staged through shared memory, the rest below
-        const int64_t ntiles = d / KB_TC;
-        const cudaError_t err = preagg ? run_bulk<K3_P, true>(g, n, ntiles, ld, sel, theta, bulk_ctas, out, sm_count, stream)
-                                       : run_bulk<K3_P, false>(g, n, ntiles, ld, sel, theta, bulk_ctas, out, sm_count, stream);
+    if (bulk_ctas > 0) {                         // whole tiles staged through shared memory, the rest below
+        const cudaError_t err = preagg ? run_bulk<K3_P, true>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0)
+                                       : run_bulk<K3_P, false>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0);
         if (err != cudaSuccess) return err;
-        t0 = ntiles * KB_TC;
         if (t0 == d) return cudaSuccess;
     }
     // 4-wide vectors are only compiled for small slot counts (register budget)
@@ -127,11 +142,8 @@ cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, cons
 
 // CTAs per SM the staged kernel would get for n gradients and theta slots (0: it cannot run).
 template <>
-int bulk_ctas_for<K3_P>(int n, int theta) {
-    const size_t per_cta = bulk_pool_min(n, theta) + 3584;
-    int ctas = int((225 * 1024) / per_cta);
-    const int by_threads = 2048 / KB_THREADS;
-    return ctas < by_threads ? ctas : by_threads;
+int bulk_ctas_for<K3_P>(int n, int theta, int preagg) {
+    return preagg ? bulk_ctas<true>(n, theta) : bulk_ctas<false>(n, theta);
 }
 
 }  // namespace gar
