@@ -43,10 +43,10 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
     // Staging through shared memory by bulk copies needs 16-byte aligned row segments.  With
     // pre-aggregation it is the faster kernel at every slot count; without (Bulyan, median, Krum:
     // the winners are all that is read) the register kernel with 2- or 4-wide loads keeps up with
-    // memory and wins until it has to fall back to scalar loads, from 25 slots on.
+    // memory and wins while the slot count is a compile-time constant, up to 32 slots.
     static const char* env_bulk = std::getenv("GAR_K3_BULK");          // tuning aids: 0 = off, else the slot count it starts at
     static const char* env_ctas = std::getenv("GAR_K3_BULK_CTAS");     // CTAs per SM
-    int bulk_from = preagg ? 1 : 25;
+    int bulk_from = preagg ? 1 : 33;
     if (env_bulk) bulk_from = std::atoi(env_bulk) > 0 ? std::atoi(env_bulk) : 1 << 30;
     const bool bulk = vec_max == 4 && theta >= bulk_from;
 #define K3_TRY(P)                                                                                              \

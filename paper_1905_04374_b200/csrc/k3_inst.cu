@@ -21,8 +21,9 @@ static inline void preagg_shape(int loose_cap, int V, int* threads, size_t* smem
     *smem = per_thread * t;
 }
 
-// Coordinates per thread of the staged kernel for this slot count (registers: 2 K3_P V values).
-template <bool PREAGG> struct BulkV { static constexpr int V = K3_P <= 8 ? 4 : (K3_P <= (PREAGG ? 12 : 24) ? 2 : 1); };
+// Coordinates per thread of the staged kernel for this slot count (registers: 2 K3_P V values);
+// measured on B200: 4 up to 12 slots with pre-aggregation (8 without), 2 up to 32, else 1.
+template <bool PREAGG> struct BulkV { static constexpr int V = K3_P <= (PREAGG ? 12 : 8) ? 4 : (K3_P <= 32 ? 2 : 1); };
 
 // Shared memory the staged kernel needs for one stage in the worst case (every gradient staged,
 // a correction in every slot, theta * n additions in the plan).
