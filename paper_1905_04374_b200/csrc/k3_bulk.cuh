@@ -47,10 +47,13 @@ struct KBPlan {
     int64_t  roff[GAR_MAX_N];                 // staged row -> element offset of its gradient
     int      theta, beta, median_of_agr, lo_pads;
     int      nrows, nbase, ncorr, nstages;
+    int      cols_in_stage;                   // the correction columns reuse dead rows of the stage
+    uint8_t  col_row[GAR_MAX_N + 1];          // correction column -> row that holds it
+    uint8_t  corr_dst[GAR_MAX_N];             // row the j-th correction is written to
     int      error;
     int      loose_row[GAR_MAX_N];            // loose gradient -> staged row
     int      saved_col[GAR_MAX_SAVED];
-    uint8_t  corr_src[GAR_MAX_N];             // column the correction starts from
+    uint8_t  corr_src[GAR_MAX_N];             // row of the column the correction starts from
     uint8_t  corr_nadd[GAR_MAX_N];
 };
 
@@ -132,6 +135,7 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
         // that adds loose gradients).  A slot that only restarts from zero, continues, or takes up
         // a saved sum just names the column that already holds its value.
         int ncorr = 0, col = 0;
+        int slot_col[GAR_MAX_N], src_col[GAR_MAX_N];
         if (PREAGG) {
             for (int s = 0; s < theta; ++s) {
                 if ((sel->corr_mask >> s) & 1ull) {
@@ -141,18 +145,41 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
                     if (nadd == 0) {
                         col = from;
                     } else {
-                        plan.corr_src[ncorr] = uint8_t(from);
+                        src_col[ncorr] = from;
                         plan.corr_nadd[ncorr] = uint8_t(nadd);
                         col = ++ncorr;
                     }
                     const int sv = sel->slot_save[s];
                     if (sv != GAR_SAVE_NONE) plan.saved_col[sv] = col;
                 }
-                plan.slot[s].coff = col * KB_ROW_BYTES;
+                slot_col[s] = col;
             }
         }
         plan.ncorr = ncorr;
-        const int fixed = ((nadds + 15) & ~15) + (ncorr + 1) * KB_ROW_BYTES;
+        // Where the columns live.  Rows of a stage that are dead by the time the corrections are
+        // formed can hold them: the base rows (already summed) and the winners' rows (already in
+        // registers) that no loose gradient shares.  If there are enough of them the columns cost
+        // no shared memory and the ring gets it; else they get an area of their own.
+        int nfree = 0;
+        if (PREAGG) {
+            for (int k = 0; k < nbase && nfree <= ncorr; ++k) plan.col_row[nfree++] = uint8_t(theta + k);
+            for (int s = 0; s < theta && nfree <= ncorr; ++s) {
+                bool shared_row = false;
+                for (int u = 0; u < nloose; ++u) shared_row |= plan.loose_row[u] == s;
+                if (!shared_row) plan.col_row[nfree++] = uint8_t(s);
+            }
+        }
+        const bool in_stage = PREAGG && nfree >= ncorr + 1;
+        plan.cols_in_stage = in_stage ? 1 : 0;
+        if (!in_stage)
+            for (int c = 0; c <= ncorr; ++c) plan.col_row[c] = uint8_t(c);
+        for (int j = 0; j < ncorr; ++j) {
+            plan.corr_src[j] = plan.col_row[src_col[j]];
+            plan.corr_dst[j] = plan.col_row[j + 1];
+        }
+        if (PREAGG)
+            for (int s = 0; s < theta; ++s) plan.slot[s].coff = int(plan.col_row[slot_col[s]]) * KB_ROW_BYTES;
+        const int fixed = ((nadds + 15) & ~15) + (in_stage ? 0 : (ncorr + 1) * KB_ROW_BYTES);
         int nst = (pool_bytes - fixed) / (nrows * KB_ROW_BYTES);
         if (nst > KB_MAX_STAGES) nst = KB_MAX_STAGES;
         plan.nstages = nst;
@@ -168,9 +195,11 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
     for (int k = tid; k < nadds; k += KB_THREADS) add_row[k] = uint8_t(plan.loose_row[sel->add_pos[k]]);
     const int ncorr = plan.ncorr, nrows = plan.nrows, nstages = plan.nstages;
     float* const ccol = reinterpret_cast<float*>(kb_dyn + ((nadds + 15) & ~15));
-    unsigned char* const stages = reinterpret_cast<unsigned char*>(ccol) + (ncorr + 1) * KB_ROW_BYTES;
+    const bool cols_in_stage = plan.cols_in_stage != 0;
+    unsigned char* const stages = reinterpret_cast<unsigned char*>(ccol) + (cols_in_stage ? 0 : (ncorr + 1) * KB_ROW_BYTES);
     const unsigned stage_bytes = unsigned(nrows) * KB_ROW_BYTES;
-    for (int c = tid; c < KB_TC; c += KB_THREADS) ccol[c] = 0.0f;
+    if (!cols_in_stage)
+        for (int c = tid; c < KB_TC; c += KB_THREADS) ccol[c] = 0.0f;
     __syncthreads();
     volatile int* error = &plan.error;
 
@@ -208,7 +237,6 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
         const float inv_beta = 1.0f / float(beta);
         const int lo_pads = EXACT ? 0 : plan.lo_pads;
         const bool med_agr = PREAGG && plan.median_of_agr != 0;
-        float* const mycol = ccol + tid * V;
         int st = 0;
         unsigned parity = 0;
         bool ok = !*error;
@@ -219,7 +247,9 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(failed) : "r"(*error), "r"(KB_BAR_COMPUTE), "r"(KB_CT) : "memory");
             if (failed) break;
-            const float* sv = reinterpret_cast<const float*>(stages + size_t(st) * stage_bytes) + tid * V;
+            float* const svw = reinterpret_cast<float*>(stages + size_t(st) * stage_bytes) + tid * V;
+            const float* sv = svw;
+            float* const mycol = cols_in_stage ? svw : ccol + tid * V;   // this thread's entries of the correction columns' rows
             float e[P][V], a[P][V];
 #pragma unroll
             for (int s = 0; s < P; ++s) {
@@ -250,6 +280,12 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
                     for (int v = 0; v < V; ++v) T[v] += x0[v];
                     bp += KB_TC;
                 }
+                {                                        // column 0: zero (its row's value has been used)
+                    float z[V];
+#pragma unroll
+                    for (int v = 0; v < V; ++v) z[v] = 0.0f;
+                    store_vec<V>(mycol + int(plan.col_row[0]) * KB_TC, z);
+                }
                 int kadd = 0;
                 for (int j = 0; j < ncorr; ++j) {
                     float C[V];
@@ -261,7 +297,7 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
 #pragma unroll
                         for (int v = 0; v < V; ++v) C[v] += x[v];
                     }
-                    store_vec<V>(mycol + (j + 1) * KB_TC, C);
+                    store_vec<V>(mycol + int(plan.corr_dst[j]) * KB_TC, C);
                 }
 #pragma unroll
                 for (int s = 0; s < P; ++s) {
@@ -281,7 +317,9 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
                     for (int v = 0; v < V; ++v) a[s][v] = e[s][v];
                 }
             }
-            // the stage's values are in registers (or folded into T and C): hand it back
+            // the stage's values are in registers (or folded into T and C): hand it back; what this
+            // thread wrote there must be ordered before the bulk copies that will overwrite it
+            if (cols_in_stage) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0)
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(kb_smem_u32(&plan.empty[st])) : "memory");
