@@ -25,6 +25,7 @@
 #include <cstdlib>
 
 #include "gar_internal.cuh"
+#include "mbar.cuh"
 
 namespace gar {
 namespace {
@@ -241,6 +242,163 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
         dist[j * N + i] = s;
     });
     for (int i = tid; i < N; i += K1R_THREADS) dist[i * N + i] = 0.0;
+    if (tid == 0) *ticket = 0u;               // ready for the next call
+}
+
+// ================================================ direct kernel, n <= 16, rows staged by bulk copies
+// Same arithmetic as k1_direct with V = 4; the rows travel differently.  A tile is K1B_TC
+// consecutive coordinates of all N rows; a producer warp fetches it with one bulk copy per row
+// (4 KB, contiguous) into a ring of shared-memory stages whose mbarriers count the bytes in, and
+// the compute threads read their four coordinates of every row at fixed offsets.  Copies of that
+// size keep HBM busier than 16-byte requests per thread do.  Needs 16-byte aligned rows
+// (base address and row stride); coordinates after the last whole tile are added by CTA 0 with
+// plain loads.  A wait that gives up (bounded) raises the CTA's error slot: the last CTA then
+// fills the matrix with NaN and sets the workspace's error word.
+constexpr int K1B_CT = 256;                    // compute threads
+constexpr int K1B_THREADS = K1B_CT + 32;       // + the producer warp
+constexpr int K1B_TC = K1B_CT * 4;             // coordinates per tile
+constexpr int K1B_ROW_BYTES = K1B_TC * 4;
+constexpr int K1B_STAGES = 3;
+constexpr int K1B_BAR_COMPUTE = 1;
+
+template <int N>
+__global__ void __launch_bounds__(K1B_THREADS)
+k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
+               double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word) {
+    constexpr int NP = N * (N - 1) / 2;
+    constexpr int NPAD = (NP + 31) / 32 * 32;
+    constexpr int PER_LANE = NPAD / 32;
+    constexpr int WARPS = K1B_CT / 32;
+    constexpr unsigned STAGE_BYTES = unsigned(N) * K1B_ROW_BYTES;
+    extern __shared__ __align__(128) unsigned char stages[];          // [stage][row][K1B_TC floats]
+    __shared__ double sums[WARPS][NPAD];
+    __shared__ unsigned long long full[K1B_STAGES], empty[K1B_STAGES];
+    __shared__ int error_flag;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < WARPS * NPAD; i += K1B_THREADS) (&sums[0][0])[i] = 0.0;
+    if (tid == 0) {
+        for (int st = 0; st < K1B_STAGES; ++st) { kb_init(&full[st], 1u); kb_init(&empty[st], unsigned(WARPS)); }
+        error_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    volatile int* error = &error_flag;
+
+    const int64_t ntiles = d / K1B_TC;
+    const int64_t first = blockIdx.x, step = gridDim.x;
+    const int64_t mine = first < ntiles ? (ntiles - first + step - 1) / step : 0;
+
+    if (warp == WARPS) {
+        // ================================================================ producer: lane r fetches row r
+        int st = 0;
+        unsigned parity = 1;                         // the phase before the first one: the first waits pass
+        int64_t i = 0;
+        for (; i < mine; ++i) {
+            if (!__all_sync(0xffffffffu, kb_wait(kb_smem_u32(&empty[st]), parity, error))) break;
+            const unsigned bar = kb_smem_u32(&full[st]);
+            if (lane == 0) kb_expect_tx(bar, STAGE_BYTES);
+            __syncwarp();
+            if (lane < N)
+                kb_bulk_load(kb_smem_u32(stages) + unsigned(st) * STAGE_BYTES + unsigned(lane) * K1B_ROW_BYTES,
+                             g + int64_t(lane) * ld + (first + i * step) * K1B_TC, unsigned(K1B_ROW_BYTES), bar);
+            if (++st == K1B_STAGES) { st = 0; parity ^= 1u; }
+        }
+        // no copy may be in flight when the CTA leaves: wait (bounded) for the last tiles issued
+        for (int64_t j = i > K1B_STAGES ? i - K1B_STAGES : 0; j < i; ++j)
+            kb_wait(kb_smem_u32(&full[j % K1B_STAGES]), unsigned(j / K1B_STAGES) & 1u, error, true);
+    } else {
+        // ================================================================ compute: four coordinates per thread
+        float acc[NPAD];
+#pragma unroll
+        for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
+        const int sbase = scatter_base<NPAD, 32>(lane);
+        auto flush = [&]() {
+            reduce_scatter<NPAD, 32>(acc, lane);
+#pragma unroll
+            for (int i = 0; i < PER_LANE; ++i) sums[warp][sbase + i] += double(acc[i]);
+#pragma unroll
+            for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
+        };
+        int st = 0, since = 0;
+        unsigned parity = 0;
+        for (int64_t it = 0; it < mine; ++it) {
+            // one warp waits on the stage's barrier, the others sleep in a hardware barrier meanwhile
+            if (warp == 0) kb_wait(kb_smem_u32(&full[st]), parity, error);
+            unsigned failed;                      // the same answer in every compute thread
+            asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                         : "=r"(failed) : "r"(*error), "r"(K1B_BAR_COMPUTE), "r"(K1B_CT) : "memory");
+            if (failed) break;
+            const float4* src = reinterpret_cast<const float4*>(stages + size_t(st) * STAGE_BYTES) + tid;
+            float x[N][4];
+#pragma unroll
+            for (int r = 0; r < N; ++r) {
+                const float4 q = src[r * (K1B_TC / 4)];
+                x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w;
+            }
+            __syncwarp();                         // the rows are in registers: hand the stage back
+            if (lane == 0) kb_arrive(&empty[st]);
+            int p = 0;
+#pragma unroll
+            for (int i = 0; i < N; ++i) {
+#pragma unroll
+                for (int j = i + 1; j < N; ++j) {
+                    float t = acc[p];
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) { const float df = x[i][v] - x[j][v]; t = fmaf(df, df, t); }
+                    acc[p] = t;
+                    ++p;
+                }
+            }
+            if (++since == K1R_FLUSH) { flush(); since = 0; }
+            if (++st == K1B_STAGES) { st = 0; parity ^= 1u; }
+        }
+        // coordinates after the last whole tile: CTA 0, plain loads
+        if (blockIdx.x == 0) {
+            for (int64_t t = ntiles * K1B_TC + tid; t < d; t += K1B_CT) {
+                float x[N];
+#pragma unroll
+                for (int r = 0; r < N; ++r) x[r] = __ldg(g + int64_t(r) * ld + t);
+                int p = 0;
+#pragma unroll
+                for (int i = 0; i < N; ++i) {
+#pragma unroll
+                    for (int j = i + 1; j < N; ++j) { const float df = x[i] - x[j]; acc[p] = fmaf(df, df, acc[p]); ++p; }
+                }
+            }
+        }
+        __syncwarp();
+        flush();
+    }
+    __syncthreads();
+
+    double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
+    for (int i = tid; i < NP; i += K1B_THREADS) {
+        double s = 0.0;
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) s += sums[w][i];
+        my_partial[i] = s;
+    }
+    if (tid == 0) my_partial[2302] = double(error_flag);
+    if (!last_cta_ticket(ticket)) return;
+    __shared__ int any_error;
+    if (tid == 0) {
+        unsigned err = 0u;
+        for (unsigned b = 0; b < gridDim.x; ++b) err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2302));
+        any_error = int(err);
+        if (err) *error_word = 1u;
+    }
+    __syncthreads();
+    const bool failed = any_error != 0;
+    reduce_partials(partials, NP, K1B_THREADS, [&](int p, double s) {
+        // pair index -> (i, j), pairs enumerated (0,1),(0,2),..,(0,N-1),(1,2),..
+        int i = 0, rem = p;
+        while (rem >= N - 1 - i) { rem -= N - 1 - i; ++i; }
+        const int j = i + 1 + rem;
+        if (failed) s = __longlong_as_double(0x7ff8000000000000ll);
+        dist[i * N + j] = s;
+        dist[j * N + i] = s;
+    });
+    for (int i = tid; i < N; i += K1B_THREADS) dist[i * N + i] = 0.0;
     if (tid == 0) *ticket = 0u;               // ready for the next call
 }
 
@@ -541,8 +699,24 @@ cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, c
 }
 
 template <int N>
+cudaError_t launch_direct_bulk(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
+                               cudaStream_t stream) {
+    static int per_sm_cache[64] = {0};
+    const size_t smem = size_t(K1B_STAGES) * N * K1B_ROW_BYTES;
+    int64_t grid = 0;
+    cudaError_t err = persistent_grid(k1_direct_bulk<N>, K1B_THREADS, smem, sm_count, per_sm_cache, d / K1B_TC, &grid);
+    if (err != cudaSuccess) return err;
+    k1_direct_bulk<N><<<unsigned(grid), K1B_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error());
+    return cudaGetLastError();
+}
+
+template <int N>
 cudaError_t launch_direct_n(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                             cudaStream_t stream, int vec) {
+    // 16-byte aligned rows and enough whole tiles for every SM: rows staged by bulk copies
+    static const char* env = std::getenv("GAR_K1_BULK");            // tuning aid: 0 = off
+    if (vec >= 4 && d >= int64_t(sm_count) * K1B_TC && !(env && std::atoi(env) == 0))
+        return launch_direct_bulk<N>(g, d, ld, dist, ws, sm_count, stream);
     // few rows: wide vectors keep enough bytes in flight; many rows: narrow ones keep the registers in check
     if constexpr (N <= 8) {
         if (vec >= 4) return launch_direct<N, 4>(g, d, ld, dist, ws, sm_count, stream);

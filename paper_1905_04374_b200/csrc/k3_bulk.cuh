@@ -19,6 +19,7 @@
 // before slot s (column 0 holds zero).
 #pragma once
 #include "k3_coordinate.cuh"
+#include "mbar.cuh"
 
 namespace gar {
 
@@ -30,7 +31,6 @@ template <int V> struct KBShape {
     static constexpr int ROW_BYTES = TC * 4;            // one staged row of a tile (one bulk copy)
 };
 constexpr int KB_MAX_STAGES = 4;
-constexpr unsigned KB_SPIN_LIMIT = 1u << 20;  // suspended waits of a barrier before a wait gives up
 constexpr int KB_BAR_COMPUTE = 1;             // named barrier of the compute warps
 
 struct alignas(16) KBSlot {
@@ -56,28 +56,6 @@ struct KBPlan {
     uint8_t  corr_src[GAR_MAX_N];             // row of the column the correction starts from
     uint8_t  corr_nadd[GAR_MAX_N];
 };
-
-__device__ __forceinline__ unsigned kb_smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
-
-// One wait for the phase with the given parity: the thread is suspended in the barrier unit until the
-// phase completes or a hardware time limit passes, whichever comes first; true if it completed.
-__device__ __forceinline__ bool kb_try_wait(unsigned bar, unsigned parity) {
-    unsigned done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    return done != 0;
-}
-// Bounded wait for the phase with the given parity; a waiting warp sleeps in the barrier unit and
-// leaves the issue slots to the computing ones.  False: the wait gave up (error flag raised) or,
-// unless `ignore_flag`, somebody else raised the flag.
-__device__ __forceinline__ bool kb_wait(unsigned bar, unsigned parity, volatile int* error, bool ignore_flag = false) {
-    for (unsigned spin = 0; spin < KB_SPIN_LIMIT; ++spin) {
-        if (kb_try_wait(bar, parity)) return true;
-        if (!ignore_flag && *error) return false;
-    }
-    *error = 1;
-    return false;
-}
 
 // Dynamic shared memory: [staged-row indices of the plan's additions, 16-byte padded]
 // [correction columns (ncorr + 1) x TC floats] [stages: nrows x TC floats each].

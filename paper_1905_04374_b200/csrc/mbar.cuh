@@ -1,0 +1,44 @@
+// mbarrier helpers shared by the kernels that stage tiles through shared memory with bulk copies.
+#pragma once
+
+namespace gar {
+
+constexpr unsigned KB_SPIN_LIMIT = 1u << 20;  // suspended waits of a barrier before a wait gives up
+
+__device__ __forceinline__ unsigned kb_smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
+
+// One wait for the phase with the given parity: the thread is suspended in the barrier unit until the
+// phase completes or a hardware time limit passes, whichever comes first; true if it completed.
+__device__ __forceinline__ bool kb_try_wait(unsigned bar, unsigned parity) {
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait for the phase with the given parity; a waiting warp sleeps in the barrier unit and
+// leaves the issue slots to the computing ones.  False: the wait gave up (error flag raised) or,
+// unless `ignore_flag`, somebody else raised the flag.
+__device__ __forceinline__ bool kb_wait(unsigned bar, unsigned parity, volatile int* error, bool ignore_flag = false) {
+    for (unsigned spin = 0; spin < KB_SPIN_LIMIT; ++spin) {
+        if (kb_try_wait(bar, parity)) return true;
+        if (!ignore_flag && *error) return false;
+    }
+    *error = 1;
+    return false;
+}
+__device__ __forceinline__ void kb_init(unsigned long long* bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(kb_smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void kb_arrive(unsigned long long* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(kb_smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void kb_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// bytes from global memory to this CTA's shared memory (both 16-byte aligned, a multiple of 16), counted in on `bar`
+__device__ __forceinline__ void kb_bulk_load(unsigned dst, const void* src, unsigned bytes, unsigned bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+}  // namespace gar
