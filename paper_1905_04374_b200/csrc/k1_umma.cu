@@ -81,16 +81,29 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
                  : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return done != 0;
 }
-// Bounded wait for the phase with the given parity, the same answer in every lane of the warp.  A
-// waiting warp sleeps in the barrier unit and leaves the issue slots to the working ones.
+__device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
+    unsigned done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Bounded wait for the phase with the given parity, the same answer in every lane of the warp.
+// `polls` quick tests first (a hand-off that is about to happen is seen soonest that way, which
+// matters when the whole kernel is a few dozen slabs), then suspended waits: a warp that waits long
+// sleeps in the barrier unit and leaves the issue slots to the working ones.
 // False: the wait gave up (error flag raised) or another role raised the flag.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* error,
-                                          unsigned limit = KU_SPIN_LIMIT) {
+                                          unsigned polls = 64, unsigned limit = KU_SPIN_LIMIT) {
     bool ok = false;
-    for (unsigned spin = 0; spin < limit; ++spin) {
-        if (mbar_try_wait(bar, parity)) { ok = true; break; }
-        if (*error) break;
-        if (spin + 1 == limit) *error = 1;
+    for (unsigned spin = 0; spin < polls; ++spin) {
+        if (mbar_test(bar, parity)) { ok = true; break; }
+    }
+    if (!ok) {
+        for (unsigned spin = 0; spin < limit; ++spin) {
+            if (mbar_try_wait(bar, parity)) { ok = true; break; }
+            if (*error) break;
+            if (spin + 1 == limit) *error = 1;
+        }
     }
     return __all_sync(0xffffffffu, ok);
 }
@@ -417,7 +430,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         for (int k = 0;; ++k) {
             const int set = k & 1;
             // a set closes rarely: poll slowly; then agree over the four warps (they meet at named barriers below)
-            const bool ok = mbar_wait(&sm.accfull[set], unsigned(k >> 1) & 1u, error);
+            const bool ok = mbar_wait(&sm.accfull[set], unsigned(k >> 1) & 1u, error, 0u);
             unsigned all_ok;
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(all_ok) : "r"(unsigned(ok)), "r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");

@@ -48,7 +48,8 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
     static const char* env_ctas = std::getenv("GAR_K3_BULK_CTAS");     // CTAs per SM
     int bulk_from = preagg ? 1 : 33;
     if (env_bulk) bulk_from = std::atoi(env_bulk) > 0 ? std::atoi(env_bulk) : 1 << 30;
-    const bool bulk = vec_max == 4 && theta >= bulk_from;
+    // (a few hundred thousand coordinates amortise its set-up: the plan, the barriers, the first tiles)
+    const bool bulk = vec_max == 4 && theta >= bulk_from && (d >= 400000 || env_bulk);
 #define K3_TRY(P)                                                                                              \
     if (theta <= P) {                                                                                          \
         int ctas = bulk ? bulk_ctas_for<P>(n, theta, preagg) : 0;                                                      \
