@@ -25,10 +25,9 @@ struct K2Smem {
     double   sv[NMAX][NMAX];      // per row: other rows' distances, ascending
     uint8_t  sj[NMAX][NMAX];      // per row: their indices
     double   score[NMAX];
-    double   pick[4];             // s(1), s(2), s(m), s(m+1)
-    unsigned set_bits[2];
+    double   pick[NMAX][4];       // per round: s(1), s(2), s(m), s(m+1)
+    unsigned long long setmask[NMAX];   // per round: the m best
     unsigned long long alive;
-    int      winner;
 };
 
 __device__ __forceinline__ double rel_gap(double lo, double hi) {
@@ -239,6 +238,7 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         sm.sj[i][rank] = uint8_t(j);
     }
     if (tid == 0) sm.alive = (n == 64) ? ~0ull : ((1ull << n) - 1ull);
+    if (tid < NMAX) sm.setmask[tid] = 0ull;
     __syncthreads();
 
     const bool clamp = (rule == GAR_BULYAN);
@@ -277,37 +277,42 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         }
         __syncthreads();
 
-        // 3b. rank on (score, index); winner, set, gaps
-        if (tid < 64) {
-            bool in_set = false;
-            if (tid < n && ((alive >> tid) & 1ull)) {
-                const double s = sm.score[tid];
-                int rank = 0;
-                for (int j = 0; j < n; ++j) {
-                    if (!((alive >> j) & 1ull)) continue;
-                    const double u = sm.score[j];
-                    rank += (u < s || (u == s && j < tid)) ? 1 : 0;
+        // 3b. rank on (score, index), a warp per row: the rank is the number of remaining rows that
+        // come before it.  The row of rank 0 is the winner and leaves; ranks below m form the set.
+        for (int i = warp; i < n; i += K2_THREADS / 32) {
+            if ((alive >> i) & 1ull) {
+                const double s = sm.score[i];
+                const int j0 = lane, j1 = lane + 32;
+                bool c0 = false, c1 = false;
+                if (j0 < n && ((alive >> j0) & 1ull)) { const double u = sm.score[j0]; c0 = u < s || (u == s && j0 < i); }
+                if (j1 < n && ((alive >> j1) & 1ull)) { const double u = sm.score[j1]; c1 = u < s || (u == s && j1 < i); }
+                const int rank = __popc(__ballot_sync(0xffffffffu, c0)) + __popc(__ballot_sync(0xffffffffu, c1));
+                if (lane == 0) {
+                    if (rank == 0) {
+                        sm.pick[r][0] = s;
+                        sel->winners[r] = i;
+                        sm.alive = alive & ~(1ull << i);        // everybody holds this round's mask in a register
+                    }
+                    if (rank == 1) sm.pick[r][1] = s;
+                    if (rank == m - 1) sm.pick[r][2] = s;
+                    if (rank == m) sm.pick[r][3] = s;
+                    if (rank < m) atomicOr(&sm.setmask[r], 1ull << i);
                 }
-                if (rank == 0) { sm.winner = tid; sm.pick[0] = s; }
-                if (rank == 1) sm.pick[1] = s;
-                if (rank == m - 1) sm.pick[2] = s;
-                if (rank == m) sm.pick[3] = s;
-                in_set = rank < m;
             }
-            const unsigned bits = __ballot_sync(0xffffffffu, in_set);
-            if (lane == 0) sm.set_bits[warp] = bits;
-        }
-        __syncthreads();
-        if (tid == 0) {
-            const int w = sm.winner;
-            sel->winners[r] = w;
-            sel->sets[r] = (uint64_t(sm.set_bits[1]) << 32) | uint64_t(sm.set_bits[0]);
-            sel->gap_winner[r] = (k > 1) ? rel_gap(sm.pick[0], sm.pick[1]) : INFINITY;
-            sel->gap_set[r] = (m < k) ? rel_gap(sm.pick[2], sm.pick[3]) : INFINITY;
-            sm.alive = alive & ~(1ull << w);
         }
         __syncthreads();
     }
+    // sets and gaps of all rounds
+    if (tid < theta) {
+        const int r = tid, k = n - r;
+        int m = 1;
+        if (rule == GAR_MULTI_BULYAN) m = k - f - 2;
+        else if (rule == GAR_MULTI_KRUM) m = m_user > 0 ? m_user : n - f - 2;
+        sel->sets[r] = sm.setmask[r];
+        sel->gap_winner[r] = (k > 1) ? rel_gap(sm.pick[r][0], sm.pick[r][1]) : INFINITY;
+        sel->gap_set[r] = (m < k) ? rel_gap(sm.pick[r][2], sm.pick[r][3]) : INFINITY;
+    }
+    __syncthreads();
     // 4. schedule
     build_schedule(sel, plan_smem);
 }
