@@ -211,10 +211,11 @@ def test_coordinate_phase_given_oracle_tables(pkg, cfg, n, f, rule, d):
     assert_outputs_match(out, want, G=Gh, tables=tab)
 
 
-def test_coordinate_phase_general_schedule(pkg):
+@pytest.mark.parametrize("d", [30_011, 412_347])        # register kernel; kernel staged by bulk copies (+ tail)
+def test_coordinate_phase_general_schedule(pkg, d):
     # sets that are NOT nested (a later round holds a row the earlier one lacks):
     # the summation plan must restart or reuse a saved sum
-    n, f, d = 15, 3, 30_011
+    n, f = 15, 3
     G, Gh, _ = draw(pkg, 5, d)
     winners = [4, 9, 1, 12, 6, 0, 7]
     sets = [[0, 1, 4, 6, 7, 9, 12, 13], [0, 1, 6, 9, 12, 13, 14], [1, 6, 7, 12, 13, 14],
@@ -306,6 +307,24 @@ def test_strided_rows_and_caller_workspace(pkg):
         vh = view.cpu().numpy()
         want, tab = rule_tables("multi_bulyan", vh, f)
         assert_outputs_match(out, want, G=vh, tables=tab)
+
+
+def test_staged_kernels_strided_rows_and_options(pkg):
+    # sizes at which the kernels that stage tiles through shared memory by bulk copies run
+    # (16-byte aligned rows, several tiles per SM), with a row stride larger than d, a ragged
+    # tail, and the multi-Bulyan options; the unaligned view takes the register kernels
+    n, f, d = 15, 3, 450_003
+    big, _ = pkg.workloads.make_gradients(5, d=d + 9, device=DEV)      # row stride 450,012: a multiple of 4
+    for view in (big[:, :d], big[:, 4:d + 4], big[:, 1:d + 1]):
+        vh = view.cpu().numpy()
+        for kw in (dict(), dict(median_of_agr=1), dict(theta=7)):
+            out = pkg.gar_aggregate_ex("multi_bulyan", view, f, **kw).cpu().numpy()
+            want, tab = rule_tables("multi_bulyan", vh, f, theta=kw.get("theta"), median_of_agr=bool(kw.get("median_of_agr")))
+            assert_outputs_match(out, want, G=vh, tables=tab, median_source="agr" if kw.get("median_of_agr") else "ext")
+        D = pkg.gar_pairwise_distances(view).cpu().numpy()
+        Dh = O.pairwise_sq_distances(vh)
+        assert np.max(np.abs(D - Dh) / np.maximum(Dh, 1e-300)) <= 1e-6
+        assert np.array_equal(D, D.T) and np.all(np.diag(D) == 0.0)
 
 
 def test_equal_honest_rows_give_that_row(pkg):
