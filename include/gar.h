@@ -57,7 +57,9 @@ typedef enum {
     GAR_ERR_UNSUPPORTED  = 3, /* n > GAR_MAX_N                                                       */
     GAR_ERR_WORKSPACE    = 4, /* workspace missing, misaligned (256 B) or too small                  */
     GAR_ERR_CUDA         = 5, /* a CUDA runtime call or a launch failed                              */
-    GAR_ERR_TIMEOUT      = 6  /* reserved: a bounded device-side wait gave up                        */
+    GAR_ERR_TIMEOUT      = 6  /* a bounded device-side wait gave up: never returned by a call (the
+                                 calls are asynchronous); the coordinate kernel stores it in the
+                                 selection's `status`, the distance kernels fill the matrix with NaN */
 } gar_status_t;
 
 /*
@@ -97,7 +99,9 @@ typedef struct {
     int32_t  n, f, rule, theta, beta;
     int32_t  preagg;              /* 1: G^agr[r] = mean over sets[r]; 0: G^agr = G^ext */
     int32_t  median_of_agr;       /* 1: median taken over G^agr instead of G^ext       */
-    int32_t  status;              /* gar_status_t written by the selection kernel      */
+    int32_t  status;              /* gar_status_t written by the selection kernel; the
+                                     coordinate kernel overwrites it with GAR_ERR_TIMEOUT if one
+                                     of its bounded waits gave up (the output is then undefined) */
     int32_t  winners[GAR_MAX_N];
     int32_t  m[GAR_MAX_N];
     uint64_t sets[GAR_MAX_N];
