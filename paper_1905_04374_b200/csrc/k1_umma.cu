@@ -55,6 +55,7 @@ struct KUSmem {
     unsigned long long empty[KU_NBUF];       // tcgen05.commit -> producers: the MMAs that read the buffer are done
     unsigned long long accfull[2];           // tcgen05.commit -> flush warps: the set is closed and complete
     unsigned long long accfree[2];           // flush warps -> MMA warp: the set has been read
+    unsigned long long desc[KU_NBUF][8];     // operand descriptors of a buffer's MMAs: k-step ks at [ks] (rows 0..) and [4 + ks] (rows 128..)
     unsigned tmem_base;
     int      error;
     int      grow[KU_NBUF];                  // some row of the buffer uses a larger exponent than before
@@ -216,6 +217,12 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         }
         sm.error = 0; sm.nonfinite_lo = 0u; sm.nonfinite_hi = 0u; sm.is_last = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // the MMA warp's loop is one dependent instruction stream per slab and sits on the kernel's
+    // critical path: everything it can look up instead of compute is tabulated here
+    if (tid < KU_NBUF * 8) {
+        const int b = tid >> 3, ks = tid & 3, second = (tid >> 2) & 1;
+        sm.desc[b][tid & 7] = umma_desc(smem_u32(limb) + unsigned(b) * KU_BUF_BYTES + unsigned(ks) * 2u * KU_LBO + (second ? 128u * 16u : 0u));
     }
     if (warp == KU_MMA_WARP) tmem_alloc(&sm.tmem_base, 2 * KU_SET_COLS);
     fence_async_smem();                  // the zeroed tiles are read by the tensor core (async proxy)
@@ -395,11 +402,11 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             }
             if (lane == 0) {
                 const unsigned d1 = tmem_base + unsigned(set * KU_SET_COLS), d2 = d1 + 192u;
-                const unsigned base = limb_addr + unsigned(buf) * KU_BUF_BYTES;
+                const unsigned long long* dt = sm.desc[buf];
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
-                    const unsigned long long t1 = umma_desc(base + unsigned(ks) * 2u * KU_LBO);            // rows 0..: L1, L2, L3
-                    const unsigned long long t3 = umma_desc(base + unsigned(ks) * 2u * KU_LBO + 128u * 16u);   // rows 128..: L3, then unread rows
+                    const unsigned long long t1 = dt[ks];         // rows 0..: L1, L2, L3
+                    const unsigned long long t3 = dt[4 + ks];     // rows 128..: L3, then unread rows
                     const unsigned acc = (fresh && ks == 0) ? 0u : 1u;
                     umma_i8(d1, t1, t1, IDESC_A, acc);          // [L1; L2] x [L1; L2; L3]^T
                     umma_i8(d2, t3, t3, IDESC_B, acc);          // [L3; *] x L3^T
