@@ -23,7 +23,7 @@ def score(rows, alive, i, q):
                for sub in combinations(others, q))
 
 
-def multi_krum_round(rows, alive, f, clamp=False):
+def multi_krum_round(rows, alive, f, clamp=False, m=None):
     k = len(alive)
     q = k - f - 2
     if clamp:
@@ -31,7 +31,8 @@ def multi_krum_round(rows, alive, f, clamp=False):
     sc = {i: score(rows, alive, i, q) for i in alive}
     best = min(sc.values())
     winner = min(i for i in alive if sc[i] == best)
-    m = q
+    if m is None:
+        m = q
     # (m)argmin: the m-subset with the smallest total score; among equal
     # totals the lexicographically smallest index tuple (lowest-index ties).
     best_sub = min(combinations(sorted(alive), m),
@@ -47,6 +48,21 @@ def rounds(rows, f, theta, clamp=False):
         out.append((w, S, sc))
         alive.remove(w)
     return out
+
+
+def score_gaps(sc, m):
+    """Exact relative gaps of one round: between the two smallest scores, and
+    between the m-th and the (m+1)-th smallest (None where there is no such pair)."""
+    s = sorted(sc.values())
+    gap_w = (s[1] - s[0]) / s[1] if len(s) > 1 and s[1] > 0 else None
+    gap_s = (s[m] - s[m - 1]) / s[m] if m < len(s) and s[m] > 0 else None
+    return gap_w, gap_s
+
+
+def multi_krum(rows, f, m=None):
+    """Average of the m best-scored gradients (Eq. 4's (m)arg-min), any 1 <= m <= n-f-2."""
+    _, S, _ = multi_krum_round(rows, list(range(len(rows))), f, m=m)
+    return mean_rows(rows, S)
 
 
 def lower_median(vals):

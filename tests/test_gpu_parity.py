@@ -258,6 +258,11 @@ def test_rules_end_to_end(pkg, rule, cfg, n, f, d):
     sel = pkg.read_selection(sel_dev)
     preagg = rule in ("multi_krum", "multi_bulyan")
     compared = assert_selection_match(sel, tab["rounds"], preagg)
+    # how much of the selection was really compared: all rounds at the two small sizes (their
+    # score gaps are far above 1e-6), at least the first one at the large size, where the honest
+    # scores of the later rounds come within 1e-6 of each other
+    print(f"{rule} workload {cfg} d={d}: {compared} of {len(tab['rounds'])} rounds compared exactly")
+    assert compared >= (len(tab["rounds"]) if d <= 65_540 else 1)
     if compared == len(tab["rounds"]):
         assert_outputs_match(out, want, G=Gh, tables=tab)
     else:

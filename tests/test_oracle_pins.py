@@ -33,7 +33,8 @@ def _load_examples():
                     "winner": int(tok[3]),
                     "set": [int(v) for v in tok[5].split(",")],
                     "scores": {int(p.split(":")[0]): int(p.split(":")[1])
-                               for p in tok[7].split(",")}})
+                               for p in tok[7].split(",")},
+                    "gaps": tuple(Fraction(v) for v in tok[9].split(","))})
             elif tok[0] == "expect":
                 cur["expect"][tok[1]] = Fraction(tok[2])
     return examples
@@ -136,6 +137,103 @@ def test_worked_examples_rounds(ex):
         assert {i: Fraction(s) for i, s in rnd.scores.items()} == bsc
         assert rnd.m == len(rnd.alive) - f - 2
     assert len(set(sel.winners)) == len(sel.winners)
+
+
+@pytest.mark.parametrize("ex", EXAMPLES, ids=lambda e: e["name"])
+def test_worked_examples_gaps(ex):
+    """The relative score gaps of every round: hand values of the golden file ==
+    exact fractions recomputed from the enumeration's scores == the oracle's."""
+    n, f = ex["n"], ex["f"]
+    rows = [[v] for v in ex["x"]]
+    D = O.pairwise_sq_distances(np.array(rows, dtype=np.float32))
+    sel = O.select_rounds(D, n, f, n - 2 * f - 2)
+    brute = B.rounds(rows, f, n - 2 * f - 2)
+    for rnd, gold, (_, bS, bsc) in zip(sel.rounds, ex["rounds"], brute):
+        gw, gs = B.score_gaps(bsc, len(bS))
+        assert (gw, gs) == gold["gaps"]
+        assert abs(rnd.gap_winner - float(gw)) <= 1e-15
+        assert abs(rnd.gap_set - float(gs)) <= 1e-15
+    # what a plausible mistake would give on example A, round 0 (scores 30, 31 | 63, 102):
+    # relative to the smaller score, absolute, or zero -- none equals the pinned 1/31 and 13/34
+    if ex["name"] == "A":
+        r0 = sel.rounds[0]
+        for wrong in (1 / 30, 1.0, 0.0):
+            assert abs(r0.gap_winner - wrong) > 1e-3
+        for wrong in (39 / 63, 39.0, 0.0, 21 / 63):
+            assert abs(r0.gap_set - wrong) > 1e-3
+    assert sel.min_gap == min(min(float(a), float(b)) for a, b in (g["gaps"] for g in ex["rounds"]))
+
+
+def test_gap_special_cases():
+    """Exact ties give gap 0 (both sides then break them by index); non-finite scores."""
+    # five identical rows and two far ones, f = 1: q = m = 4, the identical rows all score 0
+    x = np.array([[1.0]] * 5 + [[50.0], [-70.0]], dtype=np.float32)
+    rnd = O.multi_krum_round(O.pairwise_sq_distances(x), range(7), 1)
+    assert [rnd.scores[i] for i in range(5)] == [0.0] * 5 and rnd.scores[5] > 0
+    assert rnd.gap_winner == 0.0 and rnd.winner == 0              # s(1) = s(2) = 0: exact tie, lowest index
+    assert rnd.selected == [0, 1, 2, 3] and rnd.gap_set == 0.0     # s(4) = s(5) = 0: exact tie again
+    # equal positive scores: two mirrored pairs around a centre row
+    y = np.array([[-2.0], [-1.0], [0.0], [1.0], [2.0]], dtype=np.float32)
+    rnd = O.multi_krum_round(O.pairwise_sq_distances(y), range(5), 0)   # q = m = 3
+    assert rnd.scores[1] == rnd.scores[3] == 1 + 1 + 4 and rnd.scores[2] == 1 + 1 + 4
+    assert rnd.scores[0] == rnd.scores[4] == 1 + 4 + 9
+    assert rnd.gap_winner == 0.0 and rnd.winner == 1 and rnd.gap_set == (14.0 - 6.0) / 14.0
+    # rows with NaN / Inf are at infinite distance from everybody.  n = 6, f = 1: q = m = 3 of 5
+    # others, the four finite rows keep finite scores, the two others score +inf and stay out
+    w = np.array([[0.0], [1.0], [3.0], [6.0], [np.nan], [np.inf]], dtype=np.float32)
+    D = O.pairwise_sq_distances(w)
+    rnd = O.multi_krum_round(D, range(6), 1)
+    assert [rnd.scores[i] for i in range(4)] == [46.0, 30.0, 22.0, 70.0]
+    assert np.isinf(rnd.scores[4]) and np.isinf(rnd.scores[5])
+    assert rnd.order[:4] == [2, 1, 0, 3] and rnd.gap_winner == 8.0 / 30.0 and rnd.gap_set == 24.0 / 70.0
+    # too many non-finite rows for anybody to avoid them: every score is +inf, every gap a tie
+    rnd = O.multi_krum_round(D, [0, 1, 4, 5], 0)                   # k = 4, q = 2 of 3 others
+    assert all(np.isinf(v) for v in rnd.scores.values())
+    assert rnd.gap_winner == 0.0 and rnd.gap_set == 0.0 and rnd.winner == 0
+    # a finite score next to an infinite one cannot decide a round (a finite score needs
+    # more finite rows than m); the gap function still orders it as "clear"
+    assert O._rel_gap(3.0, np.inf) == np.inf and O._rel_gap(np.inf, np.inf) == 0.0
+    assert O._rel_gap(0.0, 0.0) == 0.0 and O._rel_gap(0.0, 5.0) == 1.0 and O._rel_gap(2.0, 8.0) == 0.75
+
+
+@pytest.mark.parametrize("n,f,m,seed", [(7, 1, 2, 0), (7, 1, 3, 1), (9, 2, 2, 2), (9, 2, 4, 3), (11, 2, 3, 4),
+                                        (11, 2, 6, 5), (10, 1, 5, 6)])
+def test_multi_krum_intermediate_m_matches_enumeration(n, f, m, seed):
+    """Section 3 allows any m <= n-f-2: the average of the m best-scored gradients."""
+    rng = np.random.default_rng(seed)
+    d = 3
+    rows = rng.integers(-30, 30, size=(n, d))
+    rows[rng.choice(n, f, replace=False)] *= 7
+    _, _, sc = B.multi_krum_round(rows.tolist(), list(range(n)), f)
+    if len(set(sc.values())) != len(sc):
+        pytest.skip("tied scores")
+    assert 1 < m < n - f - 2
+    want = B.multi_krum(rows.tolist(), f, m=m)
+    got, rnd = O.multi_krum(rows.astype(np.float32), f, m=m)
+    assert rnd.m == m and len(rnd.selected) == m
+    for t in range(d):
+        assert abs(got[t] - float(want[t])) <= 1e-12 * (1 + abs(float(want[t])))
+    gw, gs = B.score_gaps(sc, m)
+    assert abs(rnd.gap_set - float(gs)) <= 1e-15 and abs(rnd.gap_winner - float(gw)) <= 1e-15
+
+
+@pytest.mark.parametrize("n,f,theta,seed", [(9, 1, 3, 0), (9, 1, 4, 1), (10, 1, 5, 2), (11, 1, 6, 3), (11, 1, 3, 4),
+                                            (11, 2, 5, 5)])
+def test_multi_bulyan_theta_option_matches_enumeration(n, f, theta, seed):
+    """A shorter extraction loop (2f+1 <= theta <= n-2f-2 rounds): beta = theta-2f follows it."""
+    rng = np.random.default_rng(50 + seed)
+    d = 4
+    rows = rng.integers(-30, 30, size=(n, d))
+    rows[rng.choice(n, f, replace=False)] *= 9
+    for _, _, sc in B.rounds(rows.tolist(), f, theta):
+        if len(set(sc.values())) != len(sc):
+            pytest.skip("tied scores")
+    assert 2 * f + 1 <= theta <= n - 2 * f - 2
+    want = B.multi_bulyan(rows.tolist(), f, theta=theta)
+    got, sel, _ = O.multi_bulyan(rows.astype(np.float32), f, theta=theta)
+    assert sel.theta == theta and sel.beta == theta - 2 * f and len(sel.rounds) == theta
+    for t in range(d):
+        assert abs(got[t] - float(want[t])) <= 1e-12 * (1 + abs(float(want[t])))
 
 
 @pytest.mark.parametrize("ex", EXAMPLES, ids=lambda e: e["name"])
