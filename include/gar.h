@@ -23,8 +23,28 @@
  *  - Results are deterministic: the same input gives bit-identical output.
  *  - Ties (equal scores, equal distances to the median) are broken towards the
  *    lowest worker index, in the coordinate phase towards the earliest round.
- *    The median of an even count is the lower of the two middle values.
- *    A non-finite distance is treated as +infinity.
+ *    The median of an even count is the lower of the two middle values unless
+ *    GAR_EVEN_MEDIAN_MEAN is asked for.  A non-finite distance is treated as
+ *    +infinity.
+ *  - No silent wrong answer: if a kernel gives up on one of its bounded waits, or
+ *    the coordinate phase is handed an inconsistent selection, the selection's
+ *    `status` is set and `out` is filled with NaN (see GAR_ERR_TIMEOUT below).
+ *  - Thread safety: calls on distinct devices, or with distinct caller workspaces
+ *    on distinct streams, may run concurrently.  The cached per-device buffers
+ *    (NULL workspace, gar_aggregate_host, gar_pairwise_distances_static) are
+ *    created under a lock but shared: serialise the calls that use them.
+ *
+ * Distances for 16 < n <= 64 (16-byte aligned rows, d >= 32768) are formed on the
+ * tensor cores from rows rounded to a grid of 2^-21 of the largest binade each row
+ * has shown; the kernel then bounds the effect of that rounding on every D_ij from
+ * the steps it used (rounding errors taken as independent of the differences, six
+ * standard deviations, plus the worst-case bias) and, if some pair's bound exceeds
+ * 1e-6 of its distance, the same call recomputes the matrix with the fp32
+ * difference form on the CUDA cores, on the device and without a host round trip
+ * (about 2.5 times slower).  Inputs that stay on the fast path: rows whose largest
+ * entry R and typical difference to the other rows s satisfy roughly
+ * R / s <= 0.2 sqrt(d) (e.g. 100 at d = 2.6e5, 1000 at d = 2.6e7).  Rows that agree
+ * within the grid everywhere are reported at distance exactly 0.
  */
 #ifndef GAR_H_
 #define GAR_H_
@@ -37,7 +57,7 @@ extern "C" {
 #endif
 
 #define GAR_MAX_N 64
-#define GAR_VERSION 100
+#define GAR_VERSION 101
 
 typedef enum {
     GAR_AVERAGE      = 0, /* (1/n) sum_i G_i                       (Introduction)            */
@@ -57,10 +77,26 @@ typedef enum {
     GAR_ERR_UNSUPPORTED  = 3, /* n > GAR_MAX_N                                                       */
     GAR_ERR_WORKSPACE    = 4, /* workspace missing, misaligned (256 B) or too small                  */
     GAR_ERR_CUDA         = 5, /* a CUDA runtime call or a launch failed                              */
-    GAR_ERR_TIMEOUT      = 6  /* a bounded device-side wait gave up: never returned by a call (the
-                                 calls are asynchronous); the coordinate kernel stores it in the
-                                 selection's `status`, the distance kernels fill the matrix with NaN */
+    GAR_ERR_TIMEOUT      = 6  /* a bounded device-side wait gave up.  The asynchronous calls cannot
+                                 return it; it travels on the device instead: a distance kernel that
+                                 gives up fills the whole matrix, diagonal included, with NaN; the
+                                 selection kernel answers a NaN diagonal with status = GAR_ERR_TIMEOUT
+                                 and selects nothing; the coordinate kernel answers any status other
+                                 than GAR_OK by filling `out` with NaN, and stores GAR_ERR_TIMEOUT
+                                 itself if one of its own waits gives up.  gar_aggregate_host, which
+                                 is synchronous, returns the status. */
 } gar_status_t;
+
+typedef enum {
+    GAR_EVEN_MEDIAN_LOWER = 0, /* median of an even count = the lower middle value (what the Median
+                                  comparator of Section 5, PyTorch's, returns)                      */
+    GAR_EVEN_MEDIAN_MEAN  = 1  /* = the mean of the two middle values                               */
+} gar_even_median_t;
+
+typedef enum {
+    GAR_DISTANCES_AUTO       = 0, /* tensor-core Gram product where it applies, checked as described above */
+    GAR_DISTANCES_DIFFERENCE = 1  /* always the fp32 difference form on the CUDA cores                     */
+} gar_distance_mode_t;
 
 /*
  * Result of the scoring / selection step (Eq. 4; Algorithm 1, multi-Krum and
@@ -99,9 +135,13 @@ typedef struct {
     int32_t  n, f, rule, theta, beta;
     int32_t  preagg;              /* 1: G^agr[r] = mean over sets[r]; 0: G^agr = G^ext */
     int32_t  median_of_agr;       /* 1: median taken over G^agr instead of G^ext       */
-    int32_t  status;              /* gar_status_t written by the selection kernel; the
-                                     coordinate kernel overwrites it with GAR_ERR_TIMEOUT if one
-                                     of its bounded waits gave up (the output is then undefined) */
+    int32_t  status;              /* gar_status_t written by the selection kernel (GAR_ERR_TIMEOUT if
+                                     the distance matrix carries a NaN diagonal); the coordinate
+                                     kernel stores GAR_ERR_TIMEOUT (a wait of its own gave up) or
+                                     GAR_ERR_INVALID_ARG (tables inconsistent with its arguments)
+                                     and fills `out` with NaN whenever this is not GAR_OK */
+    int32_t  even_median;         /* gar_even_median_t */
+    int32_t  reserved;
     int32_t  winners[GAR_MAX_N];
     int32_t  m[GAR_MAX_N];
     uint64_t sets[GAR_MAX_N];
@@ -140,9 +180,12 @@ typedef struct {
     int32_t       theta;          /* multi-Bulyan only: number of rounds, 2f+1..n-2f-2; 0 = n-2f-2 */
     int32_t       median_of_agr;  /* multi-Bulyan only: 1 = median over G^agr (reading of Section 5.2's
                                      "median ... over ... pre-aggregated gradients"); 0 = Algorithm 1 */
-    int32_t       reserved;
+    int32_t       even_median;    /* gar_even_median_t: median of an even count (Median rule of Section 5;
+                                     Median(G^ext) of Algorithm 1 when theta is even) */
     double*       dist_out;       /* optional dev [n*n]: the distance matrix */
     gar_selection_t* selection_out; /* optional dev: the selection result */
+    int32_t       distance_mode;  /* gar_distance_mode_t */
+    int32_t       reserved;
 } gar_params_t;
 
 /* Library version (GAR_VERSION).  The paper has no counterpart. */
@@ -158,7 +201,11 @@ const char* gar_status_string(int status);
 int gar_theta(int rule, int n, int f);
 int gar_beta(int rule, int n, int f);
 
-/* Bytes of device workspace a call needs (host, pure).  0 on invalid arguments. */
+/* Bytes of device workspace a call needs (host, pure).  0 on invalid arguments.
+ * The first 256 bytes are a control block of 32-bit words: [0] ticket counter of the distance
+ * kernels (zero between calls), [2] set to 1 by a distance kernel whose wait gave up, [4] how the
+ * last distance call ran: 0 = fp32 difference form, 1 = tensor-core Gram product kept,
+ * 2 = Gram product rejected by its error bound and recomputed in the difference form. */
 size_t gar_workspace_bytes(int rule, int n, int f, int64_t d);
 
 /*
@@ -191,6 +238,9 @@ int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, fl
  */
 int gar_pairwise_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
                            void* workspace, size_t workspace_bytes, void* stream);
+/* Same with a gar_distance_mode_t. */
+int gar_pairwise_distances_mode(const float* grads, int n, int64_t d, int64_t ld, double* dist,
+                                void* workspace, size_t workspace_bytes, int distance_mode, void* stream);
 
 /*
  * Step 1 alone, for callers that must not allocate: the same distance kernels, but
@@ -216,10 +266,12 @@ int gar_pairwise_distances_static(const float* grads, int n, int64_t d, int64_t 
 /*
  * Step 2 alone: scoring and iterative selection from a distance matrix
  * (Eq. 4; Algorithm 1 multi-Krum and the loop of multi-Bulyan).
- *   dist dev [n*n] fp64; sel dev, written.  m, theta as in gar_params_t (0 = default).
+ *   dist dev [n*n] fp64; sel dev, written.  m, theta, median_of_agr, even_median as in
+ *   gar_params_t (0 = default).  A NaN on the diagonal of dist (left by a distance kernel
+ *   that gave up) gives sel->status = GAR_ERR_TIMEOUT and no selection.
  */
 int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int median_of_agr,
-               gar_selection_t* sel, void* stream);
+               int even_median, gar_selection_t* sel, void* stream);
 
 /*
  * Builds the coordinate kernel's schedule for GIVEN winners and sets (e.g. the
@@ -235,9 +287,23 @@ int gar_schedule_from_tables(gar_selection_t* sel, void* stream);
  * G^ext, the beta entries of G^agr closest to it, their average) for a
  * selection already on the device.  theta and preagg repeat sel->theta and
  * sel->preagg (the host needs them to pick the kernel).  out dev [d].
+ * Before it reads a gradient the kernel checks the selection on the device: a
+ * status other than GAR_OK, a theta or preagg that differs from sel's, or a row
+ * index >= n in the tables gives out = NaN everywhere (and, for the last two,
+ * sel->status = GAR_ERR_INVALID_ARG); sel is therefore not const.
  */
 int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld,
-                         const gar_selection_t* sel, int theta, int preagg, float* out, void* stream);
+                         gar_selection_t* sel, int theta, int preagg, float* out, void* stream);
+
+/*
+ * Self-test of the bounded wait every staged kernel uses (mbarrier.try_wait in a loop with an
+ * iteration limit): one warp waits, with the given limit (1 .. 65536), on a barrier that nothing
+ * ever arrives on -- no copy and no tensor-core operation is in flight -- and reports how it
+ * ended.  result dev [2] int64: [0] = GAR_ERR_TIMEOUT if the wait gave up as it must (GAR_OK
+ * would mean it returned as if the barrier had completed), [1] = nanoseconds the wait took
+ * (%globaltimer).  The paper has no counterpart (diagnostic aid).
+ */
+int gar_selftest_bounded_wait(unsigned int limit, long long* result, void* stream);
 
 /* Frees every cached device buffer of every device.  Synchronises. */
 void gar_shutdown(void);

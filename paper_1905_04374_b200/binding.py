@@ -14,6 +14,10 @@ import torch
 
 GAR_MAX_N = 64
 RULES = {"average": 0, "median": 1, "krum": 2, "multi_krum": 3, "bulyan": 4, "multi_bulyan": 5}
+EVEN_MEDIAN = {"lower": 0, "mean": 1}
+DISTANCE_MODES = {"auto": 0, "difference": 1}
+# gar_workspace control block, word 4: how the last distance call ran
+DISTANCE_PATHS = {0: "difference", 1: "gram", 2: "gram_rejected"}
 GAR_OK = 0
 STATUS_NAMES = {0: "GAR_OK", 1: "GAR_ERR_INVALID_ARG", 2: "GAR_ERR_PRECONDITION", 3: "GAR_ERR_UNSUPPORTED",
                 4: "GAR_ERR_WORKSPACE", 5: "GAR_ERR_CUDA", 6: "GAR_ERR_TIMEOUT"}
@@ -27,6 +31,7 @@ class GarSelection(C.Structure):
     _fields_ = [
         ("n", C.c_int32), ("f", C.c_int32), ("rule", C.c_int32), ("theta", C.c_int32), ("beta", C.c_int32),
         ("preagg", C.c_int32), ("median_of_agr", C.c_int32), ("status", C.c_int32),
+        ("even_median", C.c_int32), ("reserved", C.c_int32),
         ("winners", C.c_int32 * GAR_MAX_N),
         ("m", C.c_int32 * GAR_MAX_N),
         ("sets", C.c_uint64 * GAR_MAX_N),
@@ -51,8 +56,9 @@ class GarParams(C.Structure):
         ("d", C.c_int64), ("ld", C.c_int64),
         ("grads", C.c_void_p), ("out", C.c_void_p), ("stream", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-        ("m", C.c_int32), ("theta", C.c_int32), ("median_of_agr", C.c_int32), ("reserved", C.c_int32),
+        ("m", C.c_int32), ("theta", C.c_int32), ("median_of_agr", C.c_int32), ("even_median", C.c_int32),
         ("dist_out", C.c_void_p), ("selection_out", C.c_void_p),
+        ("distance_mode", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -83,9 +89,12 @@ def lib():
         L.gar_aggregate_host.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_void_p]
         L.gar_pairwise_distances.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                              C.c_size_t, C.c_void_p]
+        L.gar_pairwise_distances_mode.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                                  C.c_size_t, C.c_int, C.c_void_p]
+        L.gar_selftest_bounded_wait.argtypes = [C.c_uint, C.c_void_p, C.c_void_p]
         L.gar_pairwise_distances_static.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
-        L.gar_select.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
-                                 C.c_void_p]
+        L.gar_select.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                 C.c_void_p, C.c_void_p]
         L.gar_schedule_from_tables.argtypes = [C.c_void_p, C.c_void_p]
         L.gar_coordinate_phase.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_int, C.c_int,
                                            C.c_void_p, C.c_void_p]
@@ -96,6 +105,14 @@ def lib():
 
 def _rule(rule) -> int:
     return RULES[rule] if isinstance(rule, str) else int(rule)
+
+
+def _even(even_median) -> int:
+    return EVEN_MEDIAN[even_median] if isinstance(even_median, str) else int(even_median)
+
+
+def _mode(distance_mode) -> int:
+    return DISTANCE_MODES[distance_mode] if isinstance(distance_mode, str) else int(distance_mode)
 
 
 def _stream(stream) -> int:
@@ -161,7 +178,8 @@ def gar_aggregate(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = 
 
 def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = None, stream=None,
                      workspace: torch.Tensor | None = None, m: int = 0, theta: int = 0, median_of_agr: int = 0,
-                     dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None):
+                     dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None,
+                     even_median=0, distance_mode=0):
     """gar_aggregate_ex: row stride taken from the tensor; optional workspace
     (uint8 CUDA tensor), options and outputs (dist_out float64 [n, n];
     selection_out uint8 CUDA tensor of sizeof(gar_selection_t))."""
@@ -175,6 +193,7 @@ def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None
     if workspace is not None:
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     p.m, p.theta, p.median_of_agr = m, theta, median_of_agr
+    p.even_median, p.distance_mode = _even(even_median), _mode(distance_mode)
     if dist_out is not None:
         p.dist_out = dist_out.data_ptr()
     if selection_out is not None:
@@ -198,17 +217,38 @@ def gar_aggregate_host(rule, grads: torch.Tensor, f: int, out: torch.Tensor | No
 
 
 def gar_pairwise_distances(grads: torch.Tensor, dist: torch.Tensor | None = None, workspace=None,
-                           stream=None) -> torch.Tensor:
-    """gar_pairwise_distances: returns dist float64 [n, n] on the device."""
+                           stream=None, distance_mode=0) -> torch.Tensor:
+    """gar_pairwise_distances (gar_pairwise_distances_mode when a mode is given): returns dist
+    float64 [n, n] on the device."""
     _dev_f32(grads, "grads")
     n, d, ld = _rows(grads)
     if dist is None:
         dist = torch.empty(n, n, dtype=torch.float64, device=grads.device)
     wp, wb = (workspace.data_ptr(), workspace.numel() * workspace.element_size()) if workspace is not None else (None, 0)
     with torch.cuda.device(grads.device):
-        st = lib().gar_pairwise_distances(grads.data_ptr(), n, d, ld, dist.data_ptr(), wp, wb, _stream(stream))
+        if _mode(distance_mode) == 0:
+            st = lib().gar_pairwise_distances(grads.data_ptr(), n, d, ld, dist.data_ptr(), wp, wb, _stream(stream))
+        else:
+            st = lib().gar_pairwise_distances_mode(grads.data_ptr(), n, d, ld, dist.data_ptr(), wp, wb,
+                                                   _mode(distance_mode), _stream(stream))
     _check(st, "gar_pairwise_distances")
     return dist
+
+
+def distance_path(workspace: torch.Tensor) -> str:
+    """How the last distance call that used this caller-owned workspace ran (control block, word 4)."""
+    word = workspace[16:20].cpu().numpy().view("uint32")[0]
+    return DISTANCE_PATHS.get(int(word), str(int(word)))
+
+
+def gar_selftest_bounded_wait(limit: int, device="cuda", stream=None):
+    """gar_selftest_bounded_wait: (status, nanoseconds) of a bounded wait on a barrier nobody arrives on."""
+    res = torch.zeros(2, dtype=torch.int64, device=device)
+    with torch.cuda.device(res.device):
+        st = lib().gar_selftest_bounded_wait(limit, res.data_ptr(), _stream(stream))
+    _check(st, "gar_selftest_bounded_wait")
+    host = res.cpu()
+    return int(host[0]), int(host[1])
 
 
 def gar_pairwise_distances_static(grads: torch.Tensor, dist: torch.Tensor, stream=None) -> torch.Tensor:
@@ -243,7 +283,7 @@ def write_selection(host: GarSelection, device) -> torch.Tensor:
 
 
 def gar_select(rule, dist: torch.Tensor | None, n: int, f: int, m: int = 0, theta: int = 0, median_of_agr: int = 0,
-               sel: torch.Tensor | None = None, stream=None, device=None) -> torch.Tensor:
+               sel: torch.Tensor | None = None, stream=None, device=None, even_median=0) -> torch.Tensor:
     """gar_select: dist CUDA float64 [n, n]; returns the device gar_selection_t buffer."""
     device = dist.device if dist is not None else (device or "cuda")
     if sel is None:
@@ -254,7 +294,8 @@ def gar_select(rule, dist: torch.Tensor | None, n: int, f: int, m: int = 0, thet
             raise TypeError("dist must be a contiguous CUDA float64 tensor")
         dp = dist.data_ptr()
     with torch.cuda.device(sel.device):
-        st = lib().gar_select(_rule(rule), dp, n, f, m, theta, median_of_agr, sel.data_ptr(), _stream(stream))
+        st = lib().gar_select(_rule(rule), dp, n, f, m, theta, median_of_agr, _even(even_median), sel.data_ptr(),
+                              _stream(stream))
     _check(st, "gar_select")
     return sel
 

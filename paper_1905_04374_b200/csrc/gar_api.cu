@@ -4,6 +4,7 @@
 #include <mutex>
 
 #include "gar_internal.cuh"
+#include "mbar.cuh"
 
 namespace {
 
@@ -20,9 +21,7 @@ struct DeviceState {
     size_t  stage_grads_elems = 0;
     float*  stage_out = nullptr;
     size_t  stage_out_elems = 0;
-    cudaStream_t copy_stream = nullptr, compute_stream = nullptr;
-    cudaEvent_t  slab_ready[2] = {nullptr, nullptr};
-    cudaEvent_t  computed = nullptr;
+    cudaStream_t host_stream = nullptr;   // gar_aggregate_host: copies and kernels, in order
 };
 
 DeviceState g_dev[kMaxDevices];
@@ -71,7 +70,13 @@ int device_state(DeviceState** out, bool need_workspace) {
     }
     if (need_workspace && !st.workspace) {
         if (cudaMalloc(&st.workspace, gar::kWorkspaceBytes) != cudaSuccess) return GAR_ERR_CUDA;
-        if (cudaMemset(st.workspace, 0, gar::kCtrlBytes) != cudaSuccess) return GAR_ERR_CUDA;
+        // the control block must read zero before the first kernel of ANY stream touches it (a
+        // memset on the legacy stream is not ordered before work on a non-blocking stream)
+        if (cudaMemset(st.workspace, 0, gar::kCtrlBytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+            cudaFree(st.workspace);
+            st.workspace = nullptr;
+            return GAR_ERR_CUDA;
+        }
     }
     *out = &st;
     return GAR_OK;
@@ -97,18 +102,18 @@ bool overlaps(const void* a, size_t abytes, const void* b, size_t bbytes) {
 
 // Enqueue the whole rule for device buffers.
 int enqueue(int rule, const float* grads, int n, int f, int64_t d, int64_t ld, float* out, int m, int theta,
-            int median_of_agr, const Workspace& ws, double* dist_out, gar_selection_t* sel_out,
-            int sm_count, cudaStream_t stream) {
+            int median_of_agr, int even_median, int distance_mode, const Workspace& ws, double* dist_out,
+            gar_selection_t* sel_out, int sm_count, cudaStream_t stream) {
     const int beta = beta_for(rule, theta, f);
     double* dist = dist_out ? dist_out : ws.dist();
     gar_selection_t* sel = sel_out ? sel_out : ws.selection();
     cudaError_t err;
     const bool needs_dist = !(rule == GAR_AVERAGE || rule == GAR_MEDIAN);
     if (needs_dist) {
-        err = gar::launch_distances(grads, n, d, ld, dist, ws, sm_count, stream);
+        err = gar::launch_distances(grads, n, d, ld, dist, ws, sm_count, distance_mode, stream);
         if (err != cudaSuccess) return GAR_ERR_CUDA;
     }
-    err = gar::launch_select(rule, dist, n, f, m, theta, beta, median_of_agr, sel, stream);
+    err = gar::launch_select(rule, dist, n, f, m, theta, beta, median_of_agr, even_median, sel, stream);
     if (err != cudaSuccess) return GAR_ERR_CUDA;
     const int preagg = (rule == GAR_MULTI_BULYAN || rule == GAR_MULTI_KRUM || rule == GAR_AVERAGE) ? 1 : 0;
     err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg, out, sm_count, stream);
@@ -116,7 +121,37 @@ int enqueue(int rule, const float* grads, int n, int f, int64_t d, int64_t ld, f
     return GAR_OK;
 }
 
+bool even_median_ok(int v) { return v == GAR_EVEN_MEDIAN_LOWER || v == GAR_EVEN_MEDIAN_MEAN; }
+bool distance_mode_ok(int v) { return v == GAR_DISTANCES_AUTO || v == GAR_DISTANCES_DIFFERENCE; }
+
+// One warp, a barrier that nothing arrives on, a bounded wait: it must give up.
+__global__ void selftest_wait_kernel(unsigned limit, long long* result) {
+    __shared__ unsigned long long bar;
+    __shared__ int error_flag;
+    if (threadIdx.x == 0) {
+        gar::kb_init(&bar, 1u);
+        error_flag = 0;
+        gar::kb_fence_init();
+    }
+    __syncwarp();
+    unsigned long long t0, t1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    const bool ok = gar::kb_wait_warp(gar::kb_smem_u32(&bar), 0u, &error_flag, 4u, limit);
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t1));
+    if (threadIdx.x == 0) {
+        result[0] = (!ok && error_flag) ? GAR_ERR_TIMEOUT : GAR_OK;
+        result[1] = static_cast<long long>(t1 - t0);
+    }
+}
+
 }  // namespace
+
+namespace gar {
+cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t stream) {
+    selftest_wait_kernel<<<1, 32, 0, stream>>>(limit, result);
+    return cudaGetLastError();
+}
+}  // namespace gar
 
 extern "C" {
 
@@ -171,12 +206,14 @@ int gar_aggregate_ex(const gar_params_t* p) {
         theta = p->theta;
     }
     if (p->median_of_agr != 0 && (p->rule != GAR_MULTI_BULYAN || p->median_of_agr != 1)) return GAR_ERR_INVALID_ARG;
+    if (!even_median_ok(p->even_median) || !distance_mode_ok(p->distance_mode)) return GAR_ERR_INVALID_ARG;
     DeviceState* st = nullptr;
     Workspace ws{};
     rc = resolve_workspace(p->workspace, p->workspace_bytes, &st, &ws);
     if (rc != GAR_OK) return rc;
-    return enqueue(p->rule, p->grads, p->n, p->f, p->d, ld, p->out, m, theta, p->median_of_agr, ws, p->dist_out,
-                   p->selection_out, st->sm_count, static_cast<cudaStream_t>(p->stream));
+    return enqueue(p->rule, p->grads, p->n, p->f, p->d, ld, p->out, m, theta, p->median_of_agr, p->even_median,
+                   p->distance_mode, ws, p->dist_out, p->selection_out, st->sm_count,
+                   static_cast<cudaStream_t>(p->stream));
 }
 
 int gar_aggregate(int rule, const float* grads, int n, int f, int64_t d, float* out, void* stream) {
@@ -188,7 +225,12 @@ int gar_aggregate(int rule, const float* grads, int n, int f, int64_t d, float* 
 
 int gar_pairwise_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist, void* workspace,
                            size_t workspace_bytes, void* stream) {
-    if (!grads || !dist || n < 1 || d < 1) return GAR_ERR_INVALID_ARG;
+    return gar_pairwise_distances_mode(grads, n, d, ld, dist, workspace, workspace_bytes, GAR_DISTANCES_AUTO, stream);
+}
+
+int gar_pairwise_distances_mode(const float* grads, int n, int64_t d, int64_t ld, double* dist, void* workspace,
+                                size_t workspace_bytes, int distance_mode, void* stream) {
+    if (!grads || !dist || n < 1 || d < 1 || !distance_mode_ok(distance_mode)) return GAR_ERR_INVALID_ARG;
     if (n > GAR_MAX_N) return GAR_ERR_UNSUPPORTED;
     if (ld == 0) ld = d;
     if (ld < d) return GAR_ERR_INVALID_ARG;
@@ -196,11 +238,12 @@ int gar_pairwise_distances(const float* grads, int n, int64_t d, int64_t ld, dou
     Workspace ws{};
     int rc = resolve_workspace(workspace, workspace_bytes, &st, &ws);
     if (rc != GAR_OK) return rc;
-    cudaError_t err = gar::launch_distances(grads, n, d, ld, dist, ws, st->sm_count, static_cast<cudaStream_t>(stream));
+    cudaError_t err = gar::launch_distances(grads, n, d, ld, dist, ws, st->sm_count, distance_mode,
+                                            static_cast<cudaStream_t>(stream));
     return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }
 
-int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int median_of_agr,
+int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int median_of_agr, int even_median,
                gar_selection_t* sel, void* stream) {
     int rc = basic_checks(rule, n, f, 1);
     if (rc != GAR_OK) return rc;
@@ -214,7 +257,8 @@ int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int
         th = theta;
     }
     if (median_of_agr != 0 && (rule != GAR_MULTI_BULYAN || median_of_agr != 1)) return GAR_ERR_INVALID_ARG;
-    cudaError_t err = gar::launch_select(rule, dist, n, f, m, th, beta_for(rule, th, f), median_of_agr, sel,
+    if (!even_median_ok(even_median)) return GAR_ERR_INVALID_ARG;
+    cudaError_t err = gar::launch_select(rule, dist, n, f, m, th, beta_for(rule, th, f), median_of_agr, even_median, sel,
                                          static_cast<cudaStream_t>(stream));
     return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }
@@ -225,7 +269,7 @@ int gar_schedule_from_tables(gar_selection_t* sel, void* stream) {
     return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }
 
-int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta,
+int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta,
                          int preagg, float* out, void* stream) {
     if (!grads || !sel || !out || n < 1 || d < 1 || theta < 1 || theta > GAR_MAX_N) return GAR_ERR_INVALID_ARG;
     if (n > GAR_MAX_N) return GAR_ERR_UNSUPPORTED;
@@ -239,6 +283,11 @@ int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, const
     return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }
 
+int gar_selftest_bounded_wait(unsigned int limit, long long* result, void* stream) {
+    if (!result || limit < 1u || limit > 65536u) return GAR_ERR_INVALID_ARG;
+    return gar::launch_selftest_wait(limit, result, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+}
+
 int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, float* out) {
     int rc = basic_checks(rule, n, f, d);
     if (rc != GAR_OK) return rc;
@@ -246,38 +295,42 @@ int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, fl
     DeviceState* st = nullptr;
     rc = device_state(&st, true);
     if (rc != GAR_OK) return rc;
-    // staging buffers and streams (cached, grown on demand)
+    // staging buffers and the stream (cached, grown on demand, under the lock; the call itself
+    // uses them outside it: concurrent host calls on one device must be serialised by the caller)
     const size_t need = size_t(n) * size_t(d);
-    if (st->stage_grads_elems < need) {
-        if (st->stage_grads) cudaFree(st->stage_grads);
-        st->stage_grads = nullptr; st->stage_grads_elems = 0;
-        if (cudaMalloc(&st->stage_grads, need * sizeof(float)) != cudaSuccess) return GAR_ERR_CUDA;
-        st->stage_grads_elems = need;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (st->stage_grads_elems < need) {
+            if (st->stage_grads) cudaFree(st->stage_grads);
+            st->stage_grads = nullptr; st->stage_grads_elems = 0;
+            if (cudaMalloc(&st->stage_grads, need * sizeof(float)) != cudaSuccess) return GAR_ERR_CUDA;
+            st->stage_grads_elems = need;
+        }
+        if (st->stage_out_elems < size_t(d)) {
+            if (st->stage_out) cudaFree(st->stage_out);
+            st->stage_out = nullptr; st->stage_out_elems = 0;
+            if (cudaMalloc(&st->stage_out, size_t(d) * sizeof(float)) != cudaSuccess) return GAR_ERR_CUDA;
+            st->stage_out_elems = size_t(d);
+        }
+        if (!st->host_stream && cudaStreamCreateWithFlags(&st->host_stream, cudaStreamNonBlocking) != cudaSuccess)
+            return GAR_ERR_CUDA;
     }
-    if (st->stage_out_elems < size_t(d)) {
-        if (st->stage_out) cudaFree(st->stage_out);
-        st->stage_out = nullptr; st->stage_out_elems = 0;
-        if (cudaMalloc(&st->stage_out, size_t(d) * sizeof(float)) != cudaSuccess) return GAR_ERR_CUDA;
-        st->stage_out_elems = size_t(d);
-    }
-    if (!st->copy_stream) {
-        if (cudaStreamCreateWithFlags(&st->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return GAR_ERR_CUDA;
-        if (cudaStreamCreateWithFlags(&st->compute_stream, cudaStreamNonBlocking) != cudaSuccess) return GAR_ERR_CUDA;
-        if (cudaEventCreateWithFlags(&st->computed, cudaEventDisableTiming) != cudaSuccess) return GAR_ERR_CUDA;
-    }
-    // One bulk 2-D copy (row pitch d on both sides), then the device path; the
-    // result goes back on the same stream.
-    cudaStream_t s = st->compute_stream;
+    // rows in (one contiguous copy), the three kernels, the result and the selection's status out
+    cudaStream_t s = st->host_stream;
     if (cudaMemcpyAsync(st->stage_grads, grads, need * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
         return GAR_ERR_CUDA;
     Workspace ws{st->workspace};
     const int theta = default_theta(rule, n, f);
-    rc = enqueue(rule, st->stage_grads, n, f, d, d, st->stage_out, 0, theta, 0, ws, nullptr, nullptr, st->sm_count, s);
+    rc = enqueue(rule, st->stage_grads, n, f, d, d, st->stage_out, 0, theta, 0, GAR_EVEN_MEDIAN_LOWER, GAR_DISTANCES_AUTO,
+                 ws, nullptr, nullptr, st->sm_count, s);
     if (rc != GAR_OK) return rc;
     if (cudaMemcpyAsync(out, st->stage_out, size_t(d) * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return GAR_ERR_CUDA;
+    int32_t status = GAR_OK;
+    if (cudaMemcpyAsync(&status, &ws.selection()->status, sizeof(status), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return GAR_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return GAR_ERR_CUDA;
-    return GAR_OK;
+    return status;
 }
 
 void gar_shutdown(void) {
@@ -292,9 +345,7 @@ void gar_shutdown(void) {
         if (st.workspace) cudaFree(st.workspace);
         if (st.stage_grads) cudaFree(st.stage_grads);
         if (st.stage_out) cudaFree(st.stage_out);
-        if (st.copy_stream) cudaStreamDestroy(st.copy_stream);
-        if (st.compute_stream) cudaStreamDestroy(st.compute_stream);
-        if (st.computed) cudaEventDestroy(st.computed);
+        if (st.host_stream) cudaStreamDestroy(st.host_stream);
         st = DeviceState{};
     }
     cudaSetDevice(cur);

@@ -8,7 +8,10 @@
 namespace gar {
 
 // ---- workspace layout (device) -------------------------------------------
-// [0, 256)                control block (ticket counter of the distance kernel)
+// [0, 256)                control block, 32-bit words: [0] ticket counter of the distance kernel,
+//                          [2] a bounded wait of a distance kernel gave up, [4] path of the last
+//                          distance call (kPath*), [6] gate of the difference-form kernel that follows
+//                          the tensor-core kernel (non-zero: recompute)
 // [256, +partials)        per-CTA partial distance sums, fp64
 // [.., +n*n doubles)      distance matrix
 // [.., +sizeof(selection)) selection result / coordinate-phase schedule
@@ -30,17 +33,25 @@ struct Workspace {
     char* base;
     unsigned int*    ticket()    const { return reinterpret_cast<unsigned int*>(base); }
     unsigned int*    k1_error()  const { return reinterpret_cast<unsigned int*>(base) + 2; }   // a bounded device wait gave up
+    unsigned int*    k1_path()   const { return reinterpret_cast<unsigned int*>(base) + 4; }
+    unsigned int*    k1_gate()   const { return reinterpret_cast<unsigned int*>(base) + 6; }
     double*          partials()  const { return reinterpret_cast<double*>(base + kOffPartials); }
     double*          dist()      const { return reinterpret_cast<double*>(base + kOffDist); }
     gar_selection_t* selection() const { return reinterpret_cast<gar_selection_t*>(base + kOffSelection); }
 };
 
+constexpr unsigned kPathDifference = 0u, kPathGram = 1u, kPathGramRejected = 2u;
+
+// Slots of a CTA's partial-sum block beyond the pair sums.
+constexpr int kSlotRowExp    = 2100;    // .. +63: the tensor-core kernel's final quantisation exponent of each row
+constexpr int kSlotNonfinite = 2300;    // 2300, 2301: masks of rows that hold Inf or NaN
+constexpr int kSlotError     = 2302;    // a bounded wait gave up
+
 // ---- kernel launchers (one per translation unit) --------------------------
 // Pairwise squared distances of n rows over columns [0, d); result in dist[n*n].
-// `accumulate_only`/`finalize` allow the host path to feed column slabs:
-// slab calls add into the workspace partials, the last one finalises.
+// mode: a gar_distance_mode_t.
 cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
-                             const Workspace& ws, int sm_count, cudaStream_t stream);
+                             const Workspace& ws, int sm_count, int mode, cudaStream_t stream);
 
 // Tensor-core variant (tcgen05, accumulators in tensor memory) for 16 < n <= 64 and 16-byte
 // aligned rows, used from kMmaMinDim coordinates on.
@@ -50,12 +61,15 @@ cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t 
 
 // Scoring + iterative selection (and schedule construction) into *sel.
 cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,
-                          int median_of_agr, gar_selection_t* sel, cudaStream_t stream);
+                          int median_of_agr, int even_median, gar_selection_t* sel, cudaStream_t stream);
 cudaError_t launch_schedule_only(gar_selection_t* sel, cudaStream_t stream);
 
 // Coordinate phase.
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
-                              const gar_selection_t* sel, int theta, int preagg, float* out,
+                              gar_selection_t* sel, int theta, int preagg, float* out,
                               int sm_count, cudaStream_t stream);
+
+// One warp waits, bounded, on a barrier nobody arrives on; result[0] = status, result[1] = ns.
+cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t stream);
 
 }  // namespace gar

@@ -22,7 +22,7 @@
 //    the same work.  Every pair sees the same column-to-lane assignment and the
 //    same reduction tree, so identical rows get bit-identical distances.
 //    FMA-pipe-bound.
-#include <cstdlib>
+#include <mutex>
 
 #include "gar_internal.cuh"
 #include "mbar.cuh"
@@ -103,6 +103,48 @@ __device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) {
     return is_last != 0;
 }
 
+// ---- pieces the two direct kernels (n <= 16) share
+// acc[p] += sum_v (x[i][v] - x[j][v])^2 over the pairs p = (0,1), (0,2), .., (0,N-1), (1,2), ..
+template <int N, int V, int NPAD>
+__device__ __forceinline__ void direct_pairs(const float (&x)[N][V], float (&acc)[NPAD]) {
+    int p = 0;
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+#pragma unroll
+        for (int j = i + 1; j < N; ++j) {
+            float t = acc[p];
+#pragma unroll
+            for (int v = 0; v < V; ++v) { const float df = x[i][v] - x[j][v]; t = fmaf(df, df, t); }
+            acc[p] = t;
+            ++p;
+        }
+    }
+}
+// One coordinate t of all rows straight from global memory (ragged ends).
+template <int N, int NPAD>
+__device__ __forceinline__ void direct_tail_coordinate(const float* __restrict__ g, int64_t ld, int64_t t, float (&acc)[NPAD]) {
+    float x[N][1];
+#pragma unroll
+    for (int r = 0; r < N; ++r) x[r][0] = __ldg(g + int64_t(r) * ld + t);
+    direct_pairs<N, 1, NPAD>(x, acc);
+}
+// The warp's fp32 accumulators -> its fp64 sums in shared memory (fixed shuffle tree), then zero.
+template <int NPAD>
+__device__ __forceinline__ void direct_flush(float (&acc)[NPAD], double* warp_sums, int lane, int sbase) {
+    reduce_scatter<NPAD, 32>(acc, lane);
+#pragma unroll
+    for (int i = 0; i < NPAD / 32; ++i) warp_sums[sbase + i] += double(acc[i]);
+#pragma unroll
+    for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
+}
+// Pair index p of direct_pairs -> (i, j).
+template <int N> __device__ __forceinline__ void direct_pair_rows(int p, int& i, int& j) {
+    i = 0;
+    int rem = p;
+    while (rem >= N - 1 - i) { rem -= N - 1 - i; ++i; }
+    j = i + 1 + rem;
+}
+
 // ======================================================== direct kernel, n <= 16
 constexpr int K1R_THREADS = 128;
 constexpr int K1R_FLUSH = 64;       // iterations between fp64 flushes
@@ -126,10 +168,9 @@ template <int N, int V> struct K1RDims {
 template <int N, int V>
 __global__ void __launch_bounds__(K1R_THREADS)
 k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
-          double* __restrict__ partials, unsigned int* __restrict__ ticket) {
+          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word) {
     constexpr int NP = N * (N - 1) / 2;
     constexpr int NPAD = (NP + 31) / 32 * 32;
-    constexpr int PER_LANE = NPAD / 32;
     constexpr int WARPS = K1R_THREADS / 32;
     extern __shared__ __align__(16) float ring[];            // [stage][row][thread][V]
     __shared__ double sums[WARPS][NPAD];
@@ -142,13 +183,7 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
     const int sbase = scatter_base<NPAD, 32>(lane);
 
-    auto flush = [&]() {
-        reduce_scatter<NPAD, 32>(acc, lane);
-#pragma unroll
-        for (int i = 0; i < PER_LANE; ++i) sums[warp][sbase + i] += double(acc[i]);
-#pragma unroll
-        for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
-    };
+    auto flush = [&]() { direct_flush<NPAD>(acc, sums[warp], lane, sbase); };
     // request the rows of vector index vi into ring stage st (zeros past the end)
     auto request = [&](int st, int64_t vi, bool valid) {
         float* slot = ring + (size_t(st) * N * K1R_THREADS + tid) * V;
@@ -173,18 +208,7 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
             else if constexpr (V == 2) { float2 q = *reinterpret_cast<const float2*>(src); x[r][0] = q.x; x[r][1] = q.y; }
             else { x[r][0] = *src; }
         }
-        int p = 0;
-#pragma unroll
-        for (int i = 0; i < N; ++i) {
-#pragma unroll
-            for (int j = i + 1; j < N; ++j) {
-                float t = acc[p];
-#pragma unroll
-                for (int v = 0; v < V; ++v) { const float df = x[i][v] - x[j][v]; t = fmaf(df, df, t); }
-                acc[p] = t;
-                ++p;
-            }
-        }
+        direct_pairs<N, V, NPAD>(x, acc);
     };
 
     // the loop bound is per warp, so that the flush (warp-collective) is uniform
@@ -209,17 +233,7 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     cp_async_wait<0>();
     // ragged tail: the last d % V coordinates, one thread
     if (V > 1 && blockIdx.x == 0 && tid == 0) {
-        for (int64_t t = nvec * V; t < d; ++t) {
-            float x[N];
-#pragma unroll
-            for (int r = 0; r < N; ++r) x[r] = __ldg(g + int64_t(r) * ld + t);
-            int p = 0;
-#pragma unroll
-            for (int i = 0; i < N; ++i) {
-#pragma unroll
-                for (int j = i + 1; j < N; ++j) { const float df = x[i] - x[j]; acc[p] = fmaf(df, df, acc[p]); ++p; }
-            }
-        }
+        for (int64_t t = nvec * V; t < d; ++t) direct_tail_coordinate<N, NPAD>(g, ld, t, acc);
     }
     __syncwarp();
     flush();
@@ -234,15 +248,13 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     }
     if (!last_cta_ticket(ticket)) return;
     reduce_partials(partials, NP, K1R_THREADS, [&](int p, double s) {
-        // pair index -> (i, j), pairs enumerated (0,1),(0,2),..,(0,N-1),(1,2),..
-        int i = 0, rem = p;
-        while (rem >= N - 1 - i) { rem -= N - 1 - i; ++i; }
-        const int j = i + 1 + rem;
+        int i, j;
+        direct_pair_rows<N>(p, i, j);
         dist[i * N + j] = s;
         dist[j * N + i] = s;
     });
     for (int i = tid; i < N; i += K1R_THREADS) dist[i * N + i] = 0.0;
-    if (tid == 0) *ticket = 0u;               // ready for the next call
+    if (tid == 0) { *ticket = 0u; *path_word = kPathDifference; }   // ready for the next call
 }
 
 // ================================================ direct kernel, n <= 16, rows staged by bulk copies
@@ -253,7 +265,7 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
 // size keep HBM busier than 16-byte requests per thread do.  Needs 16-byte aligned rows
 // (base address and row stride); coordinates after the last whole tile are added by CTA 0 with
 // plain loads.  A wait that gives up (bounded) raises the CTA's error slot: the last CTA then
-// fills the matrix with NaN and sets the workspace's error word.
+// fills the matrix, diagonal included, with NaN and sets the workspace's error word.
 constexpr int K1B_CT = 256;                    // compute threads
 constexpr int K1B_THREADS = K1B_CT + 32;       // + the producer warp
 constexpr int K1B_TC = K1B_CT * 4;             // coordinates per tile
@@ -264,10 +276,10 @@ constexpr int K1B_BAR_COMPUTE = 1;
 template <int N>
 __global__ void __launch_bounds__(K1B_THREADS)
 k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
-               double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word) {
+               double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
+               unsigned int* __restrict__ path_word) {
     constexpr int NP = N * (N - 1) / 2;
     constexpr int NPAD = (NP + 31) / 32 * 32;
-    constexpr int PER_LANE = NPAD / 32;
     constexpr int WARPS = K1B_CT / 32;
     constexpr unsigned STAGE_BYTES = unsigned(N) * K1B_ROW_BYTES;
     extern __shared__ __align__(128) unsigned char stages[];          // [stage][row][K1B_TC floats]
@@ -312,13 +324,7 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
 #pragma unroll
         for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
         const int sbase = scatter_base<NPAD, 32>(lane);
-        auto flush = [&]() {
-            reduce_scatter<NPAD, 32>(acc, lane);
-#pragma unroll
-            for (int i = 0; i < PER_LANE; ++i) sums[warp][sbase + i] += double(acc[i]);
-#pragma unroll
-            for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
-        };
+        auto flush = [&]() { direct_flush<NPAD>(acc, sums[warp], lane, sbase); };
         int st = 0, since = 0;
         unsigned parity = 0;
         for (int64_t it = 0; it < mine; ++it) {
@@ -337,34 +343,13 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
             }
             __syncwarp();                         // the rows are in registers: hand the stage back
             if (lane == 0) kb_arrive(&empty[st]);
-            int p = 0;
-#pragma unroll
-            for (int i = 0; i < N; ++i) {
-#pragma unroll
-                for (int j = i + 1; j < N; ++j) {
-                    float t = acc[p];
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) { const float df = x[i][v] - x[j][v]; t = fmaf(df, df, t); }
-                    acc[p] = t;
-                    ++p;
-                }
-            }
+            direct_pairs<N, 4, NPAD>(x, acc);
             if (++since == K1R_FLUSH) { flush(); since = 0; }
             if (++st == K1B_STAGES) { st = 0; parity ^= 1u; }
         }
         // coordinates after the last whole tile: CTA 0, plain loads
         if (blockIdx.x == 0) {
-            for (int64_t t = ntiles * K1B_TC + tid; t < d; t += K1B_CT) {
-                float x[N];
-#pragma unroll
-                for (int r = 0; r < N; ++r) x[r] = __ldg(g + int64_t(r) * ld + t);
-                int p = 0;
-#pragma unroll
-                for (int i = 0; i < N; ++i) {
-#pragma unroll
-                    for (int j = i + 1; j < N; ++j) { const float df = x[i] - x[j]; acc[p] = fmaf(df, df, acc[p]); ++p; }
-                }
-            }
+            for (int64_t t = ntiles * K1B_TC + tid; t < d; t += K1B_CT) direct_tail_coordinate<N, NPAD>(g, ld, t, acc);
         }
         __syncwarp();
         flush();
@@ -378,28 +363,28 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
         for (int w = 0; w < WARPS; ++w) s += sums[w][i];
         my_partial[i] = s;
     }
-    if (tid == 0) my_partial[2302] = double(error_flag);
+    if (tid == 0) my_partial[kSlotError] = double(error_flag);
     if (!last_cta_ticket(ticket)) return;
     __shared__ int any_error;
     if (tid == 0) {
         unsigned err = 0u;
-        for (unsigned b = 0; b < gridDim.x; ++b) err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2302));
+        for (unsigned b = 0; b < gridDim.x; ++b) err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + kSlotError));
         any_error = int(err);
         if (err) *error_word = 1u;
     }
     __syncthreads();
     const bool failed = any_error != 0;
+    const double nan = __longlong_as_double(0x7ff8000000000000ll);
     reduce_partials(partials, NP, K1B_THREADS, [&](int p, double s) {
-        // pair index -> (i, j), pairs enumerated (0,1),(0,2),..,(0,N-1),(1,2),..
-        int i = 0, rem = p;
-        while (rem >= N - 1 - i) { rem -= N - 1 - i; ++i; }
-        const int j = i + 1 + rem;
-        if (failed) s = __longlong_as_double(0x7ff8000000000000ll);
+        int i, j;
+        direct_pair_rows<N>(p, i, j);
+        if (failed) s = nan;
         dist[i * N + j] = s;
         dist[j * N + i] = s;
     });
-    for (int i = tid; i < N; i += K1B_THREADS) dist[i * N + i] = 0.0;
-    if (tid == 0) *ticket = 0u;               // ready for the next call
+    // a NaN diagonal tells the selection kernel that the matrix is not to be used
+    for (int i = tid; i < N; i += K1B_THREADS) dist[i * N + i] = failed ? nan : 0.0;
+    if (tid == 0) { *ticket = 0u; *path_word = kPathDifference; }   // ready for the next call
 }
 
 // ========================================================= tiled kernel, n > 16
@@ -470,7 +455,11 @@ __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ 
 template <int NB, bool VEC>
 __global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
 k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
-         double* __restrict__ partials, unsigned int* __restrict__ ticket) {
+         double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
+         const unsigned int* __restrict__ gate) {
+    // launched behind the tensor-core kernel, this one only runs if that kernel rejected its own
+    // result (the gate word is written before this grid starts: same stream)
+    if (gate != nullptr && *gate == 0u) return;
     using D = K1Dims<NB>;
     constexpr int NSTAGE = D::NSTAGE;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -637,7 +626,10 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
         }
     });
     for (int i = tid; i < n; i += D::THREADS) dist[i * n + i] = 0.0;
-    if (tid == 0) *ticket = 0u;               // ready for the next call
+    if (tid == 0) {
+        *ticket = 0u;                           // ready for the next call
+        if (gate == nullptr) *path_word = kPathDifference;
+    }
 }
 
 // ------------------------------------------------------------------ launchers
@@ -673,14 +665,15 @@ cudaError_t persistent_grid(K kern, int threads, size_t smem, int sm_count, int*
 
 template <int NB, bool VEC>
 cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
-                         int sm_count, cudaStream_t stream) {
+                         int sm_count, bool gated, cudaStream_t stream) {
     using D = K1Dims<NB>;
     static int per_sm_cache[64] = {0};
     int64_t grid = 1;
     cudaError_t err = persistent_grid(k1_tiled<NB, VEC>, D::THREADS, D::SMEM_BYTES, sm_count, per_sm_cache,
                                       (d + D::TK - 1) / D::TK, &grid);
     if (err != cudaSuccess) return err;
-    k1_tiled<NB, VEC><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket());
+    k1_tiled<NB, VEC><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket(),
+                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr);
     return cudaGetLastError();
 }
 
@@ -694,7 +687,7 @@ cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, c
     cudaError_t err = persistent_grid(k1_direct<N, V>, K1R_THREADS, smem, sm_count, per_sm_cache,
                                       (nvec + K1R_THREADS - 1) / K1R_THREADS, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket());
+    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_path());
     return cudaGetLastError();
 }
 
@@ -706,7 +699,8 @@ cudaError_t launch_direct_bulk(const float* g, int64_t d, int64_t ld, double* di
     int64_t grid = 0;
     cudaError_t err = persistent_grid(k1_direct_bulk<N>, K1B_THREADS, smem, sm_count, per_sm_cache, d / K1B_TC, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct_bulk<N><<<unsigned(grid), K1B_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error());
+    k1_direct_bulk<N><<<unsigned(grid), K1B_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
+                                                                     ws.k1_path());
     return cudaGetLastError();
 }
 
@@ -714,8 +708,7 @@ template <int N>
 cudaError_t launch_direct_n(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                             cudaStream_t stream, int vec) {
     // 16-byte aligned rows and enough whole tiles for every SM: rows staged by bulk copies
-    static const char* env = std::getenv("GAR_K1_BULK");            // tuning aid: 0 = off
-    if (vec >= 4 && d >= int64_t(sm_count) * K1B_TC && !(env && std::atoi(env) == 0))
+    if (vec >= 4 && d >= int64_t(sm_count) * K1B_TC)
         return launch_direct_bulk<N>(g, d, ld, dist, ws, sm_count, stream);
     // few rows: wide vectors keep enough bytes in flight; many rows: narrow ones keep the registers in check
     if constexpr (N <= 8) {
@@ -728,33 +721,33 @@ cudaError_t launch_direct_n(const float* g, int64_t d, int64_t ld, double* dist,
 }  // namespace
 
 cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
-                             const Workspace& ws, int sm_count, cudaStream_t stream) {
+                             const Workspace& ws, int sm_count, int mode, cudaStream_t stream) {
     const uintptr_t addr = reinterpret_cast<uintptr_t>(grads);
     int vec = 1;
     if (addr % 16 == 0 && ld % 4 == 0) vec = 4;
     else if (addr % 8 == 0 && ld % 2 == 0) vec = 2;
-    static const char* env = std::getenv("GAR_K1_VEC");   // tuning aid: cap the vector width
-    if (env) {
-        const int cap = std::atoi(env);
-        if ((cap == 1 || cap == 2) && n <= 16) vec = vec < cap ? vec : cap;
-    }
     if (n == 1) return cudaMemsetAsync(dist, 0, sizeof(double), stream);
-    // many rows and a long dimension: exact integer Gram product on the tensor cores (HBM-bound);
-    // short dimensions keep the FP32 difference form, whose per-term error does not rely on averaging
-    static const bool no_mma = std::getenv("GAR_K1_NO_MMA") != nullptr;   // tuning aid: CUDA-core kernel instead
-    if (n > 16 && vec == 4 && d >= kMmaMinDim && !no_mma)
-        return launch_distances_umma(grads, n, d, ld, dist, ws, sm_count, stream);
 #define GAR_K1_DIRECT(NV) case NV: return launch_direct_n<NV>(grads, d, ld, dist, ws, sm_count, stream, vec);
-#define GAR_K1_TILED(NBV)                                                                          \
-    case NBV:                                                                                      \
-        return vec == 4 ? launch_tiled<NBV, true>(grads, n, d, ld, dist, ws, sm_count, stream)      \
-                        : launch_tiled<NBV, false>(grads, n, d, ld, dist, ws, sm_count, stream);
+#define GAR_K1_TILED(NBV)                                                                                  \
+    case NBV:                                                                                              \
+        return vec == 4 ? launch_tiled<NBV, true>(grads, n, d, ld, dist, ws, sm_count, gated, stream)       \
+                        : launch_tiled<NBV, false>(grads, n, d, ld, dist, ws, sm_count, gated, stream);
     if (n <= 16) {
         switch (n) {
             GAR_K1_DIRECT(2) GAR_K1_DIRECT(3) GAR_K1_DIRECT(4) GAR_K1_DIRECT(5) GAR_K1_DIRECT(6) GAR_K1_DIRECT(7)
             GAR_K1_DIRECT(8) GAR_K1_DIRECT(9) GAR_K1_DIRECT(10) GAR_K1_DIRECT(11) GAR_K1_DIRECT(12)
             GAR_K1_DIRECT(13) GAR_K1_DIRECT(14) GAR_K1_DIRECT(15) GAR_K1_DIRECT(16)
         }
+    }
+    // Many rows and a long dimension: exact integer Gram product of rounded rows on the tensor
+    // cores (HBM-bound), followed by the difference-form kernel behind a gate that the first one
+    // opens only if its own bound on the rounding's effect is too large for some pair.  Short
+    // dimensions keep the FP32 difference form, whose per-term error does not rely on averaging.
+    bool gated = false;
+    if (n > 16 && vec == 4 && d >= kMmaMinDim && mode == GAR_DISTANCES_AUTO) {
+        const cudaError_t err = launch_distances_umma(grads, n, d, ld, dist, ws, sm_count, stream);
+        if (err != cudaSuccess) return err;
+        gated = true;
     }
     switch ((n + 7) / 8) {
         GAR_K1_TILED(3) GAR_K1_TILED(4) GAR_K1_TILED(5) GAR_K1_TILED(6) GAR_K1_TILED(7) GAR_K1_TILED(8)
@@ -789,6 +782,7 @@ struct StaticScratchState {
     int   sm_count = 0;
 };
 StaticScratchState g_static_state[64];
+std::mutex g_static_mutex;             // guards the once-per-device set-up below
 }  // namespace
 
 }  // namespace gar
@@ -803,6 +797,7 @@ extern "C" int gar_pairwise_distances_static(const float* grads, int n, int64_t 
     if (cudaGetDevice(&dev) != cudaSuccess) return GAR_ERR_CUDA;
     if (dev < 0 || dev >= 64) return GAR_ERR_UNSUPPORTED;
     gar::StaticScratchState& st = gar::g_static_state[dev];
+    std::unique_lock<std::mutex> lock(gar::g_static_mutex);
     if (!st.ready) {
         // Once per device, with that device current: in host code the array's name is only a
         // stand-in; the address the kernels need comes from the runtime.
@@ -813,10 +808,11 @@ extern "C" int gar_pairwise_distances_static(const float* grads, int n, int64_t 
         st.ptr = static_cast<char*>(p);
         st.ready = true;
     }
+    lock.unlock();
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps the previous call's contents: the ticket counter must start at zero
     // (the partial sums are overwritten before they are read)
     if (cudaMemsetAsync(st.ptr, 0, gar::kCtrlBytes, s) != cudaSuccess) return GAR_ERR_CUDA;
     gar::Workspace ws{st.ptr};
-    return gar::launch_distances(grads, n, d, ld, dist, ws, st.sm_count, s) == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return gar::launch_distances(grads, n, d, ld, dist, ws, st.sm_count, GAR_DISTANCES_AUTO, s) == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }

@@ -30,6 +30,7 @@
 #include <cstdlib>
 
 #include "gar_internal.cuh"
+#include "mbar.cuh"
 
 namespace gar {
 namespace {
@@ -46,9 +47,9 @@ constexpr int KU_SET_COLS = 256;             // tensor-memory columns per accumu
 constexpr int KU_FLUSH_WARPS = 4;            // warps 0..3: tensor-memory lanes 32 w .. 32 w + 31
 constexpr int KU_MMA_WARP = 4;
 constexpr int KU_FIRST_PRODUCER = 5;
-constexpr unsigned KU_SPIN_LIMIT = 1u << 20; // suspended waits of a barrier before a wait gives up
 constexpr int KU_BAR_FLUSH = 1;              // named barrier of the flush warps
 constexpr int KU_TRI = 2080;
+constexpr double kGramRelBound = 1e-6;      // largest accepted bound on a distance's relative rounding error
 
 struct KUSmem {
     unsigned long long full[KU_NBUF];        // producers -> MMA warp: the buffer's tiles are written
@@ -64,50 +65,11 @@ struct KUSmem {
     int      set_exp[2][64];                 // exponents of the rows while the set was accumulated
     unsigned nonfinite_lo, nonfinite_hi;
     int      is_last;
+    int      final_exp[64];                  // exponent each row ended with in this CTA (they only grow)
+    int      reject;                         // last CTA: some distance's rounding bound is too large
 };
 
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// One wait for the phase with the given parity: the thread is suspended in the barrier unit until the
-// phase completes or a hardware time limit passes, whichever comes first; true if it completed.
-__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
-    unsigned done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return done != 0;
-}
-__device__ __forceinline__ bool mbar_test(unsigned long long* bar, unsigned parity) {
-    unsigned done;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return done != 0;
-}
-// Bounded wait for the phase with the given parity, the same answer in every lane of the warp.
-// `polls` quick tests first (a hand-off that is about to happen is seen soonest that way, which
-// matters when the whole kernel is a few dozen slabs), then suspended waits: a warp that waits long
-// sleeps in the barrier unit and leaves the issue slots to the working ones.
-// False: the wait gave up (error flag raised) or another role raised the flag.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* error,
-                                          unsigned polls = 64, unsigned limit = KU_SPIN_LIMIT) {
-    bool ok = false;
-    for (unsigned spin = 0; spin < polls; ++spin) {
-        if (mbar_test(bar, parity)) { ok = true; break; }
-    }
-    if (!ok) {
-        for (unsigned spin = 0; spin < limit; ++spin) {
-            if (mbar_try_wait(bar, parity)) { ok = true; break; }
-            if (*error) break;
-            if (spin + 1 == limit) *error = 1;
-        }
-    }
-    return __all_sync(0xffffffffu, ok);
-}
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return kb_smem_u32(p); }
 
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -181,7 +143,8 @@ template <int NST, int MAXT, bool FULL>
 __global__ void __launch_bounds__(MAXT, 1)
 k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
         double* __restrict__ partials, unsigned int* __restrict__ ticket,
-        unsigned int* __restrict__ error_word) {
+        unsigned int* __restrict__ error_word, unsigned int* __restrict__ path_word,
+        unsigned int* __restrict__ gate_word) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     KUSmem& sm = *reinterpret_cast<KUSmem*>(smem_raw);
     constexpr int HEAD = (int(sizeof(KUSmem)) + 127) & ~127;
@@ -201,22 +164,23 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         for (int b = 0; b < KU_NBUF; ++b) sm.slab_exp[b][tid] = KU_MIN_EXP;
         sm.set_exp[0][tid] = KU_MIN_EXP;
         sm.set_exp[1][tid] = KU_MIN_EXP;
+        sm.final_exp[tid] = KU_MIN_EXP;
     }
     if (tid == 0) {
 #pragma unroll
         for (int b = 0; b < KU_NBUF; ++b) {
-            mbar_init(&sm.full[b], unsigned(pw));
-            mbar_init(&sm.empty[b], 1u);
+            kb_init(&sm.full[b], unsigned(pw));
+            kb_init(&sm.empty[b], 1u);
             sm.grow[b] = 0;
         }
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
-            mbar_init(&sm.accfull[s], 1u);
-            mbar_init(&sm.accfree[s], unsigned(KU_FLUSH_WARPS));
+            kb_init(&sm.accfull[s], 1u);
+            kb_init(&sm.accfree[s], unsigned(KU_FLUSH_WARPS));
             sm.set_last[s] = 0;
         }
         sm.error = 0; sm.nonfinite_lo = 0u; sm.nonfinite_hi = 0u; sm.is_last = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        kb_fence_init();
     }
     // the MMA warp's loop is one dependent instruction stream per slab and sits on the kernel's
     // critical path: everything it can look up instead of compute is tabulated here
@@ -342,7 +306,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
                 exp_stores = KU_NBUF;                // every tile buffer gets the new exponents once
             }
             // the MMAs that read this buffer three slabs ago are done
-            if (!mbar_wait(&sm.empty[buf], empty_parity, error)) break;
+            if (!kb_wait_warp(kb_smem_u32(&sm.empty[buf]), empty_parity, error)) break;
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
                 if (valid[jr]) {
@@ -365,11 +329,16 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             if (grew && lane == 0) sm.grow[buf] = 1;
             fence_async_smem();                      // generic-proxy stores -> visible to the tensor core's reads
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.full[buf]);
+            if (lane == 0) kb_arrive(&sm.full[buf]);
             buf_off += KU_BUF_BYTES;
             if (++buf == KU_NBUF) { buf = 0; buf_off = 0; empty_parity ^= 1u; }
         }
         cp_async_wait<0>();
+        if (lane == 0) {
+#pragma unroll
+            for (int jr = 0; jr < KU_JR; ++jr)
+                if (valid[jr]) sm.final_exp[p + jr * pw] = row_exp[jr];
+        }
     } else if (warp == KU_MMA_WARP) {
         // ================================================================ MMA issue
         constexpr unsigned IDESC_A = umma_idesc(128, 192), IDESC_B = umma_idesc(128, 64);
@@ -380,7 +349,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         int buf = 0;
         unsigned full_parity = 0;
         for (int64_t it = 0; it < mine; ++it) {
-            if (!mbar_wait(&sm.full[buf], full_parity, error)) break;
+            if (!kb_wait_warp(kb_smem_u32(&sm.full[buf]), full_parity, error)) break;
             tc_fence_after();
             const bool grow = *reinterpret_cast<volatile int*>(&sm.grow[buf]) != 0;
             if (!have_open || grow || since == KU_PERIOD) {
@@ -390,7 +359,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
                     set ^= 1;
                 }
                 const int opened = set ? opened1 : opened0;
-                if (opened > 0 && !mbar_wait(&sm.accfree[set], unsigned(opened - 1) & 1u, error)) break;
+                if (opened > 0 && !kb_wait_warp(kb_smem_u32(&sm.accfree[set]), unsigned(opened - 1) & 1u, error)) break;
                 tc_fence_after();
                 sm.set_exp[set][lane] = sm.slab_exp[buf][lane];
                 sm.set_exp[set][lane + 32] = sm.slab_exp[buf][lane + 32];
@@ -437,7 +406,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         for (int k = 0;; ++k) {
             const int set = k & 1;
             // a set closes rarely: poll slowly; then agree over the four warps (they meet at named barriers below)
-            const bool ok = mbar_wait(&sm.accfull[set], unsigned(k >> 1) & 1u, error, 0u);
+            const bool ok = kb_wait_warp(kb_smem_u32(&sm.accfull[set]), unsigned(k >> 1) & 1u, error, 0u);
             unsigned all_ok;
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(all_ok) : "r"(unsigned(ok)), "r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
@@ -487,7 +456,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.accfree[set]);
+            if (lane == 0) kb_arrive(&sm.accfree[set]);
             if (last) break;
         }
     }
@@ -497,8 +466,8 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     if (warp == KU_MMA_WARP) tmem_dealloc(tmem_base, 2 * KU_SET_COLS);
 
     // CTA partial: P_ij = px_ij + (pz_ij + pz_ji) for i <= j (the same expression on the diagonal, so
-    // identical rows give bit-identical P_ii, P_ij, P_jj); slots 2300/2301: non-finite row masks,
-    // 2302: error flag
+    // identical rows give bit-identical P_ii, P_ij, P_jj); then the rows' final exponents, the
+    // non-finite row masks and the error flag
     double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
     for (int idx = tid; idx < 64 * 64; idx += nthreads) {
         const int i = idx >> 6, j = idx & 63;
@@ -508,10 +477,11 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             my_partial[tri_slot(i, j)] = v;
         }
     }
+    if (tid < 64) my_partial[kSlotRowExp + tid] = double(sm.final_exp[tid]);
     if (tid == 0) {
-        my_partial[2300] = double(sm.nonfinite_lo);
-        my_partial[2301] = double(sm.nonfinite_hi);
-        my_partial[2302] = double(sm.error);
+        my_partial[kSlotNonfinite] = double(sm.nonfinite_lo);
+        my_partial[kSlotNonfinite + 1] = double(sm.nonfinite_hi);
+        my_partial[kSlotError] = double(sm.error);
     }
     __threadfence();
     __syncthreads();
@@ -537,16 +507,30 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     if (tid == 0) {
         unsigned lo = 0u, hi = 0u, err = 0u;
         for (unsigned b = 0; b < gridDim.x; ++b) {
-            lo |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2300));
-            hi |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2301));
-            err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + 2302));
+            lo |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + kSlotNonfinite));
+            hi |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + kSlotNonfinite + 1));
+            err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + kSlotError));
         }
         sm.nonfinite_lo = lo; sm.nonfinite_hi = hi; sm.error = int(err);
         if (err) *error_word = 1u;
     }
+    if (tid >= 64 && tid < 128) {                 // the coarsest grid any CTA used for each row
+        int e = KU_MIN_EXP;
+        for (unsigned b = 0; b < gridDim.x; ++b) e = max(e, int(__ldcg(partials + size_t(b) * kPairSlots + kSlotRowExp + (tid - 64))));
+        sm.final_exp[tid - 64] = e;
+    }
     __syncthreads();
     const unsigned long long bad = (static_cast<unsigned long long>(sm.nonfinite_hi) << 32) | sm.nonfinite_lo;
     const bool failed = sm.error != 0;
+    // What the rounding of the rows can have done to a distance.  With steps s_i, s_j (the coarsest
+    // each row saw) the rounding errors e_i, e_j of a coordinate lie within half a step:
+    //   D'_ij - D_ij = sum (e_i - e_j)^2 + 2 sum (x_i - x_j)(e_i - e_j),
+    // a bias of at most d (s_i^2 + s_j^2) / 12 on average and a zero-mean term of standard deviation
+    // 2 sqrt(D_ij (s_i^2 + s_j^2) / 12) when the errors are independent of the differences; six
+    // standard deviations are allowed for.  A pair whose bound exceeds 1e-6 of its distance rejects
+    // the matrix (the caller's next kernel recomputes it from differences).  Rows that agree within
+    // the grid everywhere give exactly 0 and are left at that.
+    bool reject = false;
     for (int idx = tid; idx < n * n; idx += nthreads) {
         const int i = idx / n, j = idx - i * n;
         double v = 0.0;
@@ -554,11 +538,23 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             const int lo = i < j ? i : j, hi = i < j ? j : i;
             v = ptot[tri_slot(lo, lo)] + ptot[tri_slot(hi, hi)] - 2.0 * ptot[tri_slot(lo, hi)];
             if (v < 0.0) v = 0.0;
-            if (((bad >> i) | (bad >> j)) & 1ull) v = INFINITY;
+            if (((bad >> i) | (bad >> j)) & 1ull) {
+                v = INFINITY;
+            } else if (v > 0.0) {
+                const double m2 = pow2(2 * (sm.final_exp[i] - 148)) + pow2(2 * (sm.final_exp[j] - 148));
+                const double bound = double(d) * m2 * (1.0 / 12.0) + 12.0 * sqrt(v * m2 * (1.0 / 12.0));
+                reject |= bound > kGramRelBound * v;
+            }
         }
         dist[idx] = failed ? __longlong_as_double(0x7ff8000000000000ll) : v;
     }
-    if (tid == 0) *ticket = 0u;               // ready for the next call
+    const int any_reject = __syncthreads_or(reject ? 1 : 0);
+    if (tid == 0) {
+        const bool redo = any_reject && !failed;
+        *gate_word = redo ? 1u : 0u;
+        *path_word = redo ? kPathGramRejected : kPathGram;
+        *ticket = 0u;                           // ready for the next call
+    }
 }
 
 template <int NST, int MAXT, bool FULL>
@@ -580,7 +576,7 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     if (grid > kMaxCtasK1) grid = kMaxCtasK1;
     if (grid > nslabs) grid = nslabs;
     k1_umma<NST, MAXT, FULL><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
-        g, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error());
+        g, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(), ws.k1_path(), ws.k1_gate());
     return cudaGetLastError();
 }
 

@@ -186,7 +186,7 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
 
 __global__ void __launch_bounds__(K2_THREADS)
 k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, int rule, int n, int f,
-          int m_user, int theta, int beta, int median_of_agr) {
+          int m_user, int theta, int beta, int median_of_agr, int even_median) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     K2Smem& sm = *reinterpret_cast<K2Smem*>(smem_raw);
     __shared__ PlanSmem plan_smem;
@@ -197,6 +197,8 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         sel->n = n; sel->f = f; sel->rule = rule; sel->theta = theta; sel->beta = beta;
         sel->preagg = preagg ? 1 : 0;
         sel->median_of_agr = median_of_agr;
+        sel->even_median = even_median;
+        sel->reserved = 0;
         sel->status = GAR_OK;
     }
 
@@ -214,15 +216,21 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         return;
     }
 
-    // 1. load
+    // 1. load.  A NaN on the diagonal is how a distance kernel that gave up on a wait marks its
+    // matrix: nothing is selected from it (selecting by index from all-infinite scores would hand
+    // arbitrary, possibly Byzantine, gradients to the coordinate phase as if nothing had happened).
+    bool poisoned = false;
     for (int idx = tid; idx < n * n; idx += K2_THREADS) {
         const int i = idx / n, j = idx - i * n;
         double v = dist[idx];
+        if (i == j) { poisoned |= (v != v); v = 0.0; }
         if (!isfinite(v)) v = INFINITY;
-        if (i == j) v = 0.0;
         sm.dm[i][j] = v;
     }
-    __syncthreads();
+    if (__syncthreads_or(poisoned ? 1 : 0)) {
+        if (tid == 0) sel->status = GAR_ERR_TIMEOUT;
+        return;
+    }
     // 2. sort every row's other entries on (value, index) by counting
     for (int idx = tid; idx < n * n; idx += K2_THREADS) {
         const int i = idx / n, j = idx - i * n;
@@ -325,7 +333,7 @@ __global__ void __launch_bounds__(64) k2_schedule_only(gar_selection_t* sel) {
 }  // namespace
 
 cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,
-                          int median_of_agr, gar_selection_t* sel, cudaStream_t stream) {
+                          int median_of_agr, int even_median, gar_selection_t* sel, cudaStream_t stream) {
     static bool configured[64] = {false};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -335,7 +343,7 @@ cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k2_select<<<1, K2_THREADS, sizeof(K2Smem), stream>>>(dist, sel, rule, n, f, m, theta, beta, median_of_agr);
+    k2_select<<<1, K2_THREADS, sizeof(K2Smem), stream>>>(dist, sel, rule, n, f, m, theta, beta, median_of_agr, even_median);
     return cudaGetLastError();
 }
 

@@ -46,6 +46,7 @@ struct KBPlan {
     KBSlot   slot[GAR_MAX_N];
     int64_t  roff[GAR_MAX_N];                 // staged row -> element offset of its gradient
     int      theta, beta, median_of_agr, lo_pads;
+    int      even_mean, median_only;
     int      nrows, nbase, ncorr, nstages;
     int      cols_in_stage;                   // the correction columns reuse dead rows of the stage
     uint8_t  col_row[GAR_MAX_N + 1];          // correction column -> row that holds it
@@ -61,13 +62,22 @@ struct KBPlan {
 // [correction columns (ncorr + 1) x TC floats] [stages: nrows x TC floats each].
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(KBShape<V>::THREADS)
-k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t* __restrict__ sel,
+k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64_t ld, gar_selection_t* __restrict__ sel,
         float* __restrict__ out, int pool_bytes) {
     constexpr int KB_TC = KBShape<V>::TC, KB_CT = KBShape<V>::CT, KB_THREADS = KBShape<V>::THREADS;
     constexpr int KB_ROW_BYTES = KBShape<V>::ROW_BYTES;
     __shared__ KBPlan plan;
     extern __shared__ __align__(128) unsigned char kb_dyn[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    {
+        const int status = k3_check(sel, n, theta_arg, PREAGG);
+        if (status != GAR_OK) {                   // nothing usable: the output says so
+            for (int64_t i = blockIdx.x; i < ntiles; i += gridDim.x)
+                for (int c = tid; c < KB_TC; c += KB_THREADS) out[i * KB_TC + c] = CUDART_NAN_F;
+            if (blockIdx.x == 0 && tid == 0 && sel->status == GAR_OK) sel->status = status;
+            return;
+        }
+    }
     const int theta = EXACT ? P : sel->theta;
 
     // ---- plan -----------------------------------------------------------------------------
@@ -107,6 +117,8 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
         plan.theta = theta;
         plan.beta = sel->beta;
         plan.median_of_agr = sel->median_of_agr;
+        plan.even_mean = sel->even_median == GAR_EVEN_MEDIAN_MEAN ? 1 : 0;
+        plan.median_only = sel->rule == GAR_MEDIAN ? 1 : 0;
         plan.lo_pads = (P - 1) / 2 - (theta - 1) / 2;
         plan.error = 0;
         // Corrections: column 0 holds zero, column j + 1 the j-th sum that has to be formed (a slot
@@ -215,6 +227,7 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
         const float inv_beta = 1.0f / float(beta);
         const int lo_pads = EXACT ? 0 : plan.lo_pads;
         const bool med_agr = PREAGG && plan.median_of_agr != 0;
+        const bool even_mean = plan.even_mean != 0, median_only = plan.median_only != 0;
         int st = 0;
         unsigned parity = 0;
         bool ok = !*error;
@@ -302,7 +315,7 @@ k3_bulk(const float* __restrict__ g, int64_t ntiles, int64_t ld, gar_selection_t
             if (lane == 0)
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(kb_smem_u32(&plan.empty[st])) : "memory");
             float res[V];
-            k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, med_agr, res);
+            k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, med_agr, even_mean, median_only, res);
             store_vec<V>(out + (first + i * step) * KB_TC + tid * V, res);
             if (++st == nstages) { st = 0; parity ^= 1u; }
         }

@@ -39,7 +39,7 @@ constexpr int K3_THREADS = 256;
 constexpr int K3_LOOSE_CAP = 32;      // loose gradients parked in shared memory; more: read from global
 
 struct K3Plan {
-    int      theta, beta, median_of_agr, lo_pads, nbase, nloose, loose_in_smem;
+    int      theta, beta, median_of_agr, lo_pads, nbase, nloose, loose_in_smem, even_mean, median_only;
     unsigned long long chain_mask, corr_mask;
     int64_t  woff[GAR_MAX_N];       // slot -> winner row offset (elements)
     int64_t  boff[GAR_MAX_N];       // base row offsets
@@ -77,7 +77,8 @@ __device__ __forceinline__ void cmpswap(float& lo, float& hi) {
 
 // Comparator list of Batcher's odd-even merge sort for any N (ascending), built
 // at compile time and pruned to the comparators that the output at index
-// (N-1)/2 depends on (walked backwards from that output).
+// (N-1)/2 -- and, for even N, the one at N/2 -- depends on (walked backwards from
+// those outputs): the lower and the upper middle value.
 template <int N> struct MedianNet {
     static constexpr int MAXC = (N < 4) ? 8 : N * 10;
     struct Data {
@@ -99,6 +100,7 @@ template <int N> struct MedianNet {
                         }
         bool live[N > 0 ? N : 1] = {};
         live[(N - 1) / 2] = true;
+        live[N / 2] = true;
         bool keep[MAXC] = {};
         for (int c = cnt - 1; c >= 0; --c) {
             if (live[all.a[c]] || live[all.b[c]]) {
@@ -127,18 +129,20 @@ __device__ __forceinline__ void median_network_apply(float (&x)[N][V], std::inde
     (cmpswap_vec<V>(x[MedianNet<N>::data.a[C]], x[MedianNet<N>::data.b[C]]), ...);
 }
 
-// After the call x[(N-1)/2] holds the lower median; other entries are unspecified.
+// After the call x[(N-1)/2] holds the lower and x[N/2] the upper middle value; other entries are unspecified.
 template <int N, int V> __device__ __forceinline__ void median_network(float (&x)[N][V]) {
     median_network_apply<N, V>(x, std::make_index_sequence<MedianNet<N>::data.count>{});
 }
 
-// Last part of a coordinate's work, on V coordinates at once: M = lower median of the theta real
-// values of e (of a when median_of_a), then the average of the beta values of a closest to M
-// (Algorithm 1, multi-Bulyan: Median, Argpartition, Average).  e and a hold P slots of which the
-// first theta are real; e is destroyed.
+// Last part of a coordinate's work, on V coordinates at once: M = median of the theta real values
+// of e (of a when median_of_a; for an even count the lower middle value, or the mean of the two
+// middle ones when even_mean), then the average of the beta values of a closest to M
+// (Algorithm 1, multi-Bulyan: Median, Argpartition, Average) -- or M itself when median_only (the
+// Median rule).  e and a hold P slots of which the first theta are real; e is destroyed.
 template <int P, int V>
 __device__ __forceinline__ void k3_finish(float (&e)[P][V], float (&a)[P][V], int theta, int beta, float inv_beta,
-                                          int lo_pads, bool median_of_a, float (&res)[V]) {
+                                          int lo_pads, bool median_of_a, bool even_mean, bool median_only,
+                                          float (&res)[V]) {
     // median of the theta real values (lower middle), padding split around them
     float srt[P][V];
 #pragma unroll
@@ -151,12 +155,24 @@ __device__ __forceinline__ void k3_finish(float (&e)[P][V], float (&a)[P][V], in
         }
     }
     median_network<P, V>(srt);
+    // the real values sit at sorted positions lo_pads .. lo_pads + theta - 1: the lower middle one
+    // at (P-1)/2 and, for an even theta (then P is even too), the upper one at P/2
+    float med[V];
+    const bool two = even_mean && (theta & 1) == 0;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+        med[v] = two ? 0.5f * srt[(P - 1) / 2][v] + 0.5f * srt[P / 2][v] : srt[(P - 1) / 2][v];
+    if (median_only) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) res[v] = med[v];
+        return;
+    }
     float key[P][V];
 #pragma unroll
     for (int s = 0; s < P; ++s) {
 #pragma unroll
         for (int v = 0; v < V; ++v)
-            key[s][v] = (s < theta) ? fabsf(a[s][v] - srt[(P - 1) / 2][v]) : CUDART_INF_F;
+            key[s][v] = (s < theta) ? fabsf(a[s][v] - med[v]) : CUDART_INF_F;
     }
 
     // The beta smallest keys.  beta == 1: the minimum key, then one scan that keeps the
@@ -231,6 +247,43 @@ __device__ __forceinline__ void k3_finish(float (&e)[P][V], float (&a)[P][V], in
     for (int v = 0; v < V; ++v) res[v] = sum[v] * inv_beta;
 }
 
+// Checked by every CTA of a coordinate kernel before it forms an address from the selection: the
+// status the selection kernel left, and that the tables agree with the arguments the host chose
+// the kernel by (theta, pre-aggregation) and only name gradients below n.  The whole CTA calls it;
+// the answer (a gar_status_t) is the same in every thread.
+__device__ __forceinline__ int k3_check(const gar_selection_t* __restrict__ sel, int n, int theta, bool preagg) {
+    const int tid = threadIdx.x, nthreads = blockDim.x;
+    const int status = sel->status;
+    bool bad = n < 1 || n > GAR_MAX_N || theta < 1 || theta > GAR_MAX_N;
+    bad |= sel->theta != theta || (sel->preagg != 0) != preagg || sel->beta < 1 || sel->beta > theta;
+    const int nbase = sel->nbase, nloose = sel->nloose, nadds = sel->total_adds;
+    if (preagg) bad |= nbase < 0 || nbase > n || nloose < 0 || nloose > n || nadds < 0 || nadds > GAR_MAX_N * GAR_MAX_N;
+    if (!bad && status == GAR_OK) {
+        for (int s = tid; s < theta; s += nthreads) {
+            bad |= unsigned(sel->winners[s]) >= unsigned(n);
+            if (preagg) {
+                bad |= sel->m[s] < 1 || sel->m[s] > n;
+                const int src = sel->slot_src[s], sv = sel->slot_save[s];
+                bad |= !(src == GAR_SRC_ZERO || src == GAR_SRC_CONT || src < GAR_MAX_SAVED);
+                bad |= !(sv == GAR_SAVE_NONE || sv < GAR_MAX_SAVED);
+            }
+        }
+        if (preagg) {
+            for (int k = tid; k < nbase; k += nthreads) bad |= sel->base_rows[k] >= n;
+            for (int k = tid; k < nloose; k += nthreads) bad |= sel->loose_rows[k] >= n;
+            for (int k = tid; k < nadds; k += nthreads) bad |= sel->add_pos[k] >= nloose;
+            if (tid == 0) {
+                int total = 0;
+                for (int s = 0; s < theta; ++s) total += sel->slot_nadd[s];
+                bad |= total != nadds;
+            }
+        }
+    }
+    const int any_bad = __syncthreads_or(bad ? 1 : 0);
+    if (status != GAR_OK) return status;
+    return any_bad ? GAR_ERR_INVALID_ARG : GAR_OK;
+}
+
 __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* __restrict__ sel, int64_t ld, int P,
                                           bool preagg, int loose_cap) {
     const int tid = threadIdx.x;
@@ -243,6 +296,8 @@ __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* _
         plan.nbase = sel->nbase;
         plan.nloose = sel->nloose;
         plan.loose_in_smem = sel->nloose <= loose_cap ? 1 : 0;
+        plan.even_mean = sel->even_median == GAR_EVEN_MEDIAN_MEAN ? 1 : 0;
+        plan.median_only = sel->rule == GAR_MEDIAN ? 1 : 0;
         plan.chain_mask = sel->chain_mask;
         plan.corr_mask = sel->corr_mask;
     }
@@ -266,10 +321,17 @@ __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* _
 // Dynamic shared memory (PREAGG only): (loose_cap + GAR_MAX_SAVED) * blockDim * V floats.
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(K3_THREADS)
-k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64_t ld,
-              const gar_selection_t* __restrict__ sel, float* __restrict__ out, int loose_cap) {
+k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin, int64_t t_end, int64_t ld,
+              gar_selection_t* __restrict__ sel, float* __restrict__ out, int loose_cap) {
     __shared__ K3Plan plan;
     extern __shared__ __align__(16) float k3_dyn[];
+    const int status = k3_check(sel, n, theta_arg, PREAGG);
+    if (status != GAR_OK) {                       // nothing usable: the output says so
+        for (int64_t t = t_begin + int64_t(blockIdx.x) * blockDim.x + threadIdx.x; t < t_end; t += int64_t(gridDim.x) * blockDim.x)
+            out[t] = CUDART_NAN_F;
+        if (blockIdx.x == 0 && threadIdx.x == 0 && sel->status == GAR_OK) sel->status = status;
+        return;
+    }
     load_plan(plan, sel, ld, P, PREAGG, loose_cap);
     __syncthreads();
     const int theta = EXACT ? P : plan.theta;
@@ -277,6 +339,7 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
     const float inv_beta = 1.0f / float(beta);
     const int lo_pads = EXACT ? 0 : plan.lo_pads;
     const bool med_agr = plan.median_of_agr != 0;
+    const bool even_mean = plan.even_mean != 0, median_only = plan.median_only != 0;
     const int nthreads = blockDim.x;
     // this thread's private columns: loose value u at xcol[u*stride], saved sum k at tcol[k*stride]
     const int stride = nthreads * V;
@@ -403,13 +466,13 @@ k3_coordinate(const float* __restrict__ g, int64_t t_begin, int64_t t_end, int64
         }
 
         float res[V];
-        k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, PREAGG && med_agr, res);
+        k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, PREAGG && med_agr, even_mean, median_only, res);
         store_vec<V>(out + t, res);
     }
 }
 
 template <int P>
-cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
+cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
                         int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 

@@ -1,6 +1,4 @@
 // Chooses the compiled slot count and vector width of the coordinate kernel.
-#include <cstdlib>
-
 #include "gar_internal.cuh"
 
 // Slot counts the coordinate kernel is compiled for (k3_inst.cu is built once
@@ -14,18 +12,18 @@
 namespace gar {
 
 template <int P>
-cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
+cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
                         int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 #define K3_DECL(P)                                                                                              \
     template <>                                                                                                 \
-    cudaError_t launch_k3_p<P>(const float*, int, int64_t, int64_t, const gar_selection_t*, int, int, int, int, \
+    cudaError_t launch_k3_p<P>(const float*, int, int64_t, int64_t, gar_selection_t*, int, int, int, int,       \
                                float*, int, cudaStream_t);                                                      \
     template <> int bulk_ctas_for<P>(int, int, int);
 K3_P_LIST(K3_DECL)
 #undef K3_DECL
 
-cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, const gar_selection_t* sel,
+cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, gar_selection_t* sel,
                               int theta, int preagg, float* out, int sm_count, cudaStream_t stream) {
     const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out);
     int vec_max = 1;                                      // what the alignment allows
@@ -35,25 +33,16 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
     int vec = vec_max;
     if (vec == 4 && theta > 8) vec = 2;
     if (vec == 2 && theta > (preagg ? 12 : 24)) vec = 1;
-    static const char* env = std::getenv("GAR_K3_VEC");   // tuning aid: vector width, if the alignment allows it
-    if (env) {
-        const int want = std::atoi(env);
-        if (want == 1 || want == 2 || want == 4) vec = want < vec_max ? want : vec_max;
-    }
     // Staging through shared memory by bulk copies needs 16-byte aligned row segments.  With
     // pre-aggregation it is the faster kernel at every slot count; without (Bulyan, median, Krum:
     // the winners are all that is read) the register kernel with 2- or 4-wide loads keeps up with
     // memory and wins while the slot count is a compile-time constant, up to 32 slots.
-    static const char* env_bulk = std::getenv("GAR_K3_BULK");          // tuning aids: 0 = off, else the slot count it starts at
-    static const char* env_ctas = std::getenv("GAR_K3_BULK_CTAS");     // CTAs per SM
-    int bulk_from = preagg ? 1 : 33;
-    if (env_bulk) bulk_from = std::atoi(env_bulk) > 0 ? std::atoi(env_bulk) : 1 << 30;
+    const int bulk_from = preagg ? 1 : 33;
     // (a few hundred thousand coordinates amortise its set-up: the plan, the barriers, the first tiles)
-    const bool bulk = vec_max == 4 && theta >= bulk_from && (d >= 400000 || env_bulk);
+    const bool bulk = vec_max == 4 && theta >= bulk_from && d >= 400000;
 #define K3_TRY(P)                                                                                              \
     if (theta <= P) {                                                                                          \
-        int ctas = bulk ? bulk_ctas_for<P>(n, theta, preagg) : 0;                                                      \
-        if (ctas > 0 && env_ctas && std::atoi(env_ctas) > 0 && std::atoi(env_ctas) < ctas) ctas = std::atoi(env_ctas); \
+        const int ctas = bulk ? bulk_ctas_for<P>(n, theta, preagg) : 0;                                        \
         return launch_k3_p<P>(grads, n, d, ld, sel, theta, preagg, vec, ctas, out, sm_count, stream);          \
     }
     K3_P_LIST(K3_TRY)

@@ -42,7 +42,7 @@ static int bulk_ctas(int n, int theta) {
 
 // Full tiles [0, *covered) through the staged kernel, `ctas` CTAs per SM.
 template <int P, bool PREAGG>
-static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta,
+static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta,
                             int ctas, float* out, int sm_count, cudaStream_t stream, int64_t* covered) {
     constexpr bool EXACT = (K3_EXACT != 0);
     constexpr int V = BulkV<PREAGG>::V;
@@ -69,15 +69,14 @@ static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, const 
     }
     int64_t grid = int64_t(sm_count) * ctas;
     if (grid > ntiles) grid = ntiles;
-    k3_bulk<P, EXACT, PREAGG, V><<<unsigned(grid), S::THREADS, pool, stream>>>(g, ntiles, ld, const_cast<gar_selection_t*>(sel),
-                                                                                out, int(pool));
+    k3_bulk<P, EXACT, PREAGG, V><<<unsigned(grid), S::THREADS, pool, stream>>>(g, n, theta, ntiles, ld, sel, out, int(pool));
     *covered = ntiles * S::TC;
     return cudaGetLastError();
 }
 
 // Coordinates [t0, d): t0 is a multiple of 4.
 template <int P, bool PREAGG, int V>
-static cudaError_t run(const float* g, int n, int64_t t0, int64_t d, int64_t ld, const gar_selection_t* sel, float* out,
+static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, int64_t ld, gar_selection_t* sel, float* out,
                        int sm_count, cudaStream_t stream) {
     constexpr bool EXACT = (K3_EXACT != 0);
     int threads = K3_THREADS, threads1 = K3_THREADS;
@@ -109,17 +108,17 @@ static cudaError_t run(const float* g, int n, int64_t t0, int64_t d, int64_t ld,
         int64_t blocks = (nvec + threads - 1) / threads;
         const int64_t cap = int64_t(sm_count) * 8;
         if (blocks > cap) blocks = cap;
-        k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, t0, d_vec, ld, sel, out,
+        k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, n, theta, t0, d_vec, ld, sel, out,
                                                                                          loose_cap);
     }
     if (d_vec < d) {   // ragged tail (only when ld > d): scalar kernel on the last d % V coordinates
-        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, d_vec, d, ld, sel, out, loose_cap);
+        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap);
     }
     return cudaGetLastError();
 }
 
 template <>
-cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, const gar_selection_t* sel, int theta, int preagg,
+cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
                               int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream) {
     int64_t t0 = 0;
     if (bulk_ctas > 0) {                         // whole tiles staged through shared memory, the rest below
@@ -132,13 +131,13 @@ cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, cons
     constexpr bool kWide = (K3_P <= 8);
     if (vec == 4 && !kWide) vec = 2;
     if (preagg) {
-        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, t0, d, ld, sel, out, sm_count, stream);
-        if (vec == 2) return run<K3_P, true, 2>(g, n, t0, d, ld, sel, out, sm_count, stream);
-        return run<K3_P, true, 1>(g, n, t0, d, ld, sel, out, sm_count, stream);
+        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
+        if (vec == 2) return run<K3_P, true, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
+        return run<K3_P, true, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
     }
-    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, t0, d, ld, sel, out, sm_count, stream);
-    if (vec == 2) return run<K3_P, false, 2>(g, n, t0, d, ld, sel, out, sm_count, stream);
-    return run<K3_P, false, 1>(g, n, t0, d, ld, sel, out, sm_count, stream);
+    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
+    if (vec == 2) return run<K3_P, false, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
+    return run<K3_P, false, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
 }
 
 // CTAs per SM the staged kernel would get for n gradients and theta slots (0: it cannot run).

@@ -37,19 +37,22 @@ def test_every_declared_symbol_is_exported(pkg):
 def test_struct_mirrors_match_the_header(pkg, tmp_path):
     src = tmp_path / "sz.cpp"
     src.write_text('#include "gar.h"\n#include <cstdio>\n#include <cstddef>\n'
-                   'int main(){printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(gar_selection_t),'
+                   'int main(){printf("%zu %zu %zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(gar_selection_t),'
                    'offsetof(gar_selection_t,sets), offsetof(gar_selection_t,nu),'
-                   'offsetof(gar_selection_t,add_pos), offsetof(gar_selection_t,scores), sizeof(gar_params_t));}')
+                   'offsetof(gar_selection_t,add_pos), offsetof(gar_selection_t,scores), sizeof(gar_params_t),'
+                   'offsetof(gar_selection_t,even_median), offsetof(gar_selection_t,winners),'
+                   'offsetof(gar_params_t,even_median), offsetof(gar_params_t,distance_mode));}')
     exe = tmp_path / "sz"
     subprocess.check_call(["g++", "-I" + os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(v) for v in subprocess.check_output([str(exe)]).split()]
     S = pkg.GarSelection
+    P = pkg.GarParams
     assert got == [C.sizeof(S), S.sets.offset, S.nu.offset, S.add_pos.offset, S.scores.offset,
-                   C.sizeof(pkg.GarParams)]
+                   C.sizeof(P), S.even_median.offset, S.winners.offset, P.even_median.offset, P.distance_mode.offset]
 
 
 def test_version_and_strings(pkg):
-    assert pkg.gar_version() == 100
+    assert pkg.gar_version() == 101
     assert pkg.gar_status_string(0) == "ok"
     assert "4f+3" in pkg.gar_status_string(2)
 
@@ -97,6 +100,15 @@ def test_errors_before_any_launch(pkg):
     assert L.gar_aggregate_ex(C.byref(p)) == 1
     p.theta = 4                                                            # theta < 2f+1
     assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.theta, p.even_median = 0, 2                                          # unknown even-median mode
+    assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.even_median, p.distance_mode = 0, 7                                  # unknown distance mode
+    assert L.gar_aggregate_ex(C.byref(p)) == 1
+    assert L.gar_pairwise_distances_mode(fake, 11, 100, 100, fake, None, 0, 5, None) == 1
+    assert L.gar_select(5, fake, 11, 2, 0, 0, 0, 3, fake, None) == 1       # unknown even-median mode
+    assert L.gar_selftest_bounded_wait(0, fake, None) == 1
+    assert L.gar_selftest_bounded_wait(100, None, None) == 1
+    assert L.gar_selftest_bounded_wait(1 << 20, fake, None) == 1           # limit above the documented maximum
 
 
 def test_missing_library_fails_loudly(pkg, monkeypatch):
