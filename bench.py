@@ -1,12 +1,17 @@
 #!/usr/bin/env python
 """Benchmark of the multi-Bulyan aggregation path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--d D] [--quick] [--impl reference]
 
 A step is one whole aggregation GAR(f, [G_1..G_n]) (distances -> selection ->
 coordinate phase) of one synthetic workload resident in HBM.  One JSON line is
-printed by rank 0.  With N > 1 (torchrun) every rank aggregates its own replica
-of the workload on its own GPU: the path has no inter-GPU step.
+printed by rank 0: the headline on the chosen workload (default: the largest,
+n = 15, d = 1e9), `per_config` with the same measurement on the three workloads
+of the d >= 1e7 regime, the CPU oracle timed on a sample, and the end-to-end
+figure through the host entry point.  `--quick --d D` runs a workload's recipe at
+another dimension and prints the device-side numbers only (the command line the
+profiler captures under profiles/ are taken on).  With N > 1 (torchrun) every
+rank aggregates its own replica of the workload on its own GPU.
 """
 from __future__ import annotations
 
@@ -45,7 +50,7 @@ def measured_hbm_peak():
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU while the timed region runs."""
 
-    def __init__(self, index: int, period: float = 0.02):
+    def __init__(self, index: int, period: float = 0.002):
         self.index, self.period = index, period
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -102,23 +107,29 @@ def physical_gpu_index(local: int) -> int:
     return local
 
 
+# columns of the CPU-baseline sample per workload: about 10 to 30 s of the numpy oracle on one core
+CPU_SAMPLE = {1: 100_000, 2: 1 << 20, 3: 1 << 22, 4: 1 << 21, 5: 1 << 25}
+REF_SAMPLE = {1: 100_000, 2: 1 << 18, 3: 1 << 18, 4: 1 << 17, 5: 1 << 21}
+
+
 def oracle_sample_time(cfg: int, d_sample: int):
     """Times the CPU oracle, as it stands, on a d_sample-column sample of the workload."""
     import numpy as np
     from oracle import gar_oracle as O
     from paper_1905_04374_b200 import workloads
     wl = workloads.WORKLOADS[cfg]
+    d_sample = min(d_sample, wl.d)
     G, _ = workloads.make_gradients(cfg, d=d_sample, device="cpu")
     Gh = G.numpy()
     t0 = time.perf_counter()
     out, _, _ = O.multi_bulyan(Gh, wl.f)
     dt = time.perf_counter() - t0
     assert np.all(np.isfinite(out))
-    return dt, wl
+    return dt, wl, d_sample
 
 
 def cpu_baseline(cfg: int, d_sample: int):
-    dt, wl = oracle_sample_time(cfg, d_sample)
+    dt, wl, d_sample = oracle_sample_time(cfg, d_sample)
     per_full = dt * (wl.d / d_sample)
     return {"value": 1.0 / per_full, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"numpy fp64 oracle on the first {d_sample} of {wl.d} coordinates of {wl.name} "
@@ -131,10 +142,10 @@ def run_reference(args):
         return
     from paper_1905_04374_b200 import workloads
     wl = workloads.WORKLOADS[args.config]
-    d_sample = args.ref_sample
+    d_sample = min(args.ref_sample or REF_SAMPLE[args.config], wl.d)
     times = []
     for i in range(args.warmup + args.steps):
-        dt, _ = oracle_sample_time(args.config, d_sample)
+        dt, _, _ = oracle_sample_time(args.config, d_sample)
         if i >= args.warmup:
             times.append(dt)
     per_step_full = (sum(times) / len(times)) * (wl.d / d_sample)
@@ -176,6 +187,138 @@ def max_over_ranks(elapsed_ms: float, world: int, device=None) -> float:
     return float(t.item())
 
 
+def launches_per_aggregation(n: int, d: int, theta: int) -> int:
+    """Kernels of this library one multi-Bulyan call launches on 16-byte aligned rows: the distance
+    kernel (for n > 16 and d >= 32768 the tensor-core kernel plus the gated difference-form kernel
+    behind it), the selection kernel, the staged coordinate kernel (from 400000 coordinates on) and
+    the register kernel for what is left after the last whole tile."""
+    k1 = 2 if (n > 16 and d >= 32768) else 1
+    if d >= 400_000:
+        tile = 512 if theta <= 12 else 256
+        k3 = 1 + (1 if d % tile else 0)
+    else:
+        k3 = 1
+    return k1 + 1 + k3
+
+
+def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant=True):
+    """Device-side measurement of one workload resident in HBM: `steps` whole aggregations timed
+    with CUDA events on the launch stream (max over ranks), then each stage alone."""
+    import torch
+    import torch.distributed as dist
+    wl = pkg.workloads.WORKLOADS[cfg]
+    n, f = wl.n, wl.f
+    d = d or wl.d
+    theta_a = pkg.gar_theta("multi_bulyan", n, f)
+    theta_b = pkg.gar_theta("bulyan", n, f)
+    G, _ = pkg.workloads.make_gradients(cfg, d=d, device=dev)
+    out = torch.empty(d, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        pkg.gar_aggregate("multi_bulyan", G, f, out=out)
+
+    for _ in range(max(warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(physical_gpu_index(local), period=0.002) as clocks:
+        torch.cuda.synchronize()
+        start.record(stream)
+        for _ in range(steps):
+            step()
+        stop.record(stream)
+        torch.cuda.synchronize()
+    elapsed_ms = max_over_ranks(start.elapsed_time(stop), world, dev)
+    if world > 1:
+        dist.barrier()
+    ms_per_step = elapsed_ms / steps
+
+    # ---- per-kernel durations, measured live with CUDA events on the launch stream
+    reps = max(5, min(50, steps))
+    ws = torch.zeros(pkg.gar_workspace_bytes("multi_bulyan", n, f, d), dtype=torch.uint8, device=dev)
+    dmat = torch.empty(n, n, dtype=torch.float64, device=dev)
+    sel = pkg.new_selection(dev)
+    pkg.gar_pairwise_distances(G, dist=dmat, workspace=ws)
+    pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel)
+    k1_ms = event_time_ms(lambda: pkg.gar_pairwise_distances(G, dist=dmat, workspace=ws), reps, stream)
+    k2_ms = event_time_ms(lambda: pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel), reps, stream)
+    k3_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, sel, theta_a, 1, out=out), reps, stream)
+    selh = pkg.read_selection(sel)
+    rows_k3 = int(selh.nu)
+    peak, peak_kind = measured_hbm_peak()
+    k1_bytes = 4.0 * n * d
+    k3_bytes = 4.0 * d * ((rows_k3 if rows_k3 else theta_a) + 1)
+    kernels = {
+        "k1_distances": {"ms": k1_ms, "algorithmic_bytes": k1_bytes, "gbs": k1_bytes / (k1_ms * 1e-3) / 1e9,
+                         "frac_of_measured_peak": k1_bytes / (k1_ms * 1e-3) / 1e9 / peak,
+                         "path": pkg.distance_path(ws)},
+        "k2_select": {"ms": k2_ms},
+        "k3_coordinate": {"ms": k3_ms, "algorithmic_bytes": k3_bytes, "gbs": k3_bytes / (k3_ms * 1e-3) / 1e9,
+                          "frac_of_measured_peak": k3_bytes / (k3_ms * 1e-3) / 1e9 / peak, "rows_read": rows_k3},
+    }
+    dom = "k1_distances" if k1_ms >= k3_ms else "k3_coordinate"
+    achieved = kernels[dom]["gbs"]
+    per_coord = NCU_DRAM_BYTES_PER_COORD.get((dom, n))
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_kind": peak_kind,
+                "traffic": per_coord * d if per_coord else None,
+                "algorithmic_bytes": kernels[dom]["algorithmic_bytes"]}
+    # whole-path effective bandwidth against the minimum traffic (n + theta + 1) * 4 d with
+    # theta = n - 2f, and against this rule's own minimum (n + |U| + 1) * 4 d
+    bytes_formula = 4.0 * d * (n + theta_b + 1)
+    bytes_own = 4.0 * d * (n + (rows_k3 if rows_k3 else theta_a) + 1)
+    path = {
+        "bytes_min_n_plus_theta_plus_1": bytes_formula,
+        "bytes_min_this_rule": bytes_own,
+        "effective_gbs": bytes_formula / (ms_per_step * 1e-3) / 1e9,
+        "effective_gbs_this_rule": bytes_own / (ms_per_step * 1e-3) / 1e9,
+    }
+    path["frac_of_nominal_8TBs"] = path["effective_gbs"] / NOMINAL_HBM_GBS
+    path["frac_of_measured_peak"] = path["effective_gbs"] / peak
+    path["frac_of_measured_peak_this_rule"] = path["effective_gbs_this_rule"] / peak
+    res = {"workload": wl.name if d == wl.d else f"{wl.name} recipe at d={d}", "n": n, "f": f, "d": d,
+           "theta": theta_a, "ms_per_aggregation": ms_per_step, "aggregations_per_sec": 1e3 / ms_per_step,
+           "steps": steps, "kernels": kernels, "roofline": roofline, "path": path, "clocks": clocks.summary(),
+           "elapsed_ms": elapsed_ms}
+    if variant:
+        # the same workload under the rule whose three-part summary speaks of theta = n - 2f iterated
+        # Krum winners and beta = theta - 2f, no pre-aggregation: GAR_BULYAN
+        k3b_sel = pkg.new_selection(dev)
+        pkg.gar_select("bulyan", dmat, n, f, sel=k3b_sel)
+        k3b_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, k3b_sel, theta_b, 0, out=out), reps, stream)
+        bulyan_ms = event_time_ms(lambda: pkg.gar_aggregate("bulyan", G, f, out=out), reps, stream)
+        res["variant_bulyan"] = {
+            "rule": "bulyan", "theta": theta_b, "beta": pkg.gar_beta("bulyan", n, f), "ms_per_aggregation": bulyan_ms,
+            "aggregations_per_sec": 1e3 / bulyan_ms, "k3_coordinate_ms": k3b_ms,
+            "effective_gbs": bytes_formula / (bulyan_ms * 1e-3) / 1e9,
+            "frac_of_measured_peak": bytes_formula / (bulyan_ms * 1e-3) / 1e9 / peak,
+            "frac_of_nominal_8TBs": bytes_formula / (bulyan_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS}
+    return res, G
+
+
+def run_e2e(pkg, cfg, G, steps):
+    """The same aggregation through the host entry point: pinned host buffers, both copies inside
+    the timed region."""
+    import torch
+    n, d = G.shape
+    f = pkg.workloads.WORKLOADS[cfg].f
+    host = torch.empty(n, d, dtype=torch.float32, pin_memory=True)
+    host.copy_(G)
+    hout = torch.empty(d, dtype=torch.float32, pin_memory=True)
+    pkg.gar_aggregate_host("multi_bulyan", host, f, out=hout)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        pkg.gar_aggregate_host("multi_bulyan", host, f, out=hout)
+    t1 = time.perf_counter()
+    return {"value": steps / (t1 - t0), "unit": UNIT, "h2d_bytes_per_step": int(4 * n * d),
+            "d2h_bytes_per_step": int(4 * d) + 4, "steps": steps,
+            "api": "gar_aggregate_host (pinned host buffers, synchronous)"}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -189,127 +332,56 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = pkg.workloads.WORKLOADS[args.config]
-    n, f, d = wl.n, wl.f, wl.d
-    theta_a = pkg.gar_theta("multi_bulyan", n, f)
-    theta_b = pkg.gar_theta("bulyan", n, f)
-    G, _ = pkg.workloads.make_gradients(args.config, device=dev)
-    out = torch.empty(d, dtype=torch.float32, device=dev)
-    stream = torch.cuda.current_stream()
-
-    def step():
-        pkg.gar_aggregate("multi_bulyan", G, f, out=out)
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with ClockSampler(physical_gpu_index(local)) as clocks:
-        torch.cuda.synchronize()
-        start.record(stream)
-        for _ in range(args.steps):
-            step()
-        stop.record(stream)
-        torch.cuda.synchronize()
-    elapsed_ms = start.elapsed_time(stop)
-    elapsed_ms = max_over_ranks(elapsed_ms, world, dev)
-    if world > 1:
-        dist.barrier()
-    ms_per_step = elapsed_ms / args.steps
-    value = world * args.steps / (elapsed_ms * 1e-3)
-
+    cfg = args.config
+    main, G = measure_workload(pkg, cfg, dev, args.steps, args.warmup, world, local, d=args.d)
+    wl = pkg.workloads.WORKLOADS[cfg]
+    n, f, d = main["n"], main["f"], main["d"]
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
+    value = world * args.steps / (main["elapsed_ms"] * 1e-3)
 
-    # ---- per-kernel durations, measured live with CUDA events on the launch stream
-    reps = max(5, min(50, args.steps))
-    dmat = torch.empty(n, n, dtype=torch.float64, device=dev)
-    sel = pkg.new_selection(dev)
-    pkg.gar_pairwise_distances(G, dist=dmat)
-    pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel)
-    k1_ms = event_time_ms(lambda: pkg.gar_pairwise_distances(G, dist=dmat), reps, stream)
-    k2_ms = event_time_ms(lambda: pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel), reps, stream)
-    k3_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, sel, theta_a, 1, out=out), reps, stream)
-    selh = pkg.read_selection(sel)
-    rows_k3 = int(selh.nu)
-    peak, peak_kind = measured_hbm_peak()
-    k1_bytes = 4.0 * n * d
-    k3_bytes = 4.0 * d * ((rows_k3 if rows_k3 else theta_a) + 1)
-    kernels = {
-        "k1_distances": {"ms": k1_ms, "algorithmic_bytes": k1_bytes, "gbs": k1_bytes / (k1_ms * 1e-3) / 1e9},
-        "k2_select": {"ms": k2_ms},
-        "k3_coordinate": {"ms": k3_ms, "algorithmic_bytes": k3_bytes, "gbs": k3_bytes / (k3_ms * 1e-3) / 1e9,
-                          "rows_read": rows_k3},
-    }
-    dom = "k1_distances" if k1_ms >= k3_ms else "k3_coordinate"
-    achieved = kernels[dom]["gbs"]
-    # DRAM bytes per coordinate from the committed ncu captures (profiles/), taken on a smaller d of
-    # the same kernel and scaled by d; None where no capture of the current kernel exists
-    ncu_bytes_per_coord = NCU_DRAM_BYTES_PER_COORD
-    per_coord = ncu_bytes_per_coord.get((dom, n))
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": peak_kind,
-                "traffic": per_coord * d if per_coord else None,
-                "algorithmic_bytes": kernels[dom]["algorithmic_bytes"]}
-    # whole-path effective bandwidth against the minimum traffic (n + theta + 1) * 4 d
-    path_bytes_northstar = 4.0 * d * (n + theta_b + 1)
-    path_bytes_own = 4.0 * d * (n + (rows_k3 if rows_k3 else theta_a) + 1)
-    path = {
-        "bytes_min_n_plus_theta_plus_1": path_bytes_northstar,
-        "bytes_min_this_rule": path_bytes_own,
-        "effective_gbs": path_bytes_northstar / (ms_per_step * 1e-3) / 1e9,
-        "effective_gbs_this_rule": path_bytes_own / (ms_per_step * 1e-3) / 1e9,
-    }
-    path["frac_of_nominal_8TBs"] = path["effective_gbs"] / NOMINAL_HBM_GBS
-    path["frac_of_measured_peak"] = path["effective_gbs"] / peak
-
-    # ---- the same workload under the rule the benchmark spec's summary describes (theta = n - 2f
-    # iterated Krum winners, beta = theta - 2f, no pre-aggregation): GAR_BULYAN
-    k3b_sel = pkg.new_selection(dev)
-    pkg.gar_select("bulyan", dmat, n, f, sel=k3b_sel)
-    k3b_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, k3b_sel, theta_b, 0, out=out), reps, stream)
-    bulyan_ms = event_time_ms(lambda: pkg.gar_aggregate("bulyan", G, f, out=out), reps, stream)
-    variant = {"rule": "bulyan", "theta": theta_b, "beta": pkg.gar_beta("bulyan", n, f), "ms_per_aggregation": bulyan_ms,
-               "aggregations_per_sec": 1e3 / bulyan_ms, "k3_coordinate_ms": k3b_ms,
-               "effective_gbs": path_bytes_northstar / (bulyan_ms * 1e-3) / 1e9,
-               "frac_of_measured_peak": path_bytes_northstar / (bulyan_ms * 1e-3) / 1e9 / peak,
-               "frac_of_nominal_8TBs": path_bytes_northstar / (bulyan_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS}
-
-    # ---- end to end through the host entry point (pinned host buffers, copies timed)
     e2e = None
     if not args.no_e2e:
-        host = torch.empty(n, d, dtype=torch.float32, pin_memory=True)
-        host.copy_(G)
-        hout = torch.empty(d, dtype=torch.float32, pin_memory=True)
-        e2e_steps = max(2, min(args.steps, args.e2e_steps))
-        pkg.gar_aggregate_host("multi_bulyan", host, f, out=hout)
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(e2e_steps):
-            pkg.gar_aggregate_host("multi_bulyan", host, f, out=hout)
-        t1 = time.perf_counter()
-        e2e = {"value": e2e_steps / (t1 - t0), "unit": UNIT, "h2d_bytes_per_step": int(4 * n * d),
-               "d2h_bytes_per_step": int(4 * d), "steps": e2e_steps,
-               "api": "gar_aggregate_host (pinned host buffers, synchronous)"}
-        del host, hout
+        try:
+            e2e = run_e2e(pkg, cfg, G, max(2, min(args.steps, args.e2e_steps)))
+        except Exception as exc:                      # e.g. the host cannot pin a 60 GB buffer
+            e2e = {"value": None, "unit": UNIT, "error": f"{type(exc).__name__}: {exc}"[:200]}
+        pkg.gar_shutdown()                            # give the host path's staging copy back
+    del G
+    torch.cuda.empty_cache()
 
-    cpu = None if args.no_cpu_baseline else cpu_baseline(args.config, args.cpu_sample)
+    # the other single-GPU workloads of the d >= 1e7 regime, same measurement, same run
+    per_config = []
+    if not args.no_per_config and args.d is None:
+        for other in (3, 4, 5):
+            if other == cfg:
+                entry = {k: main[k] for k in main if k != "elapsed_ms"}
+            else:
+                owl = pkg.workloads.WORKLOADS[other]
+                approx_ms = {3: 1.6, 4: 10.0, 5: 19.0}[other]
+                osteps = max(20, int(1000.0 / approx_ms))          # about a second of timed work
+                entry, Go = measure_workload(pkg, other, dev, osteps, 3, 1, local)
+                del Go
+                torch.cuda.empty_cache()
+                entry.pop("elapsed_ms")
+            per_config.append(entry)
+
+    cpu = None if args.no_cpu_baseline else cpu_baseline(cfg, args.cpu_sample or CPU_SAMPLE[cfg])
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": wl.name, "n": n, "f": f, "d": d, "rule": "multi_bulyan", "theta": theta_a,
+        "warmup": max(args.warmup, 3), "ms_per_step": main["ms_per_aggregation"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": main["workload"], "n": n, "f": f, "d": d, "rule": "multi_bulyan", "theta": main["theta"],
                    "beta": pkg.gar_beta("multi_bulyan", n, f), "parallelism": f"replicas x{world}",
+                   "why_this_workload": "the largest of the five configurations; it fits one GPU (60 GB of 180)",
                    "l2": "input (%.2f GB) larger than L2; no flush" % (4e-9 * n * d) if 4 * n * d > 2.6e8
                    else "input fits L2; not flushed between steps"},
-        "roofline": roofline, "path": path, "kernels": kernels, "variant_bulyan": variant, "cpu_baseline": cpu, "e2e": e2e,
-        # distances, selection, coordinate phase (+ one more coordinate kernel for a ragged tail)
-        "gpu_launches": (3 + (1 if d % 256 else 0)) * args.steps, "clocks": clocks.summary(),
+        "roofline": main["roofline"], "path": main["path"], "kernels": main["kernels"],
+        "variant_bulyan": main.get("variant_bulyan"), "per_config": per_config, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": launches_per_aggregation(n, d, main["theta"]) * args.steps, "clocks": main["clocks"],
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -319,16 +391,22 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=3, help="workload 1..5 (default 3: n=39, f=9, d=25.6M)")
+    ap.add_argument("--config", type=int, default=5,
+                    help="workload 1..5 (default 5: n=15, f=3, d=1e9, the largest single-GPU configuration)")
+    ap.add_argument("--d", type=int, default=None, help="another dimension for the workload's recipe (profiling)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--cpu-sample", type=int, default=1 << 22, help="columns of the CPU-baseline sample")
-    ap.add_argument("--ref-sample", type=int, default=1 << 18, help="columns per step of --impl reference")
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-sample", type=int, default=0, help="columns of the CPU-baseline sample (0: per workload)")
+    ap.add_argument("--ref-sample", type=int, default=0, help="columns per step of --impl reference (0: per workload)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--quick", action="store_true", help="device-side numbers of the chosen workload only")
     args = ap.parse_args()
+    if args.quick:
+        args.no_e2e = args.no_cpu_baseline = args.no_per_config = True
     if args.impl == "reference":
         run_reference(args)
     else:
