@@ -37,13 +37,26 @@ namespace {
 
 constexpr int KU_SLAB = 128;                 // columns per slab (one float4 per lane and row)
 constexpr int KU_JR = 3;                     // rows per producer warp
-constexpr int KU_NBUF = 3;                   // byte-tile buffers
-constexpr int KU_LBO = 192 * 16 + 16;        // bytes between 16-byte column chunks (192 rows + padding: conflict-free stores)
+constexpr int KU_MAX_NBUF = 6;               // byte-tile buffers at most
 constexpr int KU_SBO = 128;                  // bytes between groups of eight rows
-constexpr int KU_BUF_BYTES = 8 * KU_LBO;     // one slab: 8 chunks of 16 columns
+constexpr int KU_PACK_ROWS = 40;             // packed layout: rows per limb matrix
+// Two layouts of a byte tile.  Wide (any n <= 64): limb matrices 64 rows apart, [L1; L2; L3] in 192
+// rows, two instructions per k-step (see the file comment).  Packed (n <= 40): limb matrices 40
+// rows apart, [L1; L2; L3; 8 zero rows] in 128 rows, which is both operands of ONE 128 x 128
+// instruction per k-step that forms all nine limb products at once: half the operand bytes read
+// by the tensor core, under half its multiply-accumulates, smaller tiles (more of them in flight).
+template <bool PACKED> struct KUShape {
+    static constexpr int LIMB_ROWS = PACKED ? KU_PACK_ROWS : 64;          // tile rows between limb matrices
+    static constexpr int TILE_ROWS = PACKED ? 128 : 192;
+    static constexpr int LBO = TILE_ROWS * 16 + 16;     // bytes between 16-byte column chunks (+ padding: conflict-free stores)
+    static constexpr int BUF_BYTES = 8 * LBO;           // one slab: 8 chunks of 16 columns
+    static constexpr int SET_COLS = PACKED ? 128 : 256; // tensor-memory columns per accumulator set
+    static constexpr int NBUF = PACKED ? 5 : 3;         // byte-tile buffers
+    // fp64 sums of the CTA: packed, one 40 x 40 array per limb of the row operand; wide, px and pz (64 x 64)
+    static constexpr int SUM_DOUBLES = PACKED ? 3 * KU_PACK_ROWS * KU_PACK_ROWS : 2 * 4096;
+};
 constexpr int KU_PERIOD = 256;               // slabs per accumulator set at most: |sum| <= 256 * 128 * 2^14 = 2^29
 constexpr int KU_MIN_EXP = 21;               // smallest row exponent (keeps the scale a normal float)
-constexpr int KU_SET_COLS = 256;             // tensor-memory columns per accumulator set (192 + 64)
 constexpr int KU_FLUSH_WARPS = 4;            // warps 0..3: tensor-memory lanes 32 w .. 32 w + 31
 constexpr int KU_MMA_WARP = 4;
 constexpr int KU_FIRST_PRODUCER = 5;
@@ -52,16 +65,16 @@ constexpr int KU_TRI = 2080;
 constexpr double kGramRelBound = 1e-6;      // largest accepted bound on a distance's relative rounding error
 
 struct KUSmem {
-    unsigned long long full[KU_NBUF];        // producers -> MMA warp: the buffer's tiles are written
-    unsigned long long empty[KU_NBUF];       // tcgen05.commit -> producers: the MMAs that read the buffer are done
+    unsigned long long full[KU_MAX_NBUF];        // producers -> MMA warp: the buffer's tiles are written
+    unsigned long long empty[KU_MAX_NBUF];       // tcgen05.commit -> producers: the MMAs that read the buffer are done
     unsigned long long accfull[2];           // tcgen05.commit -> flush warps: the set is closed and complete
     unsigned long long accfree[2];           // flush warps -> MMA warp: the set has been read
-    unsigned long long desc[KU_NBUF][8];     // operand descriptors of a buffer's MMAs: k-step ks at [ks] (rows 0..) and [4 + ks] (rows 128..)
+    unsigned long long desc[KU_MAX_NBUF][8];     // operand descriptors of a buffer's MMAs: k-step ks at [ks] (rows 0..) and [4 + ks] (rows 128..)
     unsigned tmem_base;
     int      error;
-    int      grow[KU_NBUF];                  // some row of the buffer uses a larger exponent than before
+    int      grow[KU_MAX_NBUF];                  // some row of the buffer uses a larger exponent than before
     int      set_last[2];                    // the set is the CTA's last one
-    int      slab_exp[KU_NBUF][64];          // exponent each row of the buffer was quantised with
+    int      slab_exp[KU_MAX_NBUF][64];          // exponent each row of the buffer was quantised with
     int      set_exp[2][64];                 // exponents of the rows while the set was accumulated
     unsigned nonfinite_lo, nonfinite_hi;
     int      is_last;
@@ -85,9 +98,9 @@ __device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned ncols) {  
 
 // Shared-memory operand descriptor: K-major, no swizzle.  Bits [0,14) address / 16, [16,30) chunk
 // stride / 16, [32,46) eight-row-group stride / 16, [46,48) = 1 (descriptor version), layout type 0.
-__device__ __forceinline__ unsigned long long umma_desc(unsigned saddr) {
+__device__ __forceinline__ unsigned long long umma_desc(unsigned saddr, int lbo) {
     return static_cast<unsigned long long>((saddr >> 4) & 0x3fffu) |
-           (static_cast<unsigned long long>(KU_LBO >> 4) << 16) |
+           (static_cast<unsigned long long>(lbo >> 4) << 16) |
            (static_cast<unsigned long long>(KU_SBO >> 4) << 32) | (1ull << 46);
 }
 // Instruction descriptor, kind::i8: int32 accumulators (2 at bit 4), signed 8-bit A and B (1 at bits
@@ -139,7 +152,7 @@ __device__ __forceinline__ int tri_slot(int i, int j) { return i * 64 - (i * (i 
 // Shared memory: KUSmem, the byte-tile buffers, px and pz (2 x 64 x 64 doubles, stored transposed:
 // [j][i]), the raw ring float4 [NST][3 * producer warps][32].
 // FULL: n is a multiple of KU_JR, every producer warp owns KU_JR real rows (no per-row tests).
-template <int NST, int MAXT, bool FULL>
+template <int NST, int MAXT, bool FULL, bool PACKED>
 __global__ void __launch_bounds__(MAXT, 1)
 k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
         double* __restrict__ partials, unsigned int* __restrict__ ticket,
@@ -148,17 +161,19 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     extern __shared__ __align__(128) unsigned char smem_raw[];
     KUSmem& sm = *reinterpret_cast<KUSmem*>(smem_raw);
     constexpr int HEAD = (int(sizeof(KUSmem)) + 127) & ~127;
+    using S = KUShape<PACKED>;
+    constexpr int KU_NBUF = S::NBUF, KU_LBO = S::LBO, KU_BUF_BYTES = S::BUF_BYTES, KU_SET_COLS = S::SET_COLS;
     unsigned char* limb = smem_raw + HEAD;                                     // [KU_NBUF][KU_BUF_BYTES]
-    double* px_t = reinterpret_cast<double*>(limb + KU_NBUF * KU_BUF_BYTES);    // [64][64]: px_t[j * 64 + i] = px_ij
-    double* pz_t = px_t + 4096;
-    float4* ring = reinterpret_cast<float4*>(pz_t + 4096);                      // [NST][3 pw][32]
+    double* px_t = reinterpret_cast<double*>(limb + KU_NBUF * KU_BUF_BYTES);    // wide: [64][64], px_t[j * 64 + i] = px_ij
+    double* pz_t = px_t + 4096;                                                 // packed: [3][40][40] from px_t on
+    float4* ring = reinterpret_cast<float4*>(px_t + S::SUM_DOUBLES);            // [NST][3 pw][32]
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nthreads = blockDim.x;
     const int pw = (nthreads >> 5) - KU_FIRST_PRODUCER;                        // producer warps
     const int ring_rows = KU_JR * pw;
     volatile int* error = &sm.error;
 
-    for (int i = tid; i < (KU_NBUF * KU_BUF_BYTES + 2 * 4096 * 8) / 4; i += nthreads) reinterpret_cast<unsigned*>(limb)[i] = 0u;
+    for (int i = tid; i < (KU_NBUF * KU_BUF_BYTES + S::SUM_DOUBLES * 8) / 4; i += nthreads) reinterpret_cast<unsigned*>(limb)[i] = 0u;
     if (tid < 64) {
 #pragma unroll
         for (int b = 0; b < KU_NBUF; ++b) sm.slab_exp[b][tid] = KU_MIN_EXP;
@@ -186,7 +201,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     // critical path: everything it can look up instead of compute is tabulated here
     if (tid < KU_NBUF * 8) {
         const int b = tid >> 3, ks = tid & 3, second = (tid >> 2) & 1;
-        sm.desc[b][tid & 7] = umma_desc(smem_u32(limb) + unsigned(b) * KU_BUF_BYTES + unsigned(ks) * 2u * KU_LBO + (second ? 128u * 16u : 0u));
+        sm.desc[b][tid & 7] = umma_desc(smem_u32(limb) + unsigned(b) * KU_BUF_BYTES + unsigned(ks) * 2u * KU_LBO + (second ? 128u * 16u : 0u), KU_LBO);
     }
     if (warp == KU_MMA_WARP) tmem_alloc(&sm.tmem_base, 2 * KU_SET_COLS);
     fence_async_smem();                  // the zeroed tiles are read by the tensor core (async proxy)
@@ -314,8 +329,8 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
                     const unsigned h01 = prmt(w[jr][0], w[jr][1], 0x0062u), h23 = prmt(w[jr][2], w[jr][3], 0x0062u);
                     const unsigned at = limb_u32 + buf_off + tile_off[jr];
                     asm volatile("st.shared.b32 [%0], %1;" ::"r"(at), "r"(prmt(h01, h23, 0x5410u) ^ 0x80808080u) : "memory");             // l1
-                    asm volatile("st.shared.b32 [%0+1024], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x7632u) ^ 0x80808080u) : "memory");        // l2: rows 64..
-                    asm volatile("st.shared.b32 [%0+2048], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x5410u) ^ 0x80808080u) : "memory");        // l3: rows 128..
+                    asm volatile("st.shared.b32 [%0+%2], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x7632u) ^ 0x80808080u), "n"(S::LIMB_ROWS * 16) : "memory");   // l2
+                    asm volatile("st.shared.b32 [%0+%2], %1;" ::"r"(at), "r"(prmt(p01, p23, 0x5410u) ^ 0x80808080u), "n"(S::LIMB_ROWS * 32) : "memory");   // l3
                 }
             }
             if (exp_stores > 0) {                    // warp-uniform
@@ -341,7 +356,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         }
     } else if (warp == KU_MMA_WARP) {
         // ================================================================ MMA issue
-        constexpr unsigned IDESC_A = umma_idesc(128, 192), IDESC_B = umma_idesc(128, 64);
+        constexpr unsigned IDESC_A = umma_idesc(128, 192), IDESC_B = umma_idesc(128, 64), IDESC_P = umma_idesc(128, 128);
         const unsigned limb_addr = smem_u32(limb);
         int set = 0, since = 0;
         int opened0 = 0, opened1 = 0;
@@ -375,10 +390,14 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
                     const unsigned long long t1 = dt[ks];         // rows 0..: L1, L2, L3
-                    const unsigned long long t3 = dt[4 + ks];     // rows 128..: L3, then unread rows
                     const unsigned acc = (fresh && ks == 0) ? 0u : 1u;
-                    umma_i8(d1, t1, t1, IDESC_A, acc);          // [L1; L2] x [L1; L2; L3]^T
-                    umma_i8(d2, t3, t3, IDESC_B, acc);          // [L3; *] x L3^T
+                    if constexpr (PACKED) {
+                        umma_i8(d1, t1, t1, IDESC_P, acc);      // [L1; L2; L3; 0] x [L1; L2; L3; 0]^T
+                    } else {
+                        const unsigned long long t3 = dt[4 + ks]; // rows 128..: L3, then unread rows
+                        umma_i8(d1, t1, t1, IDESC_A, acc);      // [L1; L2] x [L1; L2; L3]^T
+                        umma_i8(d2, t3, t3, IDESC_B, acc);      // [L3; *] x L3^T
+                    }
                 }
                 umma_commit(&sm.empty[buf]);                    // arrives when these MMAs have read the buffer
             }
@@ -401,8 +420,10 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         // ================================================================ flush: tensor memory -> fp64
         const int q = warp;                                     // lanes 32 q .. 32 q + 31 of tensor memory
         const int L = q * 32 + lane;
-        const int i = L & 63;
-        const bool lower = L >= 64;                             // rows of L2 (L1 otherwise)
+        // wide: lanes 0..63 are the rows of L1, 64..127 those of L2; packed: 40 lanes per limb
+        const int limb_a = PACKED ? L / KU_PACK_ROWS : L >> 6;
+        const int i = PACKED ? L - limb_a * KU_PACK_ROWS : L & 63;
+        const bool lower = L >= 64;                             // wide: rows of L2 (L1 otherwise)
         for (int k = 0;; ++k) {
             const int set = k & 1;
             // a set closes rarely: poll slowly; then agree over the four warps (they meet at named barriers below)
@@ -413,46 +434,70 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             if (!all_ok) { if (lane == 0) sm.error = 1; break; }
             tc_fence_after();
             const int last = *reinterpret_cast<volatile int*>(&sm.set_last[set]);
-            const int ei = sm.set_exp[set][i] - 296;
+            const int ei = sm.set_exp[set][i & 63] - 296;
             const unsigned tbase = tmem_base + (unsigned(q * 32) << 16) + unsigned(set * KU_SET_COLS);
+            if constexpr (PACKED) {
+                // lane (a, i) holds row i of limb a against all three limbs of every row j: its share of
+                // P_ij is 2^(8(2-a)) (2^16 LaL1^T + 2^8 LaL2^T + LaL3^T)_ij, an integer below 2^47 (exact),
+                // times the rows' scales; it goes to the array of limb a, which no other lane writes
+                double* mine_p = px_t + limb_a * (KU_PACK_ROWS * KU_PACK_ROWS);
 #pragma unroll 1
-            for (int phase = 0; phase < 2; ++phase) {
-                if ((phase == 1) == lower) {                    // warp-uniform: L1 rows first, then L2 rows
-#pragma unroll 1
-                    for (int j0 = 0; j0 < n; j0 += 8) {
-                        int r0[8], r1[8], r2[8], r3[8];
-                        if (!lower) {
-                            tmem_ld8(tbase + unsigned(j0), r0);             // L1 L1^T
-                            tmem_ld8(tbase + unsigned(64 + j0), r1);        // L1 L2^T
-                            tmem_ld8(tbase + unsigned(128 + j0), r2);       // L1 L3^T
-                            tmem_ld8(tbase + unsigned(192 + j0), r3);       // L3 L3^T
-                        } else {
-                            tmem_ld8(tbase + unsigned(64 + j0), r0);        // L2 L2^T
-                            tmem_ld8(tbase + unsigned(128 + j0), r1);       // L2 L3^T
+                for (int j0 = 0; j0 < n; j0 += 8) {
+                    int r0[8], r1[8], r2[8];
+                    tmem_ld8(tbase + unsigned(j0), r0);
+                    tmem_ld8(tbase + unsigned(KU_PACK_ROWS + j0), r1);
+                    tmem_ld8(tbase + unsigned(2 * KU_PACK_ROWS + j0), r2);
+                    tmem_ld_wait();
 #pragma unroll
-                            for (int t = 0; t < 8; ++t) { r2[t] = 0; r3[t] = 0; }
-                        }
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int t = 0; t < 8; ++t) {
-                            const int j = j0 + t;
-                            const int e = ei + sm.set_exp[set][j & 63];       // s_i s_j = 2^e
-                            double x, y;                                      // exact: |sums| < 2^30
-                            if (!lower) {
-                                x = double(r0[t]) * pow2(e + 32) + double(r3[t]) * pow2(e);
-                                y = (double(r1[t]) * 256.0 + double(r2[t])) * pow2(e + 16);
-                            } else {
-                                x = double(r0[t]) * pow2(e + 16);
-                                y = double(r1[t]) * pow2(e + 8);
-                            }
-                            if (i < n && j < n) {
-                                px_t[j * 64 + i] += x;
-                                pz_t[j * 64 + i] += y;
-                            }
+                    for (int t = 0; t < 8; ++t) {
+                        const int j = j0 + t;
+                        if (limb_a < 3 && i < n && j < n) {
+                            const int e = ei + sm.set_exp[set][j] + 8 * (2 - limb_a);
+                            const double v = (double(r0[t]) * 65536.0 + double(r1[t]) * 256.0) + double(r2[t]);
+                            mine_p[j * KU_PACK_ROWS + i] += v * pow2(e);
                         }
                     }
                 }
-                asm volatile("bar.sync %0, %1;" ::"r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
+            } else {
+#pragma unroll 1
+                for (int phase = 0; phase < 2; ++phase) {
+                    if ((phase == 1) == lower) {                    // warp-uniform: L1 rows first, then L2 rows
+#pragma unroll 1
+                        for (int j0 = 0; j0 < n; j0 += 8) {
+                            int r0[8], r1[8], r2[8], r3[8];
+                            if (!lower) {
+                                tmem_ld8(tbase + unsigned(j0), r0);             // L1 L1^T
+                                tmem_ld8(tbase + unsigned(64 + j0), r1);        // L1 L2^T
+                                tmem_ld8(tbase + unsigned(128 + j0), r2);       // L1 L3^T
+                                tmem_ld8(tbase + unsigned(192 + j0), r3);       // L3 L3^T
+                            } else {
+                                tmem_ld8(tbase + unsigned(64 + j0), r0);        // L2 L2^T
+                                tmem_ld8(tbase + unsigned(128 + j0), r1);       // L2 L3^T
+#pragma unroll
+                                for (int t = 0; t < 8; ++t) { r2[t] = 0; r3[t] = 0; }
+                            }
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) {
+                                const int j = j0 + t;
+                                const int e = ei + sm.set_exp[set][j & 63];       // s_i s_j = 2^e
+                                double x, y;                                      // exact: |sums| < 2^30
+                                if (!lower) {
+                                    x = double(r0[t]) * pow2(e + 32) + double(r3[t]) * pow2(e);
+                                    y = (double(r1[t]) * 256.0 + double(r2[t])) * pow2(e + 16);
+                                } else {
+                                    x = double(r0[t]) * pow2(e + 16);
+                                    y = double(r1[t]) * pow2(e + 8);
+                                }
+                                if (i < n && j < n) {
+                                    px_t[j * 64 + i] += x;
+                                    pz_t[j * 64 + i] += y;
+                                }
+                            }
+                        }
+                    }
+                    asm volatile("bar.sync %0, %1;" ::"r"(KU_BAR_FLUSH), "r"(KU_FLUSH_WARPS * 32) : "memory");
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -473,7 +518,14 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         const int i = idx >> 6, j = idx & 63;
         if (i <= j) {
             double v = 0.0;
-            if (j < n) v = px_t[j * 64 + i] + (pz_t[j * 64 + i] + pz_t[i * 64 + j]);
+            if (j < n) {
+                if constexpr (PACKED) {
+                    constexpr int PP = KU_PACK_ROWS * KU_PACK_ROWS;
+                    v = (px_t[j * KU_PACK_ROWS + i] + px_t[PP + j * KU_PACK_ROWS + i]) + px_t[2 * PP + j * KU_PACK_ROWS + i];
+                } else {
+                    v = px_t[j * 64 + i] + (pz_t[j * 64 + i] + pz_t[i * 64 + j]);
+                }
+            }
             my_partial[tri_slot(i, j)] = v;
         }
     }
@@ -557,7 +609,7 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     }
 }
 
-template <int NST, int MAXT, bool FULL>
+template <int NST, int MAXT, bool FULL, bool PACKED>
 cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                       int pw, size_t smem, cudaStream_t stream) {
     static size_t configured[64] = {0};                        // dynamic shared memory the kernel is allowed, per device
@@ -565,7 +617,7 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64 || configured[dev] < smem) {
-        err = cudaFuncSetAttribute(k1_umma<NST, MAXT, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        err = cudaFuncSetAttribute(k1_umma<NST, MAXT, FULL, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = smem;
     }
@@ -575,7 +627,7 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     int64_t grid = sm_count;
     if (grid > kMaxCtasK1) grid = kMaxCtasK1;
     if (grid > nslabs) grid = nslabs;
-    k1_umma<NST, MAXT, FULL><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
+    k1_umma<NST, MAXT, FULL, PACKED><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
         g, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(), ws.k1_path(), ws.k1_gate());
     return cudaGetLastError();
 }
@@ -583,26 +635,38 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
 }  // namespace
 
 // 16 < n <= 64, grads 16-byte aligned, ld % 4 == 0.
-cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
-                                  int sm_count, cudaStream_t stream) {
+template <bool PACKED>
+static cudaError_t launch_umma_layout(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
+                                      int sm_count, cudaStream_t stream) {
+    using S = KUShape<PACKED>;
     const int pw = (n + KU_JR - 1) / KU_JR;                    // producer warps: three rows each
-    const size_t fixed = ((sizeof(KUSmem) + 127) & ~size_t(127)) + size_t(KU_NBUF) * KU_BUF_BYTES + 2 * 4096 * sizeof(double);
+    const size_t fixed = ((sizeof(KUSmem) + 127) & ~size_t(127)) + size_t(S::NBUF) * S::BUF_BYTES + size_t(S::SUM_DOUBLES) * sizeof(double);
     const size_t stage = size_t(KU_JR) * pw * 32 * sizeof(float4);
     constexpr size_t kSmemMax = 227 * 1024;                    // per-CTA limit of the SM
     constexpr int kSmall = 32 * (KU_FIRST_PRODUCER + 14), kLarge = 32 * (KU_FIRST_PRODUCER + 22);
     int nst = 4;
     while (nst > 2 && fixed + nst * stage > kSmemMax) --nst;   // deepest raw ring that fits
     const size_t smem = fixed + nst * stage;
-#define GAR_KU(NSTV, MAXTV)                                                                                 \
-    do {                                                                                                    \
-        if (n == KU_JR * pw) return launch_ku<NSTV, MAXTV, true>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream); \
-        return launch_ku<NSTV, MAXTV, false>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream);           \
+#define GAR_KU(NSTV, MAXTV)                                                                                           \
+    do {                                                                                                              \
+        if (n == KU_JR * pw) return launch_ku<NSTV, MAXTV, true, PACKED>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream); \
+        return launch_ku<NSTV, MAXTV, false, PACKED>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream);           \
     } while (0)
     if (pw <= 14) { if (nst == 4) GAR_KU(4, kSmall); if (nst == 3) GAR_KU(3, kSmall); GAR_KU(2, kSmall); }
-    if (nst == 4) GAR_KU(4, kLarge);
-    if (nst == 3) GAR_KU(3, kLarge);
-    GAR_KU(2, kLarge);
+    if constexpr (!PACKED) {
+        if (nst == 4) GAR_KU(4, kLarge);
+        if (nst == 3) GAR_KU(3, kLarge);
+        GAR_KU(2, kLarge);
+    }
 #undef GAR_KU
+    return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
+                                  int sm_count, cudaStream_t stream) {
+    static const char* env = std::getenv("GAR_KU_PACKED");      // experiment switch
+    if (n <= KU_PACK_ROWS && !(env && env[0] == '0')) return launch_umma_layout<true>(grads, n, d, ld, dist, ws, sm_count, stream);
+    return launch_umma_layout<false>(grads, n, d, ld, dist, ws, sm_count, stream);
 }
 
 }  // namespace gar
