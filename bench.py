@@ -10,8 +10,9 @@ n = 15, d = 1e9), `per_config` with the same measurement on the three workloads
 of the d >= 1e7 regime, the CPU oracle timed on a sample, and the end-to-end
 figure through the host entry point.  `--quick --d D` runs a workload's recipe at
 another dimension and prints the device-side numbers only (the command line the
-profiler captures under profiles/ are taken on).  With N > 1 (torchrun) every
-rank aggregates its own replica of the workload on its own GPU.
+profiler captures under profiles/ are taken on).  With N > 1 (torchrun) the workload's
+coordinates are sharded over the N GPUs and a step is one aggregation by all of them
+(paper_1905_04374_b200/sharded.py): strong scaling.
 """
 from __future__ import annotations
 
@@ -319,6 +320,93 @@ def run_e2e(pkg, cfg, G, steps):
             "api": "gar_aggregate_host (pinned host buffers, synchronous)"}
 
 
+def run_sharded(pkg, args, dev, world, rank, local):
+    """N > 1: ONE aggregation spread over the N GPUs.  The workload's coordinates are split into
+    contiguous column ranges, one per rank (whole generator chunks); a step is
+    paper_1905_04374_b200.sharded.sharded_aggregate: local distance partials, one all-gather of
+    n*n fp64 values per rank (NCCL), the sum in rank order, the replicated selection and the local
+    coordinate phase.  Total work is fixed as N grows: strong scaling."""
+    import torch
+    import torch.distributed as dist
+    from paper_1905_04374_b200 import sharded
+    cfg = args.config
+    wl = pkg.workloads.WORKLOADS[cfg]
+    n, f = wl.n, wl.f
+    d = args.d or wl.d
+    c0, c1 = pkg.workloads.shard_columns(d, world, rank)
+    if c1 > c0:
+        G, _ = pkg.workloads.make_gradients(cfg, d=d, device=dev, columns=(c0, c1))
+    else:
+        G = torch.empty(n, 0, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        return sharded.sharded_aggregate("multi_bulyan", G, f)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    dist.barrier()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(physical_gpu_index(local), period=0.002) as clocks:
+        torch.cuda.synchronize()
+        start.record(stream)
+        for _ in range(args.steps):
+            step()
+        stop.record(stream)
+        torch.cuda.synchronize()
+    elapsed_ms = max_over_ranks(start.elapsed_time(stop), world, dev)
+    dist.barrier()
+    # end to end: this rank's slice from pinned host memory, the sharded call, its slice of the result back
+    e2e_steps = max(2, min(args.steps, args.e2e_steps))
+    host = torch.empty(G.shape, dtype=torch.float32, pin_memory=True)
+    host.copy_(G)
+    hout = torch.empty(c1 - c0, dtype=torch.float32, pin_memory=True)
+    stage = torch.empty_like(G)
+
+    def e2e_step():
+        stage.copy_(host, non_blocking=True)
+        out, _, _ = sharded.sharded_aggregate("multi_bulyan", stage, f)
+        hout.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_step()
+    dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    dist.barrier()
+    e2e_s = time.perf_counter() - t0
+    e2e_ms = max_over_ranks(e2e_s * 1e3, world, dev)
+    if rank != 0:
+        return
+    ms_per_step = elapsed_ms / args.steps
+    theta_b = pkg.gar_theta("bulyan", n, f)
+    peak, peak_kind = measured_hbm_peak()
+    bytes_formula = 4.0 * d * (n + theta_b + 1)
+    line = {
+        "metric": METRIC, "value": args.steps / (elapsed_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name if d == wl.d else f"{wl.name} recipe at d={d}", "n": n, "f": f, "d": d,
+                   "rule": "multi_bulyan", "theta": pkg.gar_theta("multi_bulyan", n, f),
+                   "beta": pkg.gar_beta("multi_bulyan", n, f),
+                   "parallelism": f"coordinates sharded over {world} GPUs; one all-gather of n*n fp64 per aggregation",
+                   "l2": "every rank's slice is larger than L2; no flush"},
+        "roofline": None,
+        "path": {"bytes_min_n_plus_theta_plus_1": bytes_formula,
+                 "effective_gbs": bytes_formula / (ms_per_step * 1e-3) / 1e9,
+                 "frac_of_measured_peak_all_gpus": bytes_formula / (ms_per_step * 1e-3) / 1e9 / (peak * world)},
+        "cpu_baseline": None,
+        "e2e": {"value": e2e_steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(4 * n * d),
+                "d2h_bytes_per_step": int(4 * d), "steps": e2e_steps,
+                "api": "sharded_aggregate on slices copied from pinned host memory, result slices copied back"},
+        "gpu_launches": (launches_per_aggregation(n, max(c1 - c0, 1), pkg.gar_theta("multi_bulyan", n, f)) + 1) * args.steps,
+        "clocks": clocks.summary(),
+    }
+    print(json.dumps(line), flush=True)
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -329,10 +417,14 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    if world > 1 or args.force_sharded:
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = args.config
+    if world > 1 or args.force_sharded:
+        run_sharded(pkg, args, dev, world, rank, local)
+        dist.destroy_process_group()
+        return
     main, G = measure_workload(pkg, cfg, dev, args.steps, args.warmup, world, local, d=args.d)
     wl = pkg.workloads.WORKLOADS[cfg]
     n, f, d = main["n"], main["f"], main["d"]
@@ -404,6 +496,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--quick", action="store_true", help="device-side numbers of the chosen workload only")
+    ap.add_argument("--force-sharded", action="store_true",
+                    help="run the sharded (N > 1) code path even with one rank (under torchrun, for checking it)")
     args = ap.parse_args()
     if args.quick:
         args.no_e2e = args.no_cpu_baseline = args.no_per_config = True

@@ -243,6 +243,20 @@ int gar_pairwise_distances_mode(const float* grads, int n, int64_t d, int64_t ld
                                 void* workspace, size_t workspace_bytes, int distance_mode, void* stream);
 
 /*
+ * Sum of `count` distance matrices in the order given: dist = parts[0] + parts[1] + ... (fp64,
+ * element by element, left to right).  This is the one exchange step of an aggregation whose
+ * coordinates are sharded over several GPUs (the dimension d of the Introduction's footnote,
+ * 10^9 to 10^11, does not fit one device; Theorem 2 (ii): the work is O(d) and splits along d):
+ * every GPU computes gar_pairwise_distances on its own slice of the columns -- squared distances
+ * add over disjoint column sets -- the n*n partial matrices are all-gathered into every GPU's own
+ * memory, and each GPU adds them in rank order with this call, so that all of them hold the
+ * bit-identical matrix, select the same gradients (gar_select) and run gar_coordinate_phase on
+ * their own slice.  A NaN diagonal (a distance kernel that gave up) survives the sum.
+ *   parts dev [count][n*n] fp64, dist dev [n*n] (may be parts[0]); 1 <= count <= 1024.
+ */
+int gar_reduce_partials(const double* parts, int count, int n, double* dist, void* stream);
+
+/*
  * Step 1 alone, for callers that must not allocate: the same distance kernels, but
  * their scratch (ticket counter and per-CTA partial sums) is a fixed array inside the
  * library image instead of a workspace, so this call performs no cudaMalloc / cudaFree

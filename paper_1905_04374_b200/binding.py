@@ -91,6 +91,7 @@ def lib():
                                              C.c_size_t, C.c_void_p]
         L.gar_pairwise_distances_mode.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                                   C.c_size_t, C.c_int, C.c_void_p]
+        L.gar_reduce_partials.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
         L.gar_selftest_bounded_wait.argtypes = [C.c_uint, C.c_void_p, C.c_void_p]
         L.gar_pairwise_distances_static.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
         L.gar_select.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -232,6 +233,19 @@ def gar_pairwise_distances(grads: torch.Tensor, dist: torch.Tensor | None = None
             st = lib().gar_pairwise_distances_mode(grads.data_ptr(), n, d, ld, dist.data_ptr(), wp, wb,
                                                    _mode(distance_mode), _stream(stream))
     _check(st, "gar_pairwise_distances")
+    return dist
+
+
+def gar_reduce_partials(parts: torch.Tensor, dist: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """gar_reduce_partials: parts CUDA float64 [count, n, n] -> dist [n, n] = parts[0] + parts[1] + ... in order."""
+    if not (parts.is_cuda and parts.dtype == torch.float64 and parts.is_contiguous() and parts.dim() == 3):
+        raise TypeError("parts must be a contiguous CUDA float64 tensor [count, n, n]")
+    count, n, _ = parts.shape
+    if dist is None:
+        dist = torch.empty(n, n, dtype=torch.float64, device=parts.device)
+    with torch.cuda.device(parts.device):
+        st = lib().gar_reduce_partials(parts.data_ptr(), count, n, dist.data_ptr(), _stream(stream))
+    _check(st, "gar_reduce_partials")
     return dist
 
 

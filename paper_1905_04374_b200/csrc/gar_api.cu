@@ -144,6 +144,16 @@ __global__ void selftest_wait_kernel(unsigned limit, long long* result) {
     }
 }
 
+// dist = parts[0] + parts[1] + ... in that order (every GPU of a sharded aggregation runs this on
+// the same gathered data and gets the same bits).
+__global__ void reduce_partials_kernel(const double* __restrict__ parts, int count, int nn, double* __restrict__ dist) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= nn) return;
+    double s = parts[idx];
+    for (int r = 1; r < count; ++r) s += parts[size_t(r) * nn + idx];
+    dist[idx] = s;
+}
+
 }  // namespace
 
 namespace gar {
@@ -281,6 +291,14 @@ int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, gar_s
     cudaError_t err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg ? 1 : 0, out, st->sm_count,
                                              static_cast<cudaStream_t>(stream));
     return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+}
+
+int gar_reduce_partials(const double* parts, int count, int n, double* dist, void* stream) {
+    if (!parts || !dist || count < 1 || count > 1024 || n < 1) return GAR_ERR_INVALID_ARG;
+    if (n > GAR_MAX_N) return GAR_ERR_UNSUPPORTED;
+    const int nn = n * n;
+    reduce_partials_kernel<<<(nn + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(parts, count, nn, dist);
+    return cudaGetLastError() == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }
 
 int gar_selftest_bounded_wait(unsigned int limit, long long* result, void* stream) {

@@ -105,12 +105,15 @@ def _fill_chunk(G, c0, c1, wl: Workload, byz, seed, chunk_idx):
 
 def make_gradients(cfg: int, d: int | None = None, device="cpu", seed: int | None = None,
                    placement: str = "random", n: int | None = None, f: int | None = None,
-                   out: torch.Tensor | None = None):
+                   out: torch.Tensor | None = None, columns: tuple | None = None):
     """Draw workload `cfg` (1..5), optionally at another dimension d (and n, f).
 
     Returns (G, byz): G is an fp32 tensor [n, d] on `device`, byz the sorted
     list of Byzantine row indices.  `out`, if given, is filled instead of a
     new tensor (it must be [n, >= d] fp32; only the first d columns are set).
+    `columns` = (c0, c1), c0 a multiple of CHUNK, draws only that column range
+    of the d-dimensional workload (the slice one GPU of a sharded run owns): the
+    result is [n, c1 - c0] and equals G[:, c0:c1] of the full draw bit for bit.
     """
     wl = WORKLOADS[cfg]
     if d is not None or n is not None or f is not None:
@@ -119,10 +122,30 @@ def make_gradients(cfg: int, d: int | None = None, device="cpu", seed: int | Non
     if seed is None:
         seed = BASE_SEED + cfg
     byz = byzantine_rows(wl.n, wl.f, seed, placement)
-    G = out if out is not None else torch.empty(wl.n, wl.d, dtype=torch.float32, device=device)
-    for ci, c0 in enumerate(range(0, wl.d, CHUNK)):
-        _fill_chunk(G, c0, min(c0 + CHUNK, wl.d), wl, byz, seed, ci)
+    lo, hi = (0, wl.d) if columns is None else columns
+    if lo % CHUNK != 0 or not (0 <= lo < hi <= wl.d):
+        raise ValueError("columns must start on a multiple of CHUNK and lie inside [0, d]")
+    G = out if out is not None else torch.empty(wl.n, hi - lo, dtype=torch.float32, device=device)
+    for c0 in range(lo, hi, CHUNK):
+        c1 = min(c0 + CHUNK, wl.d, hi)
+        # a chunk is always drawn whole (its generator is consumed in a fixed order) ...
+        if c1 - c0 == min(CHUNK, wl.d - c0):
+            _fill_chunk(G, c0 - lo, c1 - lo, wl, byz, seed, c0 // CHUNK)
+        else:                                 # ... and cut afterwards when the range ends inside it
+            full = torch.empty(wl.n, min(CHUNK, wl.d - c0), dtype=torch.float32, device=G.device)
+            _fill_chunk(full, 0, full.shape[1], wl, byz, seed, c0 // CHUNK)
+            G[:, c0 - lo:c1 - lo] = full[:, :c1 - c0]
     return G, byz
+
+
+def shard_columns(d: int, world: int, rank: int):
+    """Column range [c0, c1) of rank `rank` when d columns are split over `world` GPUs in whole
+    chunks of CHUNK columns (the last rank takes the ragged end)."""
+    chunks = (d + CHUNK - 1) // CHUNK
+    per = (chunks + world - 1) // world
+    c0 = min(rank * per * CHUNK, d)
+    c1 = min((rank + 1) * per * CHUNK, d)
+    return c0, c1
 
 
 def make_uniform(n: int, d: int, device="cpu", seed: int = BASE_SEED):
