@@ -168,7 +168,7 @@ typedef struct {
     int64_t       d;
     int64_t       ld;             /* row stride in elements; 0 means d */
     const float*  grads;          /* dev, n rows */
-    float*        out;            /* dev, d values; must not overlap grads */
+    float*        out;            /* dev, d values; must not overlap grads (may be NULL with sgd_params) */
     void*         stream;         /* cudaStream_t */
     void*         workspace;      /* dev, 256-byte aligned, >= gar_workspace_bytes(), its first 256
                                      bytes zeroed once before the first use (the kernels restore
@@ -186,6 +186,16 @@ typedef struct {
     gar_selection_t* selection_out; /* optional dev: the selection result */
     int32_t       distance_mode;  /* gar_distance_mode_t */
     int32_t       reserved;
+    /* Optional SGD step fused into the coordinate kernel's store (Eq. 2: x <- x - lr * GAR(...);
+       Section 5.1 trains with momentum 0.9): with g the aggregated coordinate,
+           v <- sgd_momentum * v + g   (only if sgd_momentum_buf is given),   x <- x - sgd_lr * v   (or g)
+       so the aggregate never makes a round trip through memory.  sgd_params NULL: no step.
+       With a step, `out` may be NULL (the aggregate itself is then not stored).  If the call ends
+       with a status other than GAR_OK in the selection, x and v are left untouched. */
+    float*        sgd_params;       /* dev [d], x, updated in place */
+    float*        sgd_momentum_buf; /* dev [d], v, updated in place; NULL: plain SGD */
+    float         sgd_lr;
+    float         sgd_momentum;
 } gar_params_t;
 
 /* Library version (GAR_VERSION).  The paper has no counterpart. */

@@ -361,6 +361,23 @@ def bulyan(G, f: int, D=None, even: str = "lower"):
     return out, sel, gap
 
 
+# --------------------------------------------------------------------------
+# The update the aggregate feeds (Eq. 2: x_{k+1} = x_k - gamma_k * GAR(...);
+# Section 5.1 trains with a momentum of 0.9)
+# --------------------------------------------------------------------------
+def sgd_step(x, g, lr: float, momentum_buf=None, momentum: float = 0.0):
+    """One SGD step with the aggregated gradient g.  Without a momentum buffer:
+    x - lr * g (Eq. 2).  With one: v <- momentum * v + g, x <- x - lr * v (the
+    heavy-ball form PyTorch's SGD uses, the optimiser of Section 5.1).  fp64;
+    returns (x_new, v_new or None)."""
+    x = np.asarray(x, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    if momentum_buf is None:
+        return x - lr * g, None
+    v = momentum * np.asarray(momentum_buf, dtype=np.float64) + g
+    return x - lr * v, v
+
+
 def aggregate(rule: str, G, f: int):
     """GAR(f, [G_1..G_n]) -> fp64 vector of dimension d."""
     G = np.asarray(G)

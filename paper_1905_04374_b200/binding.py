@@ -59,6 +59,7 @@ class GarParams(C.Structure):
         ("m", C.c_int32), ("theta", C.c_int32), ("median_of_agr", C.c_int32), ("even_median", C.c_int32),
         ("dist_out", C.c_void_p), ("selection_out", C.c_void_p),
         ("distance_mode", C.c_int32), ("reserved", C.c_int32),
+        ("sgd_params", C.c_void_p), ("sgd_momentum_buf", C.c_void_p), ("sgd_lr", C.c_float), ("sgd_momentum", C.c_float),
     ]
 
 
@@ -180,17 +181,27 @@ def gar_aggregate(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = 
 def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = None, stream=None,
                      workspace: torch.Tensor | None = None, m: int = 0, theta: int = 0, median_of_agr: int = 0,
                      dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None,
-                     even_median=0, distance_mode=0):
+                     even_median=0, distance_mode=0, sgd_params: torch.Tensor | None = None,
+                     sgd_momentum_buf: torch.Tensor | None = None, sgd_lr: float = 0.0, sgd_momentum: float = 0.0,
+                     store_out: bool = True):
     """gar_aggregate_ex: row stride taken from the tensor; optional workspace
     (uint8 CUDA tensor), options and outputs (dist_out float64 [n, n];
-    selection_out uint8 CUDA tensor of sizeof(gar_selection_t))."""
+    selection_out uint8 CUDA tensor of sizeof(gar_selection_t)); optional fused SGD step on
+    sgd_params / sgd_momentum_buf (CUDA float32 [d], updated in place); store_out=False with a
+    fused step passes out = NULL (returns None)."""
     _dev_f32(grads, "grads")
     n, d, ld = _rows(grads)
-    if out is None:
+    if out is None and (store_out or sgd_params is None):
         out = torch.empty(d, dtype=torch.float32, device=grads.device)
     p = GarParams()
     p.rule, p.n, p.f, p.d, p.ld = _rule(rule), n, f, d, ld
-    p.grads, p.out, p.stream = grads.data_ptr(), out.data_ptr(), _stream(stream)
+    p.grads, p.stream = grads.data_ptr(), _stream(stream)
+    p.out = out.data_ptr() if out is not None else None
+    if sgd_params is not None:
+        p.sgd_params = _dev_f32(sgd_params, "sgd_params").data_ptr()
+        p.sgd_lr, p.sgd_momentum = sgd_lr, sgd_momentum
+    if sgd_momentum_buf is not None:
+        p.sgd_momentum_buf = _dev_f32(sgd_momentum_buf, "sgd_momentum_buf").data_ptr()
     if workspace is not None:
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     p.m, p.theta, p.median_of_agr = m, theta, median_of_agr

@@ -101,7 +101,7 @@ bool overlaps(const void* a, size_t abytes, const void* b, size_t bbytes) {
 }
 
 // Enqueue the whole rule for device buffers.
-int enqueue(int rule, const float* grads, int n, int f, int64_t d, int64_t ld, float* out, int m, int theta,
+int enqueue(int rule, const float* grads, int n, int f, int64_t d, int64_t ld, const gar::K3Out& out, int m, int theta,
             int median_of_agr, int even_median, int distance_mode, const Workspace& ws, double* dist_out,
             gar_selection_t* sel_out, int sm_count, cudaStream_t stream) {
     const int beta = beta_for(rule, theta, f);
@@ -199,11 +199,20 @@ int gar_aggregate_ex(const gar_params_t* p) {
     if (!p) return GAR_ERR_INVALID_ARG;
     int rc = basic_checks(p->rule, p->n, p->f, p->d);
     if (rc != GAR_OK) return rc;
-    if (!p->grads || !p->out) return GAR_ERR_INVALID_ARG;
+    if (!p->grads || (!p->out && !p->sgd_params)) return GAR_ERR_INVALID_ARG;
+    if (p->sgd_momentum_buf && !p->sgd_params) return GAR_ERR_INVALID_ARG;
     const int64_t ld = p->ld ? p->ld : p->d;
     if (ld < p->d) return GAR_ERR_INVALID_ARG;
-    if (overlaps(p->grads, (size_t(p->n - 1) * ld + p->d) * sizeof(float), p->out, size_t(p->d) * sizeof(float)))
-        return GAR_ERR_INVALID_ARG;
+    {
+        const size_t gbytes = (size_t(p->n - 1) * ld + p->d) * sizeof(float), vbytes = size_t(p->d) * sizeof(float);
+        const float* vecs[3] = {p->out, p->sgd_params, p->sgd_momentum_buf};
+        for (int a = 0; a < 3; ++a) {
+            if (!vecs[a]) continue;
+            if (overlaps(p->grads, gbytes, vecs[a], vbytes)) return GAR_ERR_INVALID_ARG;
+            for (int b = a + 1; b < 3; ++b)
+                if (vecs[b] && overlaps(vecs[a], vbytes, vecs[b], vbytes)) return GAR_ERR_INVALID_ARG;
+        }
+    }
     int theta = default_theta(p->rule, p->n, p->f);
     int m = 0;
     if (p->m != 0) {
@@ -221,7 +230,8 @@ int gar_aggregate_ex(const gar_params_t* p) {
     Workspace ws{};
     rc = resolve_workspace(p->workspace, p->workspace_bytes, &st, &ws);
     if (rc != GAR_OK) return rc;
-    return enqueue(p->rule, p->grads, p->n, p->f, p->d, ld, p->out, m, theta, p->median_of_agr, p->even_median,
+    const gar::K3Out out{p->out, p->sgd_params, p->sgd_momentum_buf, p->sgd_lr, p->sgd_momentum};
+    return enqueue(p->rule, p->grads, p->n, p->f, p->d, ld, out, m, theta, p->median_of_agr, p->even_median,
                    p->distance_mode, ws, p->dist_out, p->selection_out, st->sm_count,
                    static_cast<cudaStream_t>(p->stream));
 }
@@ -288,7 +298,8 @@ int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, gar_s
     DeviceState* st = nullptr;
     int rc = device_state(&st, false);
     if (rc != GAR_OK) return rc;
-    cudaError_t err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg ? 1 : 0, out, st->sm_count,
+    const gar::K3Out o{out, nullptr, nullptr, 0.0f, 0.0f};
+    cudaError_t err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg ? 1 : 0, o, st->sm_count,
                                              static_cast<cudaStream_t>(stream));
     return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
 }
@@ -339,7 +350,8 @@ int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, fl
         return GAR_ERR_CUDA;
     Workspace ws{st->workspace};
     const int theta = default_theta(rule, n, f);
-    rc = enqueue(rule, st->stage_grads, n, f, d, d, st->stage_out, 0, theta, 0, GAR_EVEN_MEDIAN_LOWER, GAR_DISTANCES_AUTO,
+    const gar::K3Out stage_out{st->stage_out, nullptr, nullptr, 0.0f, 0.0f};
+    rc = enqueue(rule, st->stage_grads, n, f, d, d, stage_out, 0, theta, 0, GAR_EVEN_MEDIAN_LOWER, GAR_DISTANCES_AUTO,
                  ws, nullptr, nullptr, st->sm_count, s);
     if (rc != GAR_OK) return rc;
     if (cudaMemcpyAsync(out, st->stage_out, size_t(d) * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)

@@ -47,6 +47,15 @@ constexpr int kSlotRowExp    = 2100;    // .. +63: the tensor-core kernel's fina
 constexpr int kSlotNonfinite = 2300;    // 2300, 2301: masks of rows that hold Inf or NaN
 constexpr int kSlotError     = 2302;    // a bounded wait gave up
 
+// Where the coordinate kernel puts a coordinate's result: the aggregate itself (out, may be null
+// when a step is fused) and/or an SGD step on x with optional momentum buffer v (Eq. 2).
+struct K3Out {
+    float* out;
+    float* x;
+    float* v;
+    float  lr, mu;
+};
+
 // ---- kernel launchers (one per translation unit) --------------------------
 // Pairwise squared distances of n rows over columns [0, d); result in dist[n*n].
 // mode: a gar_distance_mode_t.
@@ -66,7 +75,7 @@ cudaError_t launch_schedule_only(gar_selection_t* sel, cudaStream_t stream);
 
 // Coordinate phase.
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
-                              gar_selection_t* sel, int theta, int preagg, float* out,
+                              gar_selection_t* sel, int theta, int preagg, const K3Out& out,
                               int sm_count, cudaStream_t stream);
 
 // One warp waits, bounded, on a barrier nobody arrives on; result[0] = status, result[1] = ns.

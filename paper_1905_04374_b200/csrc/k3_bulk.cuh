@@ -63,7 +63,7 @@ struct KBPlan {
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(KBShape<V>::THREADS)
 k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64_t ld, gar_selection_t* __restrict__ sel,
-        float* __restrict__ out, int pool_bytes) {
+        const K3Out out, int pool_bytes) {
     constexpr int KB_TC = KBShape<V>::TC, KB_CT = KBShape<V>::CT, KB_THREADS = KBShape<V>::THREADS;
     constexpr int KB_ROW_BYTES = KBShape<V>::ROW_BYTES;
     __shared__ KBPlan plan;
@@ -73,7 +73,7 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
         const int status = k3_check(sel, n, theta_arg, PREAGG);
         if (status != GAR_OK) {                   // nothing usable: the output says so
             for (int64_t i = blockIdx.x; i < ntiles; i += gridDim.x)
-                for (int c = tid; c < KB_TC; c += KB_THREADS) out[i * KB_TC + c] = CUDART_NAN_F;
+                for (int c = tid; c < KB_TC; c += KB_THREADS) k3_store_nan(out, i * KB_TC + c);
             if (blockIdx.x == 0 && tid == 0 && sel->status == GAR_OK) sel->status = status;
             return;
         }
@@ -316,7 +316,7 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
                 asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(kb_smem_u32(&plan.empty[st])) : "memory");
             float res[V];
             k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, med_agr, even_mean, median_only, res);
-            store_vec<V>(out + (first + i * step) * KB_TC + tid * V, res);
+            k3_store<V>(out, (first + i * step) * KB_TC + tid * V, res);
             if (++st == nstages) { st = 0; parity ^= 1u; }
         }
     }

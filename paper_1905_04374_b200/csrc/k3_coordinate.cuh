@@ -65,6 +65,32 @@ template <int V> __device__ __forceinline__ void read_vec(const float* p, float 
     else { float4 t = *reinterpret_cast<const float4*>(p); x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w; }
 }
 
+// A coordinate's result goes out: the aggregate, and/or the fused SGD step (v <- mu v + g, x <- x - lr v).
+template <int V> __device__ __forceinline__ void k3_store(const K3Out& o, int64_t t, const float (&res)[V]) {
+    if (o.out) store_vec<V>(o.out + t, res);
+    if (o.x) {
+        float x[V], step[V];
+        read_vec<V>(o.x + t, x);
+        if (o.v) {
+            float v[V];
+            read_vec<V>(o.v + t, v);
+#pragma unroll
+            for (int k = 0; k < V; ++k) { v[k] = fmaf(o.mu, v[k], res[k]); step[k] = v[k]; }
+            store_vec<V>(o.v + t, v);
+        } else {
+#pragma unroll
+            for (int k = 0; k < V; ++k) step[k] = res[k];
+        }
+#pragma unroll
+        for (int k = 0; k < V; ++k) x[k] = fmaf(-o.lr, step[k], x[k]);
+        store_vec<V>(o.x + t, x);
+    }
+}
+// Nothing usable was computed: the aggregate says so; the model and its momentum stay as they are.
+__device__ __forceinline__ void k3_store_nan(const K3Out& o, int64_t t) {
+    if (o.out) o.out[t] = CUDART_NAN_F;
+}
+
 __device__ __forceinline__ void prefetch_l1(const void* p) {
     asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
 }
@@ -322,13 +348,13 @@ __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* _
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(K3_THREADS)
 k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin, int64_t t_end, int64_t ld,
-              gar_selection_t* __restrict__ sel, float* __restrict__ out, int loose_cap) {
+              gar_selection_t* __restrict__ sel, const K3Out out, int loose_cap) {
     __shared__ K3Plan plan;
     extern __shared__ __align__(16) float k3_dyn[];
     const int status = k3_check(sel, n, theta_arg, PREAGG);
     if (status != GAR_OK) {                       // nothing usable: the output says so
         for (int64_t t = t_begin + int64_t(blockIdx.x) * blockDim.x + threadIdx.x; t < t_end; t += int64_t(gridDim.x) * blockDim.x)
-            out[t] = CUDART_NAN_F;
+            k3_store_nan(out, t);
         if (blockIdx.x == 0 && threadIdx.x == 0 && sel->status == GAR_OK) sel->status = status;
         return;
     }
@@ -467,13 +493,13 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
 
         float res[V];
         k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, PREAGG && med_agr, even_mean, median_only, res);
-        store_vec<V>(out + t, res);
+        k3_store<V>(out, t, res);
     }
 }
 
 template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
-                        int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
+                        int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 
 }  // namespace gar

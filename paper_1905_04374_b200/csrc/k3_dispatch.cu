@@ -13,19 +13,20 @@ namespace gar {
 
 template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
-                        int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream);
+                        int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 #define K3_DECL(P)                                                                                              \
     template <>                                                                                                 \
     cudaError_t launch_k3_p<P>(const float*, int, int64_t, int64_t, gar_selection_t*, int, int, int, int,       \
-                               float*, int, cudaStream_t);                                                      \
+                               const K3Out&, int, cudaStream_t);                                                    \
     template <> int bulk_ctas_for<P>(int, int, int);
 K3_P_LIST(K3_DECL)
 #undef K3_DECL
 
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, gar_selection_t* sel,
-                              int theta, int preagg, float* out, int sm_count, cudaStream_t stream) {
-    const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out);
+                              int theta, int preagg, const K3Out& out, int sm_count, cudaStream_t stream) {
+    const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out.out) |
+                        reinterpret_cast<uintptr_t>(out.x) | reinterpret_cast<uintptr_t>(out.v);
     int vec_max = 1;                                      // what the alignment allows
     if (a % 16 == 0 && ld % 4 == 0) vec_max = 4;
     else if (a % 8 == 0 && ld % 2 == 0) vec_max = 2;

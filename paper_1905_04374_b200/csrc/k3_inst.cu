@@ -43,7 +43,7 @@ static int bulk_ctas(int n, int theta) {
 // Full tiles [0, *covered) through the staged kernel, `ctas` CTAs per SM.
 template <int P, bool PREAGG>
 static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta,
-                            int ctas, float* out, int sm_count, cudaStream_t stream, int64_t* covered) {
+                            int ctas, const K3Out& out, int sm_count, cudaStream_t stream, int64_t* covered) {
     constexpr bool EXACT = (K3_EXACT != 0);
     constexpr int V = BulkV<PREAGG>::V;
     using S = KBShape<V>;
@@ -76,7 +76,7 @@ static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, gar_se
 
 // Coordinates [t0, d): t0 is a multiple of 4.
 template <int P, bool PREAGG, int V>
-static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, int64_t ld, gar_selection_t* sel, float* out,
+static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, int64_t ld, gar_selection_t* sel, const K3Out& out,
                        int sm_count, cudaStream_t stream) {
     constexpr bool EXACT = (K3_EXACT != 0);
     int threads = K3_THREADS, threads1 = K3_THREADS;
@@ -119,7 +119,7 @@ static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, 
 
 template <>
 cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
-                              int vec, int bulk_ctas, float* out, int sm_count, cudaStream_t stream) {
+                              int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream) {
     int64_t t0 = 0;
     if (bulk_ctas > 0) {                         // whole tiles staged through shared memory, the rest below
         const cudaError_t err = preagg ? run_bulk<K3_P, true>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0)

@@ -41,14 +41,16 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
                    'offsetof(gar_selection_t,sets), offsetof(gar_selection_t,nu),'
                    'offsetof(gar_selection_t,add_pos), offsetof(gar_selection_t,scores), sizeof(gar_params_t),'
                    'offsetof(gar_selection_t,even_median), offsetof(gar_selection_t,winners),'
-                   'offsetof(gar_params_t,even_median), offsetof(gar_params_t,distance_mode));}')
+                   'offsetof(gar_params_t,even_median), offsetof(gar_params_t,distance_mode));'
+                   'printf("%zu %zu\\n", offsetof(gar_params_t,sgd_params), offsetof(gar_params_t,sgd_lr));}')
     exe = tmp_path / "sz"
     subprocess.check_call(["g++", "-I" + os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(v) for v in subprocess.check_output([str(exe)]).split()]
     S = pkg.GarSelection
     P = pkg.GarParams
     assert got == [C.sizeof(S), S.sets.offset, S.nu.offset, S.add_pos.offset, S.scores.offset,
-                   C.sizeof(P), S.even_median.offset, S.winners.offset, P.even_median.offset, P.distance_mode.offset]
+                   C.sizeof(P), S.even_median.offset, S.winners.offset, P.even_median.offset, P.distance_mode.offset,
+                   P.sgd_params.offset, P.sgd_lr.offset]
 
 
 def test_version_and_strings(pkg):
@@ -104,7 +106,15 @@ def test_errors_before_any_launch(pkg):
     assert L.gar_aggregate_ex(C.byref(p)) == 1
     p.even_median, p.distance_mode = 0, 7                                  # unknown distance mode
     assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.distance_mode = 0
+    p.out, p.sgd_params = None, None                                       # neither an output nor a fused step
+    assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.out, p.sgd_momentum_buf = 1 << 30, 1 << 31                            # a momentum buffer without parameters
+    assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.sgd_params = (1 << 30) + 40                                          # parameters overlapping the output
+    assert L.gar_aggregate_ex(C.byref(p)) == 1
     assert L.gar_pairwise_distances_mode(fake, 11, 100, 100, fake, None, 0, 5, None) == 1
+    assert L.gar_reduce_partials(fake, 0, 11, fake, None) == 1 and L.gar_reduce_partials(fake, 2, 65, fake, None) == 3
     assert L.gar_select(5, fake, 11, 2, 0, 0, 0, 3, fake, None) == 1       # unknown even-median mode
     assert L.gar_selftest_bounded_wait(0, fake, None) == 1
     assert L.gar_selftest_bounded_wait(100, None, None) == 1

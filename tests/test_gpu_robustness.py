@@ -293,3 +293,52 @@ def test_bounded_wait_runs_out_with_a_status(pkg):
     print(f"bounded wait: {ns / 200:.0f} ns per suspended poll at 200, {ns2 / 2000:.0f} ns at 2000")
     x = torch.ones(10, device=DEV)
     assert float(x.sum()) == 10.0
+
+
+# ----------------------------------------------------------- SGD step fused into the store
+@pytest.mark.parametrize("d", [4099, 450_048])
+@pytest.mark.parametrize("with_momentum", [False, True])
+def test_fused_sgd_step(pkg, d, with_momentum):
+    """Eq. 2 with the aggregate never written out: x <- x - lr * GAR (or through a momentum buffer),
+    three steps in a row, against the oracle's step applied to the oracle's aggregate."""
+    n, f = 15, 3
+    lr, mu = 0.05, 0.9
+    gen = torch.Generator(device=DEV).manual_seed(9)
+    x = torch.randn(d, generator=gen, device=DEV)
+    v = torch.zeros(d, device=DEV) if with_momentum else None
+    xh = x.cpu().numpy().astype(np.float64)
+    vh = np.zeros(d) if with_momentum else None
+    for step in range(3):
+        G, _ = pkg.workloads.make_gradients(5, d=d, device=DEV, seed=500 + step)
+        Gh = G.cpu().numpy()
+        keep = pkg.gar_aggregate_ex("multi_bulyan", G, f, sgd_params=x, sgd_momentum_buf=v, sgd_lr=lr, sgd_momentum=mu,
+                                    store_out=(step == 0))
+        agg, tab = rule_tables("multi_bulyan", Gh, f)
+        if step == 0:                            # the aggregate is still stored when an output is given
+            assert_outputs_match(keep.cpu().numpy(), agg, G=Gh, tables=tab)
+        else:
+            assert keep is None
+        xh, vh = O.sgd_step(xh, agg, lr, momentum_buf=vh, momentum=mu)
+        # the same tie-aware bar as for the aggregate, scaled by what multiplies it on the way to x
+        scale = lr * sum(mu ** k for k in range(step + 1)) if with_momentum else lr * (step + 1)
+        bad = np.abs(x.cpu().numpy() - xh) > 1e-5 * (1 + np.abs(xh)) + scale * 1e-5 * (1 + np.abs(agg))
+        assert bad.sum() <= max(3, int(6e-4 * d)), f"step {step}: {int(bad.sum())} coordinates of x off"
+        if with_momentum:
+            badv = np.abs(v.cpu().numpy() - vh) > 1e-5 * (1 + np.abs(vh)) * (step + 1)
+            assert badv.sum() <= max(3, int(6e-4 * d))
+        # keep the two sides from drifting apart through legitimate near-tie choices
+        xh = x.cpu().numpy().astype(np.float64)
+        if with_momentum:
+            vh = v.cpu().numpy().astype(np.float64)
+
+
+def test_fused_sgd_leaves_the_model_alone_on_failure(pkg):
+    n, f, d = 15, 3, 50_000
+    G, _ = pkg.workloads.make_gradients(5, d=d, device=DEV)
+    D = torch.full((n, n), float("nan"), dtype=torch.float64, device=DEV)
+    sel = pkg.gar_select("multi_bulyan", D, n, f)
+    assert pkg.read_selection(sel).status == 6
+    # the fused step goes through gar_aggregate_ex only; the same kernels refuse a poisoned selection
+    # for the plain output, which is what decides whether x is touched
+    out = pkg.gar_coordinate_phase(G, sel, pkg.gar_theta("multi_bulyan", n, f), 1)
+    assert bool(torch.isnan(out).all())

@@ -451,3 +451,32 @@ def test_identical_byzantine_rows_and_selection_is_honest():
         assert not (set(S) & set(byz))
     D = O.pairwise_sq_distances(G)
     assert D[2, 7] == 0 and D[7, 11] == 0
+
+
+# ------------------------------------------------------------------ the SGD step (Eq. 2)
+def test_sgd_step_closed_form_and_library():
+    rng = np.random.default_rng(3)
+    x0 = rng.standard_normal(50)
+    gs = [rng.standard_normal(50) for _ in range(4)]
+    lr, mu = 0.1, 0.9
+    # plain SGD: x_k = x_0 - lr * sum of the gradients
+    x = x0.copy()
+    for g in gs:
+        x, v = O.sgd_step(x, g, lr)
+        assert v is None
+    np.testing.assert_allclose(x, x0 - lr * np.sum(gs, axis=0), rtol=0, atol=1e-14)
+    # momentum: v_k = sum_i mu^(k-i) g_i (closed form), and PyTorch's SGD on the same numbers
+    x, v = x0.copy(), np.zeros(50)
+    px = torch.tensor(x0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.SGD([px], lr=lr, momentum=mu)
+    for k, g in enumerate(gs):
+        x, v = O.sgd_step(x, g, lr, momentum_buf=v, momentum=mu)
+        want_v = sum(mu ** (k - i) * gs[i] for i in range(k + 1))
+        np.testing.assert_allclose(v, want_v, rtol=0, atol=1e-13)
+        px.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(x, px.detach().numpy(), rtol=0, atol=1e-13)
+    # a sign or operand mix-up shows on a one-coordinate example: x = 1, g = 2, lr = 0.5 -> 0
+    assert O.sgd_step([1.0], [2.0], 0.5)[0][0] == 0.0
+    xn, vn = O.sgd_step([1.0], [2.0], 0.5, momentum_buf=[4.0], momentum=0.5)
+    assert vn[0] == 4.0 and xn[0] == -1.0
