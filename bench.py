@@ -418,6 +418,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1 or args.force_sharded:
+        os.environ.setdefault("NCCL_DEBUG", "WARN")     # keep NCCL's version banner off stdout: one JSON line
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = args.config

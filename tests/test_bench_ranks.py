@@ -47,3 +47,18 @@ def test_reference_arm_under_torchrun_prints_one_line():
     rec = json.loads(lines[0])
     assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["cpu_baseline"]["kind"] == "oracle"
     assert rec["e2e"]["h2d_bytes_per_step"] == 0 and rec["value"] > 0
+
+
+def test_paper_protocol_statistic_drops_the_two_farthest_from_the_median():
+    """Section 5.1: seven runs, the two farthest from the median removed, mean and deviation of five."""
+    from paper_1905_04374_b200.paper_sweep import robust_mean_std
+    runs = [10.0, 10.2, 9.9, 10.1, 50.0, 10.0, 0.5]          # median 10.0; 50.0 and 0.5 are the outliers
+    mean, std = robust_mean_std(runs)
+    kept = [10.0, 10.2, 9.9, 10.1, 10.0]
+    assert abs(mean - sum(kept) / 5) < 1e-12
+    assert abs(std - (sum((k - mean) ** 2 for k in kept) / 5) ** 0.5) < 1e-12
+    # both outliers on one side are dropped as well
+    mean2, _ = robust_mean_std([1.0, 1.0, 1.0, 1.0, 1.0, 9.0, 8.0])
+    assert mean2 == 1.0
+    # with five runs nothing is dropped
+    assert robust_mean_std([1.0, 2.0, 3.0, 4.0, 5.0])[0] == 3.0

@@ -350,3 +350,50 @@ def test_host_entry_point(pkg):
     out = pkg.gar_aggregate_host("multi_bulyan", host, f)
     dev = pkg.gar_aggregate("multi_bulyan", G, f).cpu()
     assert torch.equal(out, dev)
+
+
+# --------------------------------------------------- the paper's own timing inputs (Section 5.1)
+@pytest.mark.parametrize("n", list(range(7, 40, 4)) + [39])
+@pytest.mark.parametrize("rule", ["multi_bulyan", "multi_krum", "median"])
+def test_paper_grid_input_family(pkg, n, rule):
+    """n gradients i.i.d. U(0,1)^d with f = floor((n-3)/4): the inputs of the paper's timing grid."""
+    f = (n - 3) // 4
+    d = 100_000
+    G = pkg.workloads.make_uniform(n, d, device=DEV, seed=1905 + n)
+    Gh = G.cpu().numpy()
+    sel_dev = pkg.new_selection(DEV)
+    out = pkg.gar_aggregate_ex(rule, G, f, selection_out=sel_dev).cpu().numpy()
+    want, tab = rule_tables(rule, Gh, f)
+    if tab is None:
+        assert_outputs_match(out, want)
+        return
+    sel = pkg.read_selection(sel_dev)
+    compared = assert_selection_match(sel, tab["rounds"], True)
+    if compared == len(tab["rounds"]):
+        assert_outputs_match(out, want, G=Gh, tables=tab)
+    else:
+        winners = [sel.winners[r] for r in range(sel.theta)]
+        sets = [[i for i in range(n) if (sel.sets[r] >> i) & 1] for r in range(sel.theta)]
+        want2, gap2 = O.coordinate_phase(Gh, winners, sets, sel.beta)
+        assert_outputs_match(out, want2, G=Gh, tables=dict(winners=winners, sets=sets, beta=sel.beta, gap=gap2))
+
+
+@pytest.mark.parametrize("cfg,n,f", [(5, 15, 3), (2, 23, 5), (4, 51, 12)])
+def test_multi_krum_every_kind_of_m(pkg, cfg, n, f):
+    """Section 3: Theorem 1 holds for any m <= n-f-2; m = 1 is Krum."""
+    d = 50_001
+    G, Gh, _ = draw(pkg, cfg, d)
+    D = O.pairwise_sq_distances(Gh)
+    for m in sorted({1, 2, (n - f - 2) // 2, n - f - 3, n - f - 2}):
+        sel_dev = pkg.new_selection(DEV)
+        out = pkg.gar_aggregate_ex("multi_krum", G, f, m=m, selection_out=sel_dev).cpu().numpy()
+        want, tab = rule_tables("multi_krum", Gh, f, D=D, m=m)
+        sel = pkg.read_selection(sel_dev)
+        rnd = tab["rounds"][0]
+        assert sel.m[0] == m and sel.winners[0] == rnd.winner
+        if rnd.gap_set > 1e-6:
+            assert sel.sets[0] == sum(1 << i for i in rnd.selected)
+            assert_outputs_match(out, want)
+    krum = pkg.gar_aggregate("krum", G, f).cpu().numpy()
+    one = pkg.gar_aggregate_ex("multi_krum", G, f, m=1).cpu().numpy()
+    assert np.array_equal(krum, one)
