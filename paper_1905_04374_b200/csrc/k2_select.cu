@@ -26,7 +26,7 @@ struct K2Smem {
     uint8_t  sj[NMAX][NMAX];      // per row: their indices
     double   score[NMAX];
     double   pick[NMAX][4];       // per round: s(1), s(2), s(m), s(m+1)
-    unsigned long long setmask[NMAX];   // per round: the m best
+    uint8_t  order[NMAX][NMAX];   // per round: the remaining rows by rank (ranks are distinct: one writer per entry)
     unsigned long long alive;
 };
 
@@ -53,6 +53,10 @@ struct PlanSmem {
     int usage[NMAX];
     int saved[NMAX];        // slot -> saved index or -1
     int offset[NMAX + 1];
+    // shared-memory copies of what the single-threaded passes walk over (a dependent chain of
+    // global loads per slot would cost microseconds)
+    int winner_of_slot[NMAX];
+    uint8_t src[NMAX], save[NMAX];
 };
 
 __device__ __forceinline__ void plan_choose(const PlanSmem& ps, int s, bool restricted, int& src, unsigned long long& adds) {
@@ -81,8 +85,10 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
     const int tid = threadIdx.x;
     if (tid < theta) {
         const int r = theta - 1 - tid;
-        ps.slotset[tid] = sel->sets[r];
-        sel->m[r] = __popcll(sel->sets[r]);
+        const unsigned long long set_r = sel->sets[r];
+        ps.slotset[tid] = set_r;
+        ps.winner_of_slot[tid] = sel->winners[r];
+        sel->m[r] = __popcll(set_r);
         ps.usage[tid] = 0;
         ps.saved[tid] = -1;
     }
@@ -93,7 +99,7 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
         unsigned long long suffix = ~0ull, next_suffix = ~0ull;
         for (int s = theta - 1; s >= 0; --s) {
             suffix = next_suffix & ps.slotset[s];                 // present in all slots >= s
-            const int w = sel->winners[theta - 1 - s];
+            const int w = ps.winner_of_slot[s];
             if (w >= 0 && w < NMAX) {
                 u |= 1ull << w;
                 // chained: permanent from slot s on, and not already permanent from slot s+... (a winner
@@ -113,7 +119,7 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
         ps.chain = chain;
         unsigned long long covered = base, loose_all = 0ull;
         for (int s = 0; s < theta; ++s) {
-            if ((chain >> s) & 1ull) covered |= 1ull << sel->winners[theta - 1 - s];
+            if ((chain >> s) & 1ull) covered |= 1ull << ps.winner_of_slot[s];
             ps.loose[s] = ps.slotset[s] & ~covered;
             loose_all |= ps.loose[s];
         }
@@ -152,9 +158,11 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
         int src; unsigned long long adds;
         plan_choose(ps, tid, true, src, adds);
         ps.addmask[tid] = adds;
-        sel->slot_src[tid] = src == -1 ? uint8_t(GAR_SRC_ZERO) : src == -2 ? uint8_t(GAR_SRC_CONT) : uint8_t(ps.saved[src]);
+        ps.src[tid] = src == -1 ? uint8_t(GAR_SRC_ZERO) : src == -2 ? uint8_t(GAR_SRC_CONT) : uint8_t(ps.saved[src]);
+        ps.save[tid] = ps.saved[tid] >= 0 ? uint8_t(ps.saved[tid]) : uint8_t(GAR_SAVE_NONE);
+        sel->slot_src[tid] = ps.src[tid];
         sel->slot_nadd[tid] = uint8_t(__popcll(adds));
-        sel->slot_save[tid] = ps.saved[tid] >= 0 ? uint8_t(ps.saved[tid]) : uint8_t(GAR_SAVE_NONE);
+        sel->slot_save[tid] = ps.save[tid];
     }
     __syncthreads();
     if (tid == 0) {
@@ -164,8 +172,8 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
             ps.offset[s] = acc;
             const int na = __popcll(ps.addmask[s]);
             acc += na;
-            const bool noop = (na == 0) && sel->slot_save[s] == GAR_SAVE_NONE &&
-                              (sel->slot_src[s] == GAR_SRC_CONT || (s == 0 && sel->slot_src[s] == GAR_SRC_ZERO));
+            const bool noop = (na == 0) && ps.save[s] == GAR_SAVE_NONE &&
+                              (ps.src[s] == GAR_SRC_CONT || (s == 0 && ps.src[s] == GAR_SRC_ZERO));
             if (!noop) corr |= 1ull << s;
         }
         ps.offset[theta] = acc;
@@ -246,7 +254,6 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         sm.sj[i][rank] = uint8_t(j);
     }
     if (tid == 0) sm.alive = (n == 64) ? ~0ull : ((1ull << n) - 1ull);
-    if (tid < NMAX) sm.setmask[tid] = 0ull;
     __syncthreads();
 
     const bool clamp = (rule == GAR_BULYAN);
@@ -304,7 +311,7 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
                     if (rank == 1) sm.pick[r][1] = s;
                     if (rank == m - 1) sm.pick[r][2] = s;
                     if (rank == m) sm.pick[r][3] = s;
-                    if (rank < m) atomicOr(&sm.setmask[r], 1ull << i);
+                    sm.order[r][rank] = uint8_t(i);
                 }
             }
         }
@@ -316,7 +323,9 @@ k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, in
         int m = 1;
         if (rule == GAR_MULTI_BULYAN) m = k - f - 2;
         else if (rule == GAR_MULTI_KRUM) m = m_user > 0 ? m_user : n - f - 2;
-        sel->sets[r] = sm.setmask[r];
+        unsigned long long mask = 0ull;                     // the m best ranks of the round
+        for (int j = 0; j < m; ++j) mask |= 1ull << sm.order[r][j];
+        sel->sets[r] = mask;
         sel->gap_winner[r] = (k > 1) ? rel_gap(sm.pick[r][0], sm.pick[r][1]) : INFINITY;
         sel->gap_set[r] = (m < k) ? rel_gap(sm.pick[r][2], sm.pick[r][3]) : INFINITY;
     }
