@@ -33,9 +33,9 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per coordinate of the dominant kernels, from the ncu captures under
 # profiles/ (kernel, n) -> bytes; a kernel that changed since its capture has no entry.
 NCU_DRAM_BYTES_PER_COORD = {
-    ("k1_distances", 39): 331.2e6 / 2097152, ("k3_coordinate", 39): 252.4e6 / 2097152,     # k1_umma / k3_bulk<19, V=2>
-    ("k1_distances", 51): 324.8e6 / 1572864, ("k3_coordinate", 51): 316.8e6 / 1572864,     # k1_umma / k3_bulk<25, V=2>
-    ("k1_distances", 15): 256.4e6 / 4194304, ("k3_coordinate", 15): 195.2e6 / 4194304,     # k1_direct_bulk / k3_bulk<7, V=4>
+    ("k1_distances", 39): 1313.0e6 / 8388608, ("k3_coordinate", 39): 1041.5e6 / 8388608,     # k1_umma (packed) / k3_bulk<19, V=2>
+    ("k1_distances", 51): 1718.0e6 / 8388608, ("k3_coordinate", 51): 1680.0e6 / 8388608,     # k1_umma (wide) / k3_bulk<25, V=2>
+    ("k1_distances", 15): 1011.4e6 / 16777216, ("k3_coordinate", 15): 731.8e6 / 16777216,    # k1_direct_bulk / k3_bulk<7, V=4>
 }
 
 
