@@ -202,7 +202,7 @@ def launches_per_aggregation(n: int, d: int, theta: int) -> int:
     return k1 + 1 + k3
 
 
-def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant=True):
+def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant=True, distance_mode="auto"):
     """Device-side measurement of one workload resident in HBM: `steps` whole aggregations timed
     with CUDA events on the launch stream (max over ranks), then each stage alone."""
     import torch
@@ -217,7 +217,10 @@ def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant
     stream = torch.cuda.current_stream()
 
     def step():
-        pkg.gar_aggregate("multi_bulyan", G, f, out=out)
+        if distance_mode == "auto":
+            pkg.gar_aggregate("multi_bulyan", G, f, out=out)
+        else:
+            pkg.gar_aggregate_ex("multi_bulyan", G, f, out=out, distance_mode=distance_mode)
 
     for _ in range(max(warmup, 3)):
         step()
@@ -242,9 +245,10 @@ def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant
     ws = torch.zeros(pkg.gar_workspace_bytes("multi_bulyan", n, f, d), dtype=torch.uint8, device=dev)
     dmat = torch.empty(n, n, dtype=torch.float64, device=dev)
     sel = pkg.new_selection(dev)
-    pkg.gar_pairwise_distances(G, dist=dmat, workspace=ws)
+    pkg.gar_pairwise_distances(G, dist=dmat, workspace=ws, distance_mode=distance_mode)
     pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel)
-    k1_ms = event_time_ms(lambda: pkg.gar_pairwise_distances(G, dist=dmat, workspace=ws), reps, stream)
+    k1_ms = event_time_ms(lambda: pkg.gar_pairwise_distances(G, dist=dmat, workspace=ws, distance_mode=distance_mode),
+                          reps, stream)
     k2_ms = event_time_ms(lambda: pkg.gar_select("multi_bulyan", dmat, n, f, sel=sel), reps, stream)
     k3_ms = event_time_ms(lambda: pkg.gar_coordinate_phase(G, sel, theta_a, 1, out=out), reps, stream)
     selh = pkg.read_selection(sel)
@@ -426,7 +430,8 @@ def run_ours(args):
         run_sharded(pkg, args, dev, world, rank, local)
         dist.destroy_process_group()
         return
-    main, G = measure_workload(pkg, cfg, dev, args.steps, args.warmup, world, local, d=args.d)
+    main, G = measure_workload(pkg, cfg, dev, args.steps, args.warmup, world, local, d=args.d,
+                               distance_mode=args.distance_mode)
     wl = pkg.workloads.WORKLOADS[cfg]
     n, f, d = main["n"], main["f"], main["d"]
     if rank != 0:
@@ -497,6 +502,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--quick", action="store_true", help="device-side numbers of the chosen workload only")
+    ap.add_argument("--distance-mode", default="auto", choices=["auto", "difference"],
+                    help="difference: the fp32 difference-form distance kernels instead of the tensor-core one")
     ap.add_argument("--force-sharded", action="store_true",
                     help="run the sharded (N > 1) code path even with one rank (under torchrun, for checking it)")
     args = ap.parse_args()

@@ -16,7 +16,11 @@
 //   producers (3 rows each)  cp.async ring -> quantise -> byte tiles in shared memory, laid out as
 //                            the K-major, unswizzled operand of tcgen05.mma: 16-byte chunks of a
 //                            row, rows in groups of eight (128 bytes), chunk stride LBO
-//   one MMA warp             per slab 4 k-steps x 2 instructions from one lane:
+//   one MMA warp             per slab 4 k-steps from one lane.  n <= 40 ("packed" tile: limb matrices
+//                            40 rows apart, 128 rows in all): ONE 128 x 128 instruction per k-step with
+//                            the tile as both operands, all nine limb products at once, 128 tensor-memory
+//                            columns per accumulator set.  Larger n ("wide" tile, limb matrices 64 rows
+//                            apart): two instructions per k-step,
 //                            [L1; L2] x [L1; L2; L3]^T (128 x 192) and [L3; *] x L3^T (128 x 64; the lower 64
 //                            rows of the second A run on into the next chunk and their products are never read),
 //                            int32 accumulators in one of two sets of 256 tensor-memory columns
@@ -27,8 +31,10 @@
 // Hand-offs are mbarriers (producer -> MMA, tcgen05.commit -> producer / flush, flush -> MMA);
 // every wait is bounded: a wait that gives up raises an error flag, all roles leave their loops,
 // the distance matrix is filled with NaN and the control block's error word is set.
-#include <cstdlib>
-
+//
+// The last CTA also bounds what the rounding of the rows can have done to every distance (from the
+// coarsest grid each row was rounded to) and, if some pair's bound exceeds 1e-6 of its distance,
+// opens the gate of the difference-form kernel that the host has queued behind this one.
 #include "gar_internal.cuh"
 #include "mbar.cuh"
 
@@ -664,8 +670,7 @@ static cudaError_t launch_umma_layout(const float* grads, int n, int64_t d, int6
 
 cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
                                   int sm_count, cudaStream_t stream) {
-    static const char* env = std::getenv("GAR_KU_PACKED");      // experiment switch
-    if (n <= KU_PACK_ROWS && !(env && env[0] == '0')) return launch_umma_layout<true>(grads, n, d, ld, dist, ws, sm_count, stream);
+    if (n <= KU_PACK_ROWS) return launch_umma_layout<true>(grads, n, d, ld, dist, ws, sm_count, stream);
     return launch_umma_layout<false>(grads, n, d, ld, dist, ws, sm_count, stream);
 }
 

@@ -8,8 +8,8 @@
 namespace gar {
 
 // Suspended waits before a wait gives up.  One mbarrier.try_wait on a barrier that does not
-// complete returns after the hardware's own time limit (measured on B200 with
-// gar_selftest_bounded_wait: see the header); the product is the longest a kernel can be stuck.
+// complete returns after the hardware's own time limit, 4.0 microseconds on B200 (measured with
+// gar_selftest_bounded_wait); 2^20 of them bound the time a kernel can be stuck by 4.2 seconds.
 constexpr unsigned KB_SPIN_LIMIT = 1u << 20;
 
 __device__ __forceinline__ unsigned kb_smem_u32(const void* p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
