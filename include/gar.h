@@ -94,6 +94,12 @@ typedef enum {
 } gar_even_median_t;
 
 typedef enum {
+    GAR_F32  = 0, /* IEEE binary32 (the default everywhere)                                        */
+    GAR_BF16 = 1, /* bfloat16 gradients: every value is widened to fp32 exactly as it is loaded   */
+    GAR_F16  = 2  /* IEEE binary16 gradients, likewise; all arithmetic and the output stay fp32   */
+} gar_dtype_t;
+
+typedef enum {
     GAR_DISTANCES_AUTO       = 0, /* tensor-core Gram product where it applies, checked as described above */
     GAR_DISTANCES_DIFFERENCE = 1  /* always the fp32 difference form on the CUDA cores                     */
 } gar_distance_mode_t;
@@ -185,7 +191,11 @@ typedef struct {
     double*       dist_out;       /* optional dev [n*n]: the distance matrix */
     gar_selection_t* selection_out; /* optional dev: the selection result */
     int32_t       distance_mode;  /* gar_distance_mode_t */
-    int32_t       reserved;
+    int32_t       grads_dtype;    /* gar_dtype_t of `grads` (ld counts elements of that type).  16-bit
+                                     gradients halve the bytes both passes read (Section 2.1's workers may
+                                     well send 16-bit gradients); they are supported by gar_aggregate_ex
+                                     only, through the staged difference-form distance kernel for n <= 16,
+                                     the tiled one beyond, and the register coordinate kernel. */
     /* Optional SGD step fused into the coordinate kernel's store (Eq. 2: x <- x - lr * GAR(...);
        Section 5.1 trains with momentum 0.9): with g the aggregated coordinate,
            v <- sgd_momentum * v + g   (only if sgd_momentum_buf is given),   x <- x - sgd_lr * v   (or g)

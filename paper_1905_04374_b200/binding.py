@@ -16,6 +16,7 @@ GAR_MAX_N = 64
 RULES = {"average": 0, "median": 1, "krum": 2, "multi_krum": 3, "bulyan": 4, "multi_bulyan": 5}
 EVEN_MEDIAN = {"lower": 0, "mean": 1}
 DISTANCE_MODES = {"auto": 0, "difference": 1}
+GRAD_DTYPES = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 # gar_workspace control block, word 4: how the last distance call ran
 DISTANCE_PATHS = {0: "difference", 1: "gram", 2: "gram_rejected"}
 GAR_OK = 0
@@ -58,7 +59,7 @@ class GarParams(C.Structure):
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("m", C.c_int32), ("theta", C.c_int32), ("median_of_agr", C.c_int32), ("even_median", C.c_int32),
         ("dist_out", C.c_void_p), ("selection_out", C.c_void_p),
-        ("distance_mode", C.c_int32), ("reserved", C.c_int32),
+        ("distance_mode", C.c_int32), ("grads_dtype", C.c_int32),
         ("sgd_params", C.c_void_p), ("sgd_momentum_buf", C.c_void_p), ("sgd_lr", C.c_float), ("sgd_momentum", C.c_float),
     ]
 
@@ -188,8 +189,9 @@ def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None
     (uint8 CUDA tensor), options and outputs (dist_out float64 [n, n];
     selection_out uint8 CUDA tensor of sizeof(gar_selection_t)); optional fused SGD step on
     sgd_params / sgd_momentum_buf (CUDA float32 [d], updated in place); store_out=False with a
-    fused step passes out = NULL (returns None)."""
-    _dev_f32(grads, "grads")
+    fused step passes out = NULL (returns None).  grads may be float32, bfloat16 or float16."""
+    if not (grads.is_cuda and grads.dtype in GRAD_DTYPES):
+        raise TypeError("grads must be a CUDA float32, bfloat16 or float16 tensor")
     n, d, ld = _rows(grads)
     if out is None and (store_out or sgd_params is None):
         out = torch.empty(d, dtype=torch.float32, device=grads.device)
@@ -206,6 +208,7 @@ def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None
         p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
     p.m, p.theta, p.median_of_agr = m, theta, median_of_agr
     p.even_median, p.distance_mode = _even(even_median), _mode(distance_mode)
+    p.grads_dtype = GRAD_DTYPES[grads.dtype]
     if dist_out is not None:
         p.dist_out = dist_out.data_ptr()
     if selection_out is not None:

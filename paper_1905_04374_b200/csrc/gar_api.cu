@@ -103,20 +103,21 @@ bool overlaps(const void* a, size_t abytes, const void* b, size_t bbytes) {
 // Enqueue the whole rule for device buffers.
 int enqueue(int rule, const float* grads, int n, int f, int64_t d, int64_t ld, const gar::K3Out& out, int m, int theta,
             int median_of_agr, int even_median, int distance_mode, const Workspace& ws, double* dist_out,
-            gar_selection_t* sel_out, int sm_count, cudaStream_t stream) {
+            gar_selection_t* sel_out, int sm_count, cudaStream_t stream, int dtype = GAR_F32) {
     const int beta = beta_for(rule, theta, f);
     double* dist = dist_out ? dist_out : ws.dist();
     gar_selection_t* sel = sel_out ? sel_out : ws.selection();
     cudaError_t err;
     const bool needs_dist = !(rule == GAR_AVERAGE || rule == GAR_MEDIAN);
     if (needs_dist) {
-        err = gar::launch_distances(grads, n, d, ld, dist, ws, sm_count, distance_mode, stream);
+        err = dtype == GAR_F32 ? gar::launch_distances(grads, n, d, ld, dist, ws, sm_count, distance_mode, stream)
+                               : gar::launch_distances_16(grads, dtype, n, d, ld, dist, ws, sm_count, stream);
         if (err != cudaSuccess) return GAR_ERR_CUDA;
     }
     err = gar::launch_select(rule, dist, n, f, m, theta, beta, median_of_agr, even_median, sel, stream);
     if (err != cudaSuccess) return GAR_ERR_CUDA;
     const int preagg = (rule == GAR_MULTI_BULYAN || rule == GAR_MULTI_KRUM || rule == GAR_AVERAGE) ? 1 : 0;
-    err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg, out, sm_count, stream);
+    err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg, out, sm_count, stream, dtype);
     if (err != cudaSuccess) return GAR_ERR_CUDA;
     return GAR_OK;
 }
@@ -203,8 +204,10 @@ int gar_aggregate_ex(const gar_params_t* p) {
     if (p->sgd_momentum_buf && !p->sgd_params) return GAR_ERR_INVALID_ARG;
     const int64_t ld = p->ld ? p->ld : p->d;
     if (ld < p->d) return GAR_ERR_INVALID_ARG;
+    if (p->grads_dtype != GAR_F32 && p->grads_dtype != GAR_BF16 && p->grads_dtype != GAR_F16) return GAR_ERR_INVALID_ARG;
     {
-        const size_t gbytes = (size_t(p->n - 1) * ld + p->d) * sizeof(float), vbytes = size_t(p->d) * sizeof(float);
+        const size_t esize = p->grads_dtype == GAR_F32 ? sizeof(float) : 2;
+        const size_t gbytes = (size_t(p->n - 1) * ld + p->d) * esize, vbytes = size_t(p->d) * sizeof(float);
         const float* vecs[3] = {p->out, p->sgd_params, p->sgd_momentum_buf};
         for (int a = 0; a < 3; ++a) {
             if (!vecs[a]) continue;
@@ -233,7 +236,7 @@ int gar_aggregate_ex(const gar_params_t* p) {
     const gar::K3Out out{p->out, p->sgd_params, p->sgd_momentum_buf, p->sgd_lr, p->sgd_momentum};
     return enqueue(p->rule, p->grads, p->n, p->f, p->d, ld, out, m, theta, p->median_of_agr, p->even_median,
                    p->distance_mode, ws, p->dist_out, p->selection_out, st->sm_count,
-                   static_cast<cudaStream_t>(p->stream));
+                   static_cast<cudaStream_t>(p->stream), p->grads_dtype);
 }
 
 int gar_aggregate(int rule, const float* grads, int n, int f, int64_t d, float* out, void* stream) {

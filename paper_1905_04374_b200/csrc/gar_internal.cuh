@@ -56,11 +56,28 @@ struct K3Out {
     float  lr, mu;
 };
 
+// ---- 16-bit gradients ---------------------------------------------------------------------
+// One 16-bit element (bfloat16 or binary16, by `dtype`) widened to fp32, exactly.
+__device__ __forceinline__ float widen16(unsigned short raw, int dtype) {
+    if (dtype == GAR_BF16) return __uint_as_float(static_cast<unsigned>(raw) << 16);
+    float r;
+    asm("cvt.f32.f16 %0, %1;" : "=f"(r) : "h"(raw));
+    return r;
+}
+// Element `idx` of a gradient block whose elements are fp32 (dtype GAR_F32) or 16 bits wide.
+__device__ __forceinline__ float load_elem(const void* g, int64_t idx, int dtype) {
+    if (dtype == GAR_F32) return __ldg(static_cast<const float*>(g) + idx);
+    return widen16(__ldg(static_cast<const unsigned short*>(g) + idx), dtype);
+}
+
 // ---- kernel launchers (one per translation unit) --------------------------
 // Pairwise squared distances of n rows over columns [0, d); result in dist[n*n].
 // mode: a gar_distance_mode_t.
 cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, double* dist,
                              const Workspace& ws, int sm_count, int mode, cudaStream_t stream);
+// The same for 16-bit gradients (dtype GAR_BF16 or GAR_F16; grads points at 2-byte elements).
+cudaError_t launch_distances_16(const void* grads, int dtype, int n, int64_t d, int64_t ld, double* dist,
+                                const Workspace& ws, int sm_count, cudaStream_t stream);
 
 // Tensor-core variant (tcgen05, accumulators in tensor memory) for 16 < n <= 64 and 16-byte
 // aligned rows, used from kMmaMinDim coordinates on.
@@ -76,7 +93,7 @@ cudaError_t launch_schedule_only(gar_selection_t* sel, cudaStream_t stream);
 // Coordinate phase.
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
                               gar_selection_t* sel, int theta, int preagg, const K3Out& out,
-                              int sm_count, cudaStream_t stream);
+                              int sm_count, cudaStream_t stream, int dtype = GAR_F32);
 
 // One warp waits, bounded, on a barrier nobody arrives on; result[0] = status, result[1] = ns.
 cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t stream);

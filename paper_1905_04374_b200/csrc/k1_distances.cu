@@ -122,10 +122,11 @@ __device__ __forceinline__ void direct_pairs(const float (&x)[N][V], float (&acc
 }
 // One coordinate t of all rows straight from global memory (ragged ends).
 template <int N, int NPAD>
-__device__ __forceinline__ void direct_tail_coordinate(const float* __restrict__ g, int64_t ld, int64_t t, float (&acc)[NPAD]) {
+__device__ __forceinline__ void direct_tail_coordinate(const void* __restrict__ g, int64_t ld, int64_t t, float (&acc)[NPAD],
+                                                       int dtype = GAR_F32) {
     float x[N][1];
 #pragma unroll
-    for (int r = 0; r < N; ++r) x[r][0] = __ldg(g + int64_t(r) * ld + t);
+    for (int r = 0; r < N; ++r) x[r][0] = load_elem(g, int64_t(r) * ld + t, dtype);
     direct_pairs<N, 1, NPAD>(x, acc);
 }
 // The warp's fp32 accumulators -> its fp64 sums in shared memory (fixed shuffle tree), then zero.
@@ -273,15 +274,19 @@ constexpr int K1B_ROW_BYTES = K1B_TC * 4;
 constexpr int K1B_STAGES = 3;
 constexpr int K1B_BAR_COMPUTE = 1;
 
+// dtype: the gradients' element type (gar_dtype_t).  16-bit elements are staged as they are (a row of
+// a tile is then 2 KB instead of 4) and widened to fp32 when the compute threads read them.
 template <int N>
 __global__ void __launch_bounds__(K1B_THREADS)
-k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
+k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, double* __restrict__ dist,
                double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
                unsigned int* __restrict__ path_word) {
     constexpr int NP = N * (N - 1) / 2;
     constexpr int NPAD = (NP + 31) / 32 * 32;
     constexpr int WARPS = K1B_CT / 32;
-    constexpr unsigned STAGE_BYTES = unsigned(N) * K1B_ROW_BYTES;
+    const int esize = dtype == GAR_F32 ? 4 : 2;
+    const unsigned row_bytes = unsigned(K1B_TC) * unsigned(esize);
+    const unsigned STAGE_BYTES = unsigned(N) * row_bytes;
     extern __shared__ __align__(128) unsigned char stages[];          // [stage][row][K1B_TC floats]
     __shared__ double sums[WARPS][NPAD];
     __shared__ unsigned long long full[K1B_STAGES], empty[K1B_STAGES];
@@ -311,8 +316,8 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
             if (lane == 0) kb_expect_tx(bar, STAGE_BYTES);
             __syncwarp();
             if (lane < N)
-                kb_bulk_load(kb_smem_u32(stages) + unsigned(st) * STAGE_BYTES + unsigned(lane) * K1B_ROW_BYTES,
-                             g + int64_t(lane) * ld + (first + i * step) * K1B_TC, unsigned(K1B_ROW_BYTES), bar);
+                kb_bulk_load(kb_smem_u32(stages) + unsigned(st) * STAGE_BYTES + unsigned(lane) * row_bytes,
+                             static_cast<const char*>(g) + (int64_t(lane) * ld + (first + i * step) * K1B_TC) * esize, row_bytes, bar);
             if (++st == K1B_STAGES) { st = 0; parity ^= 1u; }
         }
         // no copy may be in flight when the CTA leaves: wait (bounded) for the last tiles issued
@@ -334,12 +339,24 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(failed) : "r"(*error), "r"(K1B_BAR_COMPUTE), "r"(K1B_CT) : "memory");
             if (failed) break;
-            const float4* src = reinterpret_cast<const float4*>(stages + size_t(st) * STAGE_BYTES) + tid;
             float x[N][4];
+            if (dtype == GAR_F32) {
+                const float4* src = reinterpret_cast<const float4*>(stages + size_t(st) * STAGE_BYTES) + tid;
 #pragma unroll
-            for (int r = 0; r < N; ++r) {
-                const float4 q = src[r * (K1B_TC / 4)];
-                x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w;
+                for (int r = 0; r < N; ++r) {
+                    const float4 q = src[r * (K1B_TC / 4)];
+                    x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w;
+                }
+            } else {
+                const uint2* src = reinterpret_cast<const uint2*>(stages + size_t(st) * STAGE_BYTES) + tid;
+#pragma unroll
+                for (int r = 0; r < N; ++r) {
+                    const uint2 q = src[r * (K1B_TC / 4)];
+                    x[r][0] = widen16(static_cast<unsigned short>(q.x & 0xffffu), dtype);
+                    x[r][1] = widen16(static_cast<unsigned short>(q.x >> 16), dtype);
+                    x[r][2] = widen16(static_cast<unsigned short>(q.y & 0xffffu), dtype);
+                    x[r][3] = widen16(static_cast<unsigned short>(q.y >> 16), dtype);
+                }
             }
             __syncwarp();                         // the rows are in registers: hand the stage back
             if (lane == 0) kb_arrive(&empty[st]);
@@ -349,7 +366,7 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
         }
         // coordinates after the last whole tile: CTA 0, plain loads
         if (blockIdx.x == 0) {
-            for (int64_t t = ntiles * K1B_TC + tid; t < d; t += K1B_CT) direct_tail_coordinate<N, NPAD>(g, ld, t, acc);
+            for (int64_t t = ntiles * K1B_TC + tid; t < d; t += K1B_CT) direct_tail_coordinate<N, NPAD>(g, ld, t, acc, dtype);
         }
         __syncwarp();
         flush();
@@ -391,6 +408,8 @@ k1_direct_bulk(const float* __restrict__ g, int64_t d, int64_t ld, double* __res
 template <int NB> struct K1Shape;
 // G = column groups per CTA, KQ = float4 passes of an off-diagonal lane per slab,
 // FLUSH = slabs between fp64 flushes, NSTAGE = depth of the shared-memory ring
+template <> struct K1Shape<1> { static constexpr int G = 4, KQ = 2, FLUSH = 8, NSTAGE = 3; };   // n <= 16: 16-bit gradients only
+template <> struct K1Shape<2> { static constexpr int G = 4, KQ = 2, FLUSH = 8, NSTAGE = 3; };
 template <> struct K1Shape<3> { static constexpr int G = 2, KQ = 2, FLUSH = 8, NSTAGE = 3; };
 template <> struct K1Shape<4> { static constexpr int G = 2, KQ = 2, FLUSH = 8, NSTAGE = 3; };
 template <> struct K1Shape<5> { static constexpr int G = 1, KQ = 2, FLUSH = 8, NSTAGE = 4; };
@@ -432,7 +451,7 @@ __device__ __forceinline__ void off_tile_blocks(int p, int nb, int& I, int& J) {
 // VEC path: 16-byte cp.async with zero fill past n rows / d columns.
 template <int NB, bool VEC>
 __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ g, int n, int64_t d,
-                                           int64_t ld, int64_t t0) {
+                                           int64_t ld, int64_t t0, int dtype = GAR_F32) {
     using D = K1Dims<NB>;
     if constexpr (VEC) {
         for (int idx = threadIdx.x; idx < D::R * D::TK4; idx += D::THREADS) {
@@ -447,7 +466,7 @@ __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ 
         for (int idx = threadIdx.x; idx < D::R * D::TK; idx += D::THREADS) {
             const int row = idx / D::TK, c = idx - row * D::TK;
             const int64_t col = t0 + c;
-            sm[size_t(row) * D::TK + c] = (row < n && col < d) ? __ldg(g + int64_t(row) * ld + col) : 0.0f;
+            sm[size_t(row) * D::TK + c] = (row < n && col < d) ? load_elem(g, int64_t(row) * ld + col, dtype) : 0.0f;   // widened here
         }
     }
 }
@@ -456,7 +475,7 @@ template <int NB, bool VEC>
 __global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
 k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
-         const unsigned int* __restrict__ gate) {
+         const unsigned int* __restrict__ gate, int dtype) {
     // launched behind the tensor-core kernel, this one only runs if that kernel rejected its own
     // result (the gate word is written before this grid starts: same stream)
     if (gate != nullptr && *gate == 0u) return;
@@ -530,7 +549,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
             cur = stage + size_t(it % NSTAGE) * D::R * D::TK;
         } else {
             __syncthreads();
-            stage_slab<NB, false>(stage, g, n, d, ld, (first + it * step) * D::TK);
+            stage_slab<NB, false>(stage, g, n, d, ld, (first + it * step) * D::TK, dtype);
             __syncthreads();
             cur = stage;
         }
@@ -665,7 +684,7 @@ cudaError_t persistent_grid(K kern, int threads, size_t smem, int sm_count, int*
 
 template <int NB, bool VEC>
 cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
-                         int sm_count, bool gated, cudaStream_t stream) {
+                         int sm_count, bool gated, cudaStream_t stream, int dtype = GAR_F32) {
     using D = K1Dims<NB>;
     static int per_sm_cache[64] = {0};
     int64_t grid = 1;
@@ -673,7 +692,7 @@ cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* d
                                       (d + D::TK - 1) / D::TK, &grid);
     if (err != cudaSuccess) return err;
     k1_tiled<NB, VEC><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket(),
-                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr);
+                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr, dtype);
     return cudaGetLastError();
 }
 
@@ -692,14 +711,14 @@ cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, c
 }
 
 template <int N>
-cudaError_t launch_direct_bulk(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
+cudaError_t launch_direct_bulk(const void* g, int dtype, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                                cudaStream_t stream) {
     static int per_sm_cache[64] = {0};
-    const size_t smem = size_t(K1B_STAGES) * N * K1B_ROW_BYTES;
+    const size_t smem = size_t(K1B_STAGES) * N * K1B_ROW_BYTES;      // sized for fp32 rows; 16-bit rows use half of it
     int64_t grid = 0;
     cudaError_t err = persistent_grid(k1_direct_bulk<N>, K1B_THREADS, smem, sm_count, per_sm_cache, d / K1B_TC, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct_bulk<N><<<unsigned(grid), K1B_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
+    k1_direct_bulk<N><<<unsigned(grid), K1B_THREADS, smem, stream>>>(g, dtype, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
                                                                      ws.k1_path());
     return cudaGetLastError();
 }
@@ -709,7 +728,7 @@ cudaError_t launch_direct_n(const float* g, int64_t d, int64_t ld, double* dist,
                             cudaStream_t stream, int vec) {
     // 16-byte aligned rows and enough whole tiles for every SM: rows staged by bulk copies
     if (vec >= 4 && d >= int64_t(sm_count) * K1B_TC)
-        return launch_direct_bulk<N>(g, d, ld, dist, ws, sm_count, stream);
+        return launch_direct_bulk<N>(g, GAR_F32, d, ld, dist, ws, sm_count, stream);
     // few rows: wide vectors keep enough bytes in flight; many rows: narrow ones keep the registers in check
     if constexpr (N <= 8) {
         if (vec >= 4) return launch_direct<N, 4>(g, d, ld, dist, ws, sm_count, stream);
@@ -754,6 +773,32 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
     }
 #undef GAR_K1_DIRECT
 #undef GAR_K1_TILED
+    return cudaErrorInvalidValue;
+}
+
+// 16-bit gradients (bfloat16 / binary16): the staged direct kernel for n <= 16 when the rows are
+// 16-byte aligned, else the tiled kernel's scalar staging path, which widens every element as it
+// stages it (any alignment, any n <= 64).  The arithmetic is the fp32 difference form throughout.
+cudaError_t launch_distances_16(const void* grads, int dtype, int n, int64_t d, int64_t ld, double* dist,
+                                const Workspace& ws, int sm_count, cudaStream_t stream) {
+    if (n == 1) return cudaMemsetAsync(dist, 0, sizeof(double), stream);
+    const uintptr_t addr = reinterpret_cast<uintptr_t>(grads);
+    if (n <= 16 && addr % 16 == 0 && ld % 8 == 0 && d >= int64_t(sm_count) * K1B_TC) {
+#define GAR_K1_BULK16(NV) case NV: return launch_direct_bulk<NV>(grads, dtype, d, ld, dist, ws, sm_count, stream);
+        switch (n) {
+            GAR_K1_BULK16(2) GAR_K1_BULK16(3) GAR_K1_BULK16(4) GAR_K1_BULK16(5) GAR_K1_BULK16(6) GAR_K1_BULK16(7)
+            GAR_K1_BULK16(8) GAR_K1_BULK16(9) GAR_K1_BULK16(10) GAR_K1_BULK16(11) GAR_K1_BULK16(12)
+            GAR_K1_BULK16(13) GAR_K1_BULK16(14) GAR_K1_BULK16(15) GAR_K1_BULK16(16)
+        }
+#undef GAR_K1_BULK16
+    }
+    const float* g = static_cast<const float*>(grads);       // only ever read through load_elem
+#define GAR_K1_TILED16(NBV) case NBV: return launch_tiled<NBV, false>(g, n, d, ld, dist, ws, sm_count, false, stream, dtype);
+    switch ((n + 7) / 8) {
+        GAR_K1_TILED16(1) GAR_K1_TILED16(2) GAR_K1_TILED16(3) GAR_K1_TILED16(4) GAR_K1_TILED16(5) GAR_K1_TILED16(6)
+        GAR_K1_TILED16(7) GAR_K1_TILED16(8)
+    }
+#undef GAR_K1_TILED16
     return cudaErrorInvalidValue;
 }
 

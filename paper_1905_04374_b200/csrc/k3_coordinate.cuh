@@ -91,6 +91,26 @@ __device__ __forceinline__ void k3_store_nan(const K3Out& o, int64_t t) {
     if (o.out) o.out[t] = CUDART_NAN_F;
 }
 
+// V consecutive gradient elements starting at element `idx` (naturally aligned for V elements),
+// widened to fp32: fp32 elements by default, 16-bit ones for dtype GAR_BF16 / GAR_F16.
+template <int V> __device__ __forceinline__ void load_grad(const float* g, int64_t idx, int dtype, float (&x)[V]) {
+    if (dtype == GAR_F32) { load_vec<V>(g + idx, x); return; }
+    const unsigned short* h = reinterpret_cast<const unsigned short*>(g) + idx;
+    if constexpr (V == 1) {
+        x[0] = widen16(__ldg(h), dtype);
+    } else if constexpr (V == 2) {
+        const unsigned u = __ldg(reinterpret_cast<const unsigned*>(h));
+        x[0] = widen16(static_cast<unsigned short>(u & 0xffffu), dtype);
+        x[1] = widen16(static_cast<unsigned short>(u >> 16), dtype);
+    } else {
+        const uint2 u = __ldg(reinterpret_cast<const uint2*>(h));
+        x[0] = widen16(static_cast<unsigned short>(u.x & 0xffffu), dtype);
+        x[1] = widen16(static_cast<unsigned short>(u.x >> 16), dtype);
+        x[2] = widen16(static_cast<unsigned short>(u.y & 0xffffu), dtype);
+        x[3] = widen16(static_cast<unsigned short>(u.y >> 16), dtype);
+    }
+}
+
 __device__ __forceinline__ void prefetch_l1(const void* p) {
     asm volatile("prefetch.global.L1 [%0];" ::"l"(p));
 }
@@ -348,7 +368,7 @@ __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* _
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(K3_THREADS)
 k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin, int64_t t_end, int64_t ld,
-              gar_selection_t* __restrict__ sel, const K3Out out, int loose_cap) {
+              gar_selection_t* __restrict__ sel, const K3Out out, int loose_cap, int dtype) {
     __shared__ K3Plan plan;
     extern __shared__ __align__(16) float k3_dyn[];
     const int status = k3_check(sel, n, theta_arg, PREAGG);
@@ -377,12 +397,12 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
     for (int64_t vi = int64_t(blockIdx.x) * nthreads + threadIdx.x; vi < nvec;
          vi += int64_t(gridDim.x) * nthreads) {
         const int64_t t = t_begin + vi * V;
-        const float* gt = g + t;
+        const int esh = dtype == GAR_F32 ? 2 : 1;             // log2 of the element size
         float e[P][V], a[P][V];
 #pragma unroll
         for (int s = 0; s < P; ++s) {
             if (s < theta) {
-                load_vec<V>(gt + plan.woff[s], e[s]);
+                load_grad<V>(g, t + plan.woff[s], dtype, e[s]);
             } else {
 #pragma unroll
                 for (int v = 0; v < V; ++v) e[s][v] = 0.0f;
@@ -392,15 +412,15 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
         // iteration's lines into L1 meanwhile (with many slots the extra instructions cost more)
         const int64_t vnext = vi + int64_t(gridDim.x) * nthreads;
         if (P <= 12 && vnext < nvec) {
-            const float* gn = g + t_begin + vnext * V;
+            const char* gn = reinterpret_cast<const char*>(g) + ((t_begin + vnext * V) << esh);
 #pragma unroll
             for (int s = 0; s < P; ++s) {
-                if (s < theta) prefetch_l1(gn + plan.woff[s]);
+                if (s < theta) prefetch_l1(gn + (plan.woff[s] << esh));
             }
             if constexpr (PREAGG) {
-                for (int k = 0; k < plan.nbase; ++k) prefetch_l1(gn + plan.boff[k]);
+                for (int k = 0; k < plan.nbase; ++k) prefetch_l1(gn + (plan.boff[k] << esh));
                 if (plan.loose_in_smem) {
-                    for (int k = 0; k < plan.nloose; ++k) prefetch_l1(gn + plan.loff[k]);
+                    for (int k = 0; k < plan.nloose; ++k) prefetch_l1(gn + (plan.loff[k] << esh));
                 }
             }
         }
@@ -416,7 +436,7 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
 #pragma unroll
                 for (int k = 0; k < 8; ++k) {
                     if (base + k < nbase) {
-                        load_vec<V>(gt + plan.boff[base + k], x[k]);
+                        load_grad<V>(g, t + plan.boff[base + k], dtype, x[k]);
                     } else {
 #pragma unroll
                         for (int v = 0; v < V; ++v) x[k][v] = 0.0f;
@@ -436,7 +456,7 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
                     float x[8][V];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
-                        if (base + k < nloose) load_vec<V>(gt + plan.loff[base + k], x[k]);
+                        if (base + k < nloose) load_grad<V>(g, t + plan.loff[base + k], dtype, x[k]);
                     }
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
@@ -464,7 +484,7 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
                             float x[V];
                             const int pos = plan.add_pos[kadd];
                             if (in_smem) read_vec<V>(xcol + size_t(pos) * stride, x);
-                            else load_vec<V>(gt + plan.loff[pos], x);
+                            else load_grad<V>(g, t + plan.loff[pos], dtype, x);
 #pragma unroll
                             for (int v = 0; v < V; ++v) C[v] += x[v];
                         }
@@ -499,7 +519,7 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
 
 template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
-                        int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream);
+                        int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream, int dtype);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 
 }  // namespace gar

@@ -13,23 +13,30 @@ namespace gar {
 
 template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
-                        int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream);
+                        int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream, int dtype);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 #define K3_DECL(P)                                                                                              \
     template <>                                                                                                 \
     cudaError_t launch_k3_p<P>(const float*, int, int64_t, int64_t, gar_selection_t*, int, int, int, int,       \
-                               const K3Out&, int, cudaStream_t);                                                    \
+                               const K3Out&, int, cudaStream_t, int);                                                    \
     template <> int bulk_ctas_for<P>(int, int, int);
 K3_P_LIST(K3_DECL)
 #undef K3_DECL
 
 cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, gar_selection_t* sel,
-                              int theta, int preagg, const K3Out& out, int sm_count, cudaStream_t stream) {
-    const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out.out) |
-                        reinterpret_cast<uintptr_t>(out.x) | reinterpret_cast<uintptr_t>(out.v);
+                              int theta, int preagg, const K3Out& out, int sm_count, cudaStream_t stream, int dtype) {
+    const uintptr_t o = reinterpret_cast<uintptr_t>(out.out) | reinterpret_cast<uintptr_t>(out.x) |
+                        reinterpret_cast<uintptr_t>(out.v);
+    const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | o;
     int vec_max = 1;                                      // what the alignment allows
-    if (a % 16 == 0 && ld % 4 == 0) vec_max = 4;
-    else if (a % 8 == 0 && ld % 2 == 0) vec_max = 2;
+    if (dtype == GAR_F32) {
+        if (a % 16 == 0 && ld % 4 == 0) vec_max = 4;
+        else if (a % 8 == 0 && ld % 2 == 0) vec_max = 2;
+    } else {                                              // V 16-bit elements per load, V floats per store
+        const uintptr_t ga = reinterpret_cast<uintptr_t>(grads);
+        if (ga % 8 == 0 && o % 16 == 0 && ld % 4 == 0) vec_max = 4;
+        else if (ga % 4 == 0 && o % 8 == 0 && ld % 2 == 0) vec_max = 2;
+    }
     // widest width that keeps the kernel's registers in check: large slot counts use narrower vectors
     int vec = vec_max;
     if (vec == 4 && theta > 8) vec = 2;
@@ -40,11 +47,12 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
     // memory and wins while the slot count is a compile-time constant, up to 32 slots.
     const int bulk_from = preagg ? 1 : 33;
     // (a few hundred thousand coordinates amortise its set-up: the plan, the barriers, the first tiles)
-    const bool bulk = vec_max == 4 && theta >= bulk_from && d >= 400000;
+    // (16-bit gradients go through the register kernel, which widens them as it loads)
+    const bool bulk = dtype == GAR_F32 && vec_max == 4 && theta >= bulk_from && d >= 400000;
 #define K3_TRY(P)                                                                                              \
     if (theta <= P) {                                                                                          \
         const int ctas = bulk ? bulk_ctas_for<P>(n, theta, preagg) : 0;                                        \
-        return launch_k3_p<P>(grads, n, d, ld, sel, theta, preagg, vec, ctas, out, sm_count, stream);          \
+        return launch_k3_p<P>(grads, n, d, ld, sel, theta, preagg, vec, ctas, out, sm_count, stream, dtype);   \
     }
     K3_P_LIST(K3_TRY)
 #undef K3_TRY

@@ -77,7 +77,7 @@ static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, gar_se
 // Coordinates [t0, d): t0 is a multiple of 4.
 template <int P, bool PREAGG, int V>
 static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, int64_t ld, gar_selection_t* sel, const K3Out& out,
-                       int sm_count, cudaStream_t stream) {
+                       int sm_count, cudaStream_t stream, int dtype) {
     constexpr bool EXACT = (K3_EXACT != 0);
     int threads = K3_THREADS, threads1 = K3_THREADS;
     size_t smem = 0, smem1 = 0;
@@ -109,17 +109,17 @@ static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, 
         const int64_t cap = int64_t(sm_count) * 8;
         if (blocks > cap) blocks = cap;
         k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, n, theta, t0, d_vec, ld, sel, out,
-                                                                                         loose_cap);
+                                                                                         loose_cap, dtype);
     }
     if (d_vec < d) {   // ragged tail (only when ld > d): scalar kernel on the last d % V coordinates
-        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap);
+        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap, dtype);
     }
     return cudaGetLastError();
 }
 
 template <>
 cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
-                              int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream) {
+                              int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream, int dtype) {
     int64_t t0 = 0;
     if (bulk_ctas > 0) {                         // whole tiles staged through shared memory, the rest below
         const cudaError_t err = preagg ? run_bulk<K3_P, true>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0)
@@ -131,13 +131,13 @@ cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_
     constexpr bool kWide = (K3_P <= 8);
     if (vec == 4 && !kWide) vec = 2;
     if (preagg) {
-        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
-        if (vec == 2) return run<K3_P, true, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
-        return run<K3_P, true, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
+        if constexpr (kWide) if (vec == 4) return run<K3_P, true, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
+        if (vec == 2) return run<K3_P, true, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
+        return run<K3_P, true, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
     }
-    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
-    if (vec == 2) return run<K3_P, false, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
-    return run<K3_P, false, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream);
+    if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
+    if (vec == 2) return run<K3_P, false, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
+    return run<K3_P, false, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
 }
 
 // CTAs per SM the staged kernel would get for n gradients and theta slots (0: it cannot run).

@@ -106,6 +106,9 @@ def test_errors_before_any_launch(pkg):
     assert L.gar_aggregate_ex(C.byref(p)) == 1
     p.even_median, p.distance_mode = 0, 7                                  # unknown distance mode
     assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.distance_mode, p.grads_dtype = 0, 3                                  # unknown element type
+    assert L.gar_aggregate_ex(C.byref(p)) == 1
+    p.grads_dtype = 0
     p.distance_mode = 0
     p.out, p.sgd_params = None, None                                       # neither an output nor a fused step
     assert L.gar_aggregate_ex(C.byref(p)) == 1

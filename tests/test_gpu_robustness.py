@@ -342,3 +342,55 @@ def test_fused_sgd_leaves_the_model_alone_on_failure(pkg):
     # for the plain output, which is what decides whether x is touched
     out = pkg.gar_coordinate_phase(G, sel, pkg.gar_theta("multi_bulyan", n, f), 1)
     assert bool(torch.isnan(out).all())
+
+
+# ------------------------------------------------------------ 16-bit gradient inputs
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("cfg,d", [(5, 4099), (5, 450_048), (5, 450_051), (2, 70_001), (3, 262_148), (1, 200_003)])
+def test_sixteen_bit_gradients(pkg, dtype, cfg, d):
+    """bfloat16 / binary16 gradients: every value is widened to fp32 exactly when it is loaded, so
+    the oracle, fed the same 16-bit values promoted to fp64, is the reference at the usual bars
+    (distances 1e-6 relative, outputs 1e-5 (1 + |oracle|), selection where the gap is clear)."""
+    wl = pkg.workloads.WORKLOADS[cfg]
+    n, f = wl.n, wl.f
+    G32, _ = pkg.workloads.make_gradients(cfg, d=d, device=DEV)
+    G = G32.to(dtype)
+    Gh = G.to(torch.float32).cpu().numpy()            # exact: both formats embed in fp32
+    for rule in ("multi_bulyan", "bulyan", "median", "average"):
+        sel_dev = pkg.new_selection(DEV)
+        dist = torch.empty(n, n, dtype=torch.float64, device=DEV)
+        out = pkg.gar_aggregate_ex(rule, G, f, dist_out=dist, selection_out=sel_dev).cpu().numpy()
+        want, tab = rule_tables(rule, Gh, f)
+        if tab is None:
+            assert_outputs_match(out, want)
+            continue
+        D = dist.cpu().numpy()
+        wantD = O.pairwise_sq_distances(Gh)
+        pos = wantD > 0
+        assert np.max(np.abs(D - wantD)[pos] / wantD[pos]) <= 1e-6 and np.all(D[~pos] == 0)
+        sel = pkg.read_selection(sel_dev)
+        assert sel.status == 0
+        preagg = rule == "multi_bulyan"
+        compared = assert_selection_match(sel, tab["rounds"], preagg)
+        # 16-bit values collide often (8 or 11 significant bits): exact ties between |a - M| values are
+        # a hundred times more frequent than with fp32 inputs; every one is still checked against
+        # the averages its tie admits
+        if compared == len(tab["rounds"]):
+            assert_outputs_match(out, want, G=Gh, tables=tab, max_tie_frac=1e-2)
+        else:
+            winners = [sel.winners[r] for r in range(sel.theta)]
+            sets = [[i for i in range(n) if (sel.sets[r] >> i) & 1] for r in range(sel.theta)] if preagg else None
+            want2, gap2 = O.coordinate_phase(Gh, winners, sets, sel.beta)
+            assert_outputs_match(out, want2, G=Gh, tables=dict(winners=winners, sets=sets, beta=sel.beta, gap=gap2),
+                                 max_tie_frac=1e-2)
+
+
+def test_sixteen_bit_strided_views(pkg):
+    n, f, d = 15, 3, 33_333
+    big, _ = pkg.workloads.make_gradients(5, d=d + 11, device=DEV)
+    big = big.to(torch.bfloat16)
+    for view in (big[:, :d], big[:, 1:d + 1], big[:, 2:d + 2], big[:, 8:d + 8]):
+        vh = view.to(torch.float32).cpu().numpy()
+        out = pkg.gar_aggregate_ex("multi_bulyan", view, f).cpu().numpy()
+        want, tab = rule_tables("multi_bulyan", vh, f)
+        assert_outputs_match(out, want, G=vh, tables=tab, max_tie_frac=1e-2)
