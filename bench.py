@@ -202,7 +202,8 @@ def launches_per_aggregation(n: int, d: int, theta: int) -> int:
     return k1 + 1 + k3
 
 
-def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant=True, distance_mode="auto"):
+def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant=True, distance_mode="auto",
+                     dtype="f32"):
     """Device-side measurement of one workload resident in HBM: `steps` whole aggregations timed
     with CUDA events on the launch stream (max over ranks), then each stage alone."""
     import torch
@@ -215,6 +216,32 @@ def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant
     G, _ = pkg.workloads.make_gradients(cfg, d=d, device=dev)
     out = torch.empty(d, dtype=torch.float32, device=dev)
     stream = torch.cuda.current_stream()
+    if dtype != "f32":
+        # 16-bit gradients: the same draw rounded to bfloat16 / binary16; only the whole call is timed
+        # (the stage calls of the C ABI take fp32 gradients)
+        G16 = torch.empty(n, d, dtype=torch.bfloat16 if dtype == "bf16" else torch.float16, device=dev)
+        for c0 in range(0, d, 1 << 24):
+            G16[:, c0:c0 + (1 << 24)] = G[:, c0:c0 + (1 << 24)]
+        del G
+        torch.cuda.empty_cache()
+        for _ in range(max(warmup, 3)):
+            pkg.gar_aggregate_ex("multi_bulyan", G16, f, out=out)
+        torch.cuda.synchronize()
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with ClockSampler(physical_gpu_index(local), period=0.002) as clocks:
+            start.record(stream)
+            for _ in range(steps):
+                pkg.gar_aggregate_ex("multi_bulyan", G16, f, out=out)
+            stop.record(stream)
+            torch.cuda.synchronize()
+        ms = start.elapsed_time(stop) / steps
+        peak, _ = measured_hbm_peak()
+        bytes16 = 2.0 * d * (n + theta_b) + 4.0 * d
+        return {"workload": f"{wl.name} recipe at d={d}, {dtype} gradients", "n": n, "f": f, "d": d, "theta": theta_a,
+                "ms_per_aggregation": ms, "aggregations_per_sec": 1e3 / ms, "steps": steps, "kernels": {},
+                "roofline": None, "path": {"bytes_min_16bit_rows": bytes16, "effective_gbs": bytes16 / (ms * 1e-3) / 1e9,
+                                           "frac_of_measured_peak": bytes16 / (ms * 1e-3) / 1e9 / peak},
+                "clocks": clocks.summary(), "elapsed_ms": ms * steps}, G16
 
     def step():
         if distance_mode == "auto":
@@ -431,7 +458,7 @@ def run_ours(args):
         dist.destroy_process_group()
         return
     main, G = measure_workload(pkg, cfg, dev, args.steps, args.warmup, world, local, d=args.d,
-                               distance_mode=args.distance_mode)
+                               distance_mode=args.distance_mode, dtype=args.dtype)
     wl = pkg.workloads.WORKLOADS[cfg]
     n, f, d = main["n"], main["f"], main["d"]
     if rank != 0:
@@ -474,6 +501,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": main["workload"], "n": n, "f": f, "d": d, "rule": "multi_bulyan", "theta": main["theta"],
                    "beta": pkg.gar_beta("multi_bulyan", n, f), "parallelism": f"replicas x{world}",
+                   "grads_dtype": args.dtype,
                    "why_this_workload": "the largest of the five configurations; it fits one GPU (60 GB of 180)",
                    "l2": "input (%.2f GB) larger than L2; no flush" % (4e-9 * n * d) if 4 * n * d > 2.6e8
                    else "input fits L2; not flushed between steps"},
@@ -504,9 +532,13 @@ def main():
     ap.add_argument("--quick", action="store_true", help="device-side numbers of the chosen workload only")
     ap.add_argument("--distance-mode", default="auto", choices=["auto", "difference"],
                     help="difference: the fp32 difference-form distance kernels instead of the tensor-core one")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16", "f16"],
+                    help="element type of the gradients (16-bit: whole-call timing only, implies --quick)")
     ap.add_argument("--force-sharded", action="store_true",
                     help="run the sharded (N > 1) code path even with one rank (under torchrun, for checking it)")
     args = ap.parse_args()
+    if args.dtype != "f32":
+        args.quick = True
     if args.quick:
         args.no_e2e = args.no_cpu_baseline = args.no_per_config = True
     if args.impl == "reference":

@@ -192,10 +192,10 @@ typedef struct {
     gar_selection_t* selection_out; /* optional dev: the selection result */
     int32_t       distance_mode;  /* gar_distance_mode_t */
     int32_t       grads_dtype;    /* gar_dtype_t of `grads` (ld counts elements of that type).  16-bit
-                                     gradients halve the bytes both passes read (Section 2.1's workers may
-                                     well send 16-bit gradients); they are supported by gar_aggregate_ex
-                                     only, through the staged difference-form distance kernel for n <= 16,
-                                     the tiled one beyond, and the register coordinate kernel. */
+                                     gradients halve the bytes both passes read; every value is widened to
+                                     fp32 exactly where it is loaded, all arithmetic and the output stay
+                                     fp32.  Supported by gar_aggregate_ex only (the stage calls take fp32).
+                                     The staged kernels need 16-byte aligned rows (ld a multiple of 8). */
     /* Optional SGD step fused into the coordinate kernel's store (Eq. 2: x <- x - lr * GAR(...);
        Section 5.1 trains with momentum 0.9): with g the aggregated coordinate,
            v <- sgd_momentum * v + g   (only if sgd_momentum_buf is given),   x <- x - sgd_lr * v   (or g)

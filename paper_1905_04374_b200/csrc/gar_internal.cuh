@@ -83,7 +83,7 @@ cudaError_t launch_distances_16(const void* grads, int dtype, int n, int64_t d, 
 // aligned rows, used from kMmaMinDim coordinates on.
 constexpr int64_t kMmaMinDim = 32768;
 cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist,
-                                  const Workspace& ws, int sm_count, cudaStream_t stream);
+                                  const Workspace& ws, int sm_count, cudaStream_t stream, int dtype = GAR_F32);
 
 // Scoring + iterative selection (and schedule construction) into *sel.
 cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,

@@ -449,18 +449,23 @@ __device__ __forceinline__ void off_tile_blocks(int p, int nb, int& I, int& J) {
 
 // Stage one slab (all R rows, TK columns from t0) into shared memory.
 // VEC path: 16-byte cp.async with zero fill past n rows / d columns.
-template <int NB, bool VEC>
+// ES: bytes per staged element.  4: fp32 (VEC or scalar path; the scalar path widens 16-bit
+// elements as it stages them).  2 (VEC only): 16-bit elements staged as they are, 8 per 16-byte copy,
+// and widened when the compute loop reads them.
+template <int NB, bool VEC, int ES = 4>
 __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ g, int n, int64_t d,
                                            int64_t ld, int64_t t0, int dtype = GAR_F32) {
     using D = K1Dims<NB>;
     if constexpr (VEC) {
-        for (int idx = threadIdx.x; idx < D::R * D::TK4; idx += D::THREADS) {
-            const int row = idx / D::TK4, c4 = idx - row * D::TK4;
-            const int64_t col = t0 + 4 * int64_t(c4);
+        constexpr int EPC = 16 / ES;                      // elements per 16-byte copy
+        constexpr int CPR = D::TK / EPC;                  // copies per row
+        for (int idx = threadIdx.x; idx < D::R * CPR; idx += D::THREADS) {
+            const int row = idx / CPR, cc = idx - row * CPR;
+            const int64_t col = t0 + EPC * int64_t(cc);
             const int64_t left = d - col;                 // valid coordinates from col
-            const int bytes = (row < n && left > 0) ? (left >= 4 ? 16 : int(left) * 4) : 0;
-            const float* src = bytes ? g + int64_t(row) * ld + col : g;
-            cp_async16(sm + size_t(row) * D::TK + 4 * c4, src, bytes);
+            const int bytes = (row < n && left > 0) ? (left >= EPC ? 16 : int(left) * ES) : 0;
+            const char* src = bytes ? reinterpret_cast<const char*>(g) + (int64_t(row) * ld + col) * ES : reinterpret_cast<const char*>(g);
+            cp_async16(reinterpret_cast<char*>(sm) + (size_t(row) * D::TK + EPC * cc) * ES, src, bytes);
         }
     } else {
         for (int idx = threadIdx.x; idx < D::R * D::TK; idx += D::THREADS) {
@@ -471,7 +476,18 @@ __device__ __forceinline__ void stage_slab(float* sm, const float* __restrict__ 
     }
 }
 
-template <int NB, bool VEC>
+// Four staged columns (index in units of four columns) as fp32.
+template <int ES> __device__ __forceinline__ float4 tile_ld4(const float* tile, int idx4, int dtype) {
+    if constexpr (ES == 4) {
+        return reinterpret_cast<const float4*>(tile)[idx4];
+    } else {
+        const uint2 u = reinterpret_cast<const uint2*>(tile)[idx4];
+        return make_float4(widen16(static_cast<unsigned short>(u.x & 0xffffu), dtype), widen16(static_cast<unsigned short>(u.x >> 16), dtype),
+                           widen16(static_cast<unsigned short>(u.y & 0xffffu), dtype), widen16(static_cast<unsigned short>(u.y >> 16), dtype));
+    }
+}
+
+template <int NB, bool VEC, int ES = 4>
 __global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
 k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
@@ -531,7 +547,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
 
     if constexpr (VEC) {
         for (int s = 0; s < NSTAGE - 1; ++s) {
-            if (s < mine) stage_slab<NB, true>(stage + size_t(s) * D::R * D::TK, g, n, d, ld, (first + s * step) * D::TK);
+            if (s < mine) stage_slab<NB, true, ES>(stage + size_t(s) * D::R * D::TK, g, n, d, ld, (first + s * step) * D::TK);
             cp_async_commit();
         }
     }
@@ -544,7 +560,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
             __syncthreads();
             const int64_t nxt = it + NSTAGE - 1;
             if (nxt < mine)
-                stage_slab<NB, true>(stage + size_t(nxt % NSTAGE) * D::R * D::TK, g, n, d, ld, (first + nxt * step) * D::TK);
+                stage_slab<NB, true, ES>(stage + size_t(nxt % NSTAGE) * D::R * D::TK, g, n, d, ld, (first + nxt * step) * D::TK);
             cp_async_commit();
             cur = stage + size_t(it % NSTAGE) * D::R * D::TK;
         } else {
@@ -553,18 +569,16 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
             __syncthreads();
             cur = stage;
         }
-        const float4* s4 = reinterpret_cast<const float4*>(cur) + grp * D::GQ;
+        const int pa = grp * D::GQ + (I * 8) * D::TK4 + c, pb = grp * D::GQ + (J * 8) * D::TK4 + c;   // in units of four columns
         if (off_warp) {
-            const float4* pa = s4 + (I * 8) * D::TK4 + c;
-            const float4* pb = s4 + (J * 8) * D::TK4 + c;
 #pragma unroll 1
             for (int k = 0; k < D::KQ; ++k) {          // rolled: the body is ~530 instructions already
                 float4 a[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) a[i] = pa[i * D::TK4 + k * 16];
+                for (int i = 0; i < 8; ++i) a[i] = tile_ld4<ES>(cur, pa + i * D::TK4 + k * 16, dtype);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const float4 b = pb[j * D::TK4 + k * 16];
+                    const float4 b = tile_ld4<ES>(cur, pb + j * D::TK4 + k * 16, dtype);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float dx = a[i].x - b.x, dy = a[i].y - b.y, dz = a[i].z - b.z, dw = a[i].w - b.w;
@@ -576,13 +590,11 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
             }
         } else {
             // two diagonal tiles: pairs i < j of tile I at acc[i*8+j], of tile J at acc[j*8+i]
-            const float4* pa = s4 + (I * 8) * D::TK4 + c;
-            const float4* pb = s4 + (J * 8) * D::TK4 + c;
 #pragma unroll 1
             for (int k = 0; k < D::KQ; ++k) {
                 float4 a[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) a[i] = pa[i * D::TK4 + k * 16];
+                for (int i = 0; i < 8; ++i) a[i] = tile_ld4<ES>(cur, pa + i * D::TK4 + k * 16, dtype);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
 #pragma unroll
@@ -594,7 +606,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
                     }
                 }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) a[i] = pb[i * D::TK4 + k * 16];
+                for (int i = 0; i < 8; ++i) a[i] = tile_ld4<ES>(cur, pb + i * D::TK4 + k * 16, dtype);
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
 #pragma unroll
@@ -682,16 +694,16 @@ cudaError_t persistent_grid(K kern, int threads, size_t smem, int sm_count, int*
     return cudaSuccess;
 }
 
-template <int NB, bool VEC>
+template <int NB, bool VEC, int ES = 4>
 cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
                          int sm_count, bool gated, cudaStream_t stream, int dtype = GAR_F32) {
     using D = K1Dims<NB>;
     static int per_sm_cache[64] = {0};
     int64_t grid = 1;
-    cudaError_t err = persistent_grid(k1_tiled<NB, VEC>, D::THREADS, D::SMEM_BYTES, sm_count, per_sm_cache,
+    cudaError_t err = persistent_grid(k1_tiled<NB, VEC, ES>, D::THREADS, D::SMEM_BYTES, sm_count, per_sm_cache,
                                       (d + D::TK - 1) / D::TK, &grid);
     if (err != cudaSuccess) return err;
-    k1_tiled<NB, VEC><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket(),
+    k1_tiled<NB, VEC, ES><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket(),
                                                                           ws.k1_path(), gated ? ws.k1_gate() : nullptr, dtype);
     return cudaGetLastError();
 }
@@ -777,8 +789,8 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
 }
 
 // 16-bit gradients (bfloat16 / binary16): the staged direct kernel for n <= 16 when the rows are
-// 16-byte aligned, else the tiled kernel's scalar staging path, which widens every element as it
-// stages it (any alignment, any n <= 64).  The arithmetic is the fp32 difference form throughout.
+// 16-byte aligned and d is large; else the tiled kernel, staging the raw 16-bit slabs by 16-byte
+// copies (aligned rows) or element by element (any alignment), any n <= 64.  The arithmetic is the fp32 difference form throughout.
 cudaError_t launch_distances_16(const void* grads, int dtype, int n, int64_t d, int64_t ld, double* dist,
                                 const Workspace& ws, int sm_count, cudaStream_t stream) {
     if (n == 1) return cudaMemsetAsync(dist, 0, sizeof(double), stream);
@@ -792,8 +804,20 @@ cudaError_t launch_distances_16(const void* grads, int dtype, int n, int64_t d, 
         }
 #undef GAR_K1_BULK16
     }
-    const float* g = static_cast<const float*>(grads);       // only ever read through load_elem
-#define GAR_K1_TILED16(NBV) case NBV: return launch_tiled<NBV, false>(g, n, d, ld, dist, ws, sm_count, false, stream, dtype);
+    const float* g = static_cast<const float*>(grads);       // only ever read as 16-bit elements
+    const bool vec16 = addr % 16 == 0 && ld % 8 == 0;         // rows staged raw by 16-byte copies, else element by element
+    // many rows, a long dimension, aligned rows: the tensor-core kernel (its producers widen the
+    // values before they quantise them), with the tiled kernel behind its gate as for fp32
+    bool gated = false;
+    if (n > 16 && vec16 && d >= kMmaMinDim) {
+        const cudaError_t err = launch_distances_umma(g, n, d, ld, dist, ws, sm_count, stream, dtype);
+        if (err != cudaSuccess) return err;
+        gated = true;
+    }
+#define GAR_K1_TILED16(NBV)                                                                                        \
+    case NBV:                                                                                                      \
+        return vec16 ? launch_tiled<NBV, true, 2>(g, n, d, ld, dist, ws, sm_count, gated, stream, dtype)            \
+                     : launch_tiled<NBV, false>(g, n, d, ld, dist, ws, sm_count, gated, stream, dtype);
     switch ((n + 7) / 8) {
         GAR_K1_TILED16(1) GAR_K1_TILED16(2) GAR_K1_TILED16(3) GAR_K1_TILED16(4) GAR_K1_TILED16(5) GAR_K1_TILED16(6)
         GAR_K1_TILED16(7) GAR_K1_TILED16(8)

@@ -158,9 +158,11 @@ __device__ __forceinline__ int tri_slot(int i, int j) { return i * 64 - (i * (i 
 // Shared memory: KUSmem, the byte-tile buffers, px and pz (2 x 64 x 64 doubles, stored transposed:
 // [j][i]), the raw ring float4 [NST][3 * producer warps][32].
 // FULL: n is a multiple of KU_JR, every producer warp owns KU_JR real rows (no per-row tests).
-template <int NST, int MAXT, bool FULL, bool PACKED>
+// H16: the gradients are 16-bit (bfloat16 or binary16 by `dtype`): a lane fetches 8 bytes per row and
+// slab instead of 16 and widens its four values before it quantises them; everything after is the same.
+template <int NST, int MAXT, bool FULL, bool PACKED, bool H16>
 __global__ void __launch_bounds__(MAXT, 1)
-k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
+k1_umma(const float* __restrict__ g, int dtype, int n, int64_t d, int64_t ld, double* __restrict__ dist,
         double* __restrict__ partials, unsigned int* __restrict__ ticket,
         unsigned int* __restrict__ error_word, unsigned int* __restrict__ path_word,
         unsigned int* __restrict__ gate_word) {
@@ -228,7 +230,8 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
         int row_exp[KU_JR];
         float scale[KU_JR];                            // 2^(148 - row_exp)
         int exp_stores = 0;                            // tile buffers that still lack the rows' current exponents
-        const float* nextp[KU_JR];                     // this lane's float4 of the next slab to request
+        constexpr int ES = H16 ? 2 : 4;                // bytes per gradient element
+        const char* nextp[KU_JR];                      // this lane's four columns of the next slab to request
         bool valid[KU_JR];
         unsigned tile_off[KU_JR];                      // byte offset of (row, this lane's 4 columns) in a tile buffer
 #pragma unroll
@@ -237,25 +240,29 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
             valid[jr] = FULL || row < n;
             row_exp[jr] = KU_MIN_EXP;
             scale[jr] = __uint_as_float(unsigned(275 - KU_MIN_EXP) << 23);
-            nextp[jr] = g + int64_t(valid[jr] ? row : 0) * ld + first * KU_SLAB + 4 * lane;
+            nextp[jr] = reinterpret_cast<const char*>(g) + (int64_t(valid[jr] ? row : 0) * ld + first * KU_SLAB + 4 * lane) * ES;
             tile_off[jr] = unsigned(lane >> 2) * KU_LBO + unsigned(lane & 3) * 4 + unsigned(row) * 16;
         }
-        const int64_t advance = step * KU_SLAB;                                    // floats between this CTA's slabs
+        const int64_t advance = step * KU_SLAB * ES;                               // bytes between this CTA's slabs
         const unsigned stage_bytes = unsigned(ring_rows) * 512u, row_stride = unsigned(pw) * 512u;
         const unsigned my_ring = smem_u32(ring) + unsigned(p * 32 + lane) * 16u;   // (stage 0, row p, this lane)
         const unsigned limb_u32 = smem_u32(limb);
         // the last slab of the matrix may be ragged: bytes of this lane's float4 that exist there
         const int64_t last_left = d - (nslabs - 1) * KU_SLAB - 4 * lane;
-        const int last_bytes = last_left >= 4 ? 16 : (last_left > 0 ? int(last_left) * 4 : 0);
+        const int last_bytes = last_left >= 4 ? 4 * ES : (last_left > 0 ? int(last_left) * ES : 0);
         const int last_it = (first + (mine - 1) * step == nslabs - 1) ? int(mine - 1) : -1;   // this CTA's iteration of it
         auto request = [&](unsigned stage_off, int it_req) {
-            const int bytes = it_req == last_it ? last_bytes : 16;
+            const int bytes = it_req == last_it ? last_bytes : 4 * ES;
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
                 if (valid[jr]) {
-                    const float* src = bytes ? nextp[jr] : g;                        // nothing is read when bytes == 0
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n"
-                                 ::"r"(my_ring + stage_off + unsigned(jr) * row_stride), "l"(src), "r"(bytes) : "memory");
+                    const char* src = bytes ? nextp[jr] : reinterpret_cast<const char*>(g);   // nothing is read when bytes == 0
+                    if constexpr (H16)
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;\n"
+                                     ::"r"(my_ring + stage_off + unsigned(jr) * row_stride), "l"(src), "r"(bytes) : "memory");
+                    else
+                        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n"
+                                     ::"r"(my_ring + stage_off + unsigned(jr) * row_stride), "l"(src), "r"(bytes) : "memory");
                     nextp[jr] += advance;
                 }
             }
@@ -281,10 +288,19 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
 #pragma unroll
             for (int jr = 0; jr < KU_JR; ++jr) {
                 v[jr] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (valid[jr])
-                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                 : "=f"(v[jr].x), "=f"(v[jr].y), "=f"(v[jr].z), "=f"(v[jr].w)
-                                 : "r"(my_ring + cur_off + unsigned(jr) * row_stride) : "memory");
+                if (valid[jr]) {
+                    if constexpr (H16) {
+                        unsigned lo, hi;
+                        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(lo), "=r"(hi)
+                                     : "r"(my_ring + cur_off + unsigned(jr) * row_stride) : "memory");
+                        v[jr] = make_float4(widen16(static_cast<unsigned short>(lo & 0xffffu), dtype), widen16(static_cast<unsigned short>(lo >> 16), dtype),
+                                            widen16(static_cast<unsigned short>(hi & 0xffffu), dtype), widen16(static_cast<unsigned short>(hi >> 16), dtype));
+                    } else {
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(v[jr].x), "=f"(v[jr].y), "=f"(v[jr].z), "=f"(v[jr].w)
+                                     : "r"(my_ring + cur_off + unsigned(jr) * row_stride) : "memory");
+                    }
+                }
             }
             cur_off += stage_bytes;
             if (cur_off == unsigned(NST) * stage_bytes) cur_off = 0;
@@ -615,15 +631,15 @@ k1_umma(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __res
     }
 }
 
-template <int NST, int MAXT, bool FULL, bool PACKED>
-cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
+template <int NST, int MAXT, bool FULL, bool PACKED, bool H16>
+cudaError_t launch_ku(const float* g, int dtype, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                       int pw, size_t smem, cudaStream_t stream) {
     static size_t configured[64] = {0};                        // dynamic shared memory the kernel is allowed, per device
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64 || configured[dev] < smem) {
-        err = cudaFuncSetAttribute(k1_umma<NST, MAXT, FULL, PACKED>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        err = cudaFuncSetAttribute(k1_umma<NST, MAXT, FULL, PACKED, H16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = smem;
     }
@@ -633,16 +649,16 @@ cudaError_t launch_ku(const float* g, int n, int64_t d, int64_t ld, double* dist
     int64_t grid = sm_count;
     if (grid > kMaxCtasK1) grid = kMaxCtasK1;
     if (grid > nslabs) grid = nslabs;
-    k1_umma<NST, MAXT, FULL, PACKED><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
-        g, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(), ws.k1_path(), ws.k1_gate());
+    k1_umma<NST, MAXT, FULL, PACKED, H16><<<unsigned(grid), 32 * (KU_FIRST_PRODUCER + pw), smem, stream>>>(
+        g, dtype, n, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(), ws.k1_path(), ws.k1_gate());
     return cudaGetLastError();
 }
 
 }  // namespace
 
 // 16 < n <= 64, grads 16-byte aligned, ld % 4 == 0.
-template <bool PACKED>
-static cudaError_t launch_umma_layout(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
+template <bool PACKED, bool H16>
+static cudaError_t launch_umma_layout(const float* grads, int dtype, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
                                       int sm_count, cudaStream_t stream) {
     using S = KUShape<PACKED>;
     const int pw = (n + KU_JR - 1) / KU_JR;                    // producer warps: three rows each
@@ -655,8 +671,8 @@ static cudaError_t launch_umma_layout(const float* grads, int n, int64_t d, int6
     const size_t smem = fixed + nst * stage;
 #define GAR_KU(NSTV, MAXTV)                                                                                           \
     do {                                                                                                              \
-        if (n == KU_JR * pw) return launch_ku<NSTV, MAXTV, true, PACKED>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream); \
-        return launch_ku<NSTV, MAXTV, false, PACKED>(grads, n, d, ld, dist, ws, sm_count, pw, smem, stream);           \
+        if (n == KU_JR * pw) return launch_ku<NSTV, MAXTV, true, PACKED, H16>(grads, dtype, n, d, ld, dist, ws, sm_count, pw, smem, stream); \
+        return launch_ku<NSTV, MAXTV, false, PACKED, H16>(grads, dtype, n, d, ld, dist, ws, sm_count, pw, smem, stream);           \
     } while (0)
     if (pw <= 14) { if (nst == 4) GAR_KU(4, kSmall); if (nst == 3) GAR_KU(3, kSmall); GAR_KU(2, kSmall); }
     if constexpr (!PACKED) {
@@ -669,9 +685,13 @@ static cudaError_t launch_umma_layout(const float* grads, int n, int64_t d, int6
 }
 
 cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t ld, double* dist, const Workspace& ws,
-                                  int sm_count, cudaStream_t stream) {
-    if (n <= KU_PACK_ROWS) return launch_umma_layout<true>(grads, n, d, ld, dist, ws, sm_count, stream);
-    return launch_umma_layout<false>(grads, n, d, ld, dist, ws, sm_count, stream);
+                                  int sm_count, cudaStream_t stream, int dtype) {
+    if (dtype == GAR_F32) {
+        if (n <= KU_PACK_ROWS) return launch_umma_layout<true, false>(grads, dtype, n, d, ld, dist, ws, sm_count, stream);
+        return launch_umma_layout<false, false>(grads, dtype, n, d, ld, dist, ws, sm_count, stream);
+    }
+    if (n <= KU_PACK_ROWS) return launch_umma_layout<true, true>(grads, dtype, n, d, ld, dist, ws, sm_count, stream);
+    return launch_umma_layout<false, true>(grads, dtype, n, d, ld, dist, ws, sm_count, stream);
 }
 
 }  // namespace gar

@@ -60,12 +60,36 @@ struct KBPlan {
 
 // Dynamic shared memory: [staged-row indices of the plan's additions, 16-byte padded]
 // [correction columns (ncorr + 1) x TC floats] [stages: nrows x TC floats each].
-template <int P, bool EXACT, bool PREAGG, int V>
+// V values of a staged row at `p`: fp32, or (H16) 16-bit elements widened to fp32.
+template <int V, bool H16> __device__ __forceinline__ void read_row(const unsigned char* p, int dtype, float (&x)[V]) {
+    if constexpr (!H16) {
+        read_vec<V>(reinterpret_cast<const float*>(p), x);
+    } else if constexpr (V == 1) {
+        x[0] = widen16(*reinterpret_cast<const unsigned short*>(p), dtype);
+    } else if constexpr (V == 2) {
+        const unsigned u = *reinterpret_cast<const unsigned*>(p);
+        x[0] = widen16(static_cast<unsigned short>(u & 0xffffu), dtype);
+        x[1] = widen16(static_cast<unsigned short>(u >> 16), dtype);
+    } else {
+        const uint2 u = *reinterpret_cast<const uint2*>(p);
+        x[0] = widen16(static_cast<unsigned short>(u.x & 0xffffu), dtype);
+        x[1] = widen16(static_cast<unsigned short>(u.x >> 16), dtype);
+        x[2] = widen16(static_cast<unsigned short>(u.y & 0xffffu), dtype);
+        x[3] = widen16(static_cast<unsigned short>(u.y >> 16), dtype);
+    }
+}
+
+// H16: the gradients are 16-bit (bfloat16 or binary16 by `dtype`); the rows are staged as they are
+// (half the bytes per copy) and widened when read; the correction columns stay fp32 in an area of
+// their own.
+template <int P, bool EXACT, bool PREAGG, int V, bool H16>
 __global__ void __launch_bounds__(KBShape<V>::THREADS)
 k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64_t ld, gar_selection_t* __restrict__ sel,
-        const K3Out out, int pool_bytes) {
+        const K3Out out, int pool_bytes, int dtype) {
     constexpr int KB_TC = KBShape<V>::TC, KB_CT = KBShape<V>::CT, KB_THREADS = KBShape<V>::THREADS;
-    constexpr int KB_ROW_BYTES = KBShape<V>::ROW_BYTES;
+    constexpr int ES = H16 ? 2 : 4;                                  // bytes per gradient element
+    constexpr int KB_ROW_BYTES = KB_TC * ES;                         // one staged row of a tile (one bulk copy)
+    constexpr int KB_COL_BYTES = KB_TC * 4;                          // one correction column (fp32)
     __shared__ KBPlan plan;
     extern __shared__ __align__(128) unsigned char kb_dyn[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -159,7 +183,7 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
                 if (!shared_row) plan.col_row[nfree++] = uint8_t(s);
             }
         }
-        const bool in_stage = PREAGG && nfree >= ncorr + 1;
+        const bool in_stage = PREAGG && !H16 && nfree >= ncorr + 1;
         plan.cols_in_stage = in_stage ? 1 : 0;
         if (!in_stage)
             for (int c = 0; c <= ncorr; ++c) plan.col_row[c] = uint8_t(c);
@@ -168,8 +192,8 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
             plan.corr_dst[j] = plan.col_row[j + 1];
         }
         if (PREAGG)
-            for (int s = 0; s < theta; ++s) plan.slot[s].coff = int(plan.col_row[slot_col[s]]) * KB_ROW_BYTES;
-        const int fixed = ((nadds + 15) & ~15) + (in_stage ? 0 : (ncorr + 1) * KB_ROW_BYTES);
+            for (int s = 0; s < theta; ++s) plan.slot[s].coff = int(plan.col_row[slot_col[s]]) * KB_COL_BYTES;
+        const int fixed = ((nadds + 15) & ~15) + (in_stage ? 0 : (ncorr + 1) * KB_COL_BYTES);
         int nst = (pool_bytes - fixed) / (nrows * KB_ROW_BYTES);
         if (nst > KB_MAX_STAGES) nst = KB_MAX_STAGES;
         plan.nstages = nst;
@@ -186,7 +210,7 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
     const int ncorr = plan.ncorr, nrows = plan.nrows, nstages = plan.nstages;
     float* const ccol = reinterpret_cast<float*>(kb_dyn + ((nadds + 15) & ~15));
     const bool cols_in_stage = plan.cols_in_stage != 0;
-    unsigned char* const stages = reinterpret_cast<unsigned char*>(ccol) + (cols_in_stage ? 0 : (ncorr + 1) * KB_ROW_BYTES);
+    unsigned char* const stages = reinterpret_cast<unsigned char*>(ccol) + (cols_in_stage ? 0 : (ncorr + 1) * KB_COL_BYTES);
     const unsigned stage_bytes = unsigned(nrows) * KB_ROW_BYTES;
     if (!cols_in_stage)
         for (int c = tid; c < KB_TC; c += KB_THREADS) ccol[c] = 0.0f;
@@ -209,11 +233,11 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
                 if (lane == 0)
                     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(stage_bytes) : "memory");
                 __syncwarp();
-                const float* src = g + (first + i * step) * KB_TC;
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(g) + (first + i * step) * (KB_TC * ES);
                 const unsigned dst = kb_smem_u32(stages) + unsigned(st) * stage_bytes;
                 for (int r = lane; r < nrows; r += 32)
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                                 ::"r"(dst + unsigned(r) * KB_ROW_BYTES), "l"(src + plan.roff[r]), "r"(unsigned(KB_ROW_BYTES)), "r"(bar) : "memory");
+                                 ::"r"(dst + unsigned(r) * KB_ROW_BYTES), "l"(src + plan.roff[r] * ES), "r"(unsigned(KB_ROW_BYTES)), "r"(bar) : "memory");
                 if (++st == nstages) { st = 0; parity ^= 1u; }
             }
             // no copy may be in flight when the CTA leaves: wait (bounded) for the last tiles issued,
@@ -238,14 +262,13 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
             asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
                          : "=r"(failed) : "r"(*error), "r"(KB_BAR_COMPUTE), "r"(KB_CT) : "memory");
             if (failed) break;
-            float* const svw = reinterpret_cast<float*>(stages + size_t(st) * stage_bytes) + tid * V;
-            const float* sv = svw;
-            float* const mycol = cols_in_stage ? svw : ccol + tid * V;   // this thread's entries of the correction columns' rows
+            unsigned char* const svb = stages + size_t(st) * stage_bytes + tid * V * ES;     // this thread's entries of the staged rows
+            float* const mycol = cols_in_stage ? reinterpret_cast<float*>(svb) : ccol + tid * V;   // ... and of the correction columns' rows
             float e[P][V], a[P][V];
 #pragma unroll
             for (int s = 0; s < P; ++s) {
                 if (s < theta) {
-                    read_vec<V>(sv + s * KB_TC, e[s]);
+                    read_row<V, H16>(svb + s * KB_ROW_BYTES, dtype, e[s]);
                 } else {
 #pragma unroll
                     for (int v = 0; v < V; ++v) e[s][v] = 0.0f;
@@ -255,21 +278,22 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
                 float T[V];
 #pragma unroll
                 for (int v = 0; v < V; ++v) T[v] = 0.0f;
-                const float* bp = sv + theta * KB_TC;
+                const unsigned char* bp = svb + theta * KB_ROW_BYTES;
                 int k = 0;
                 for (; k + 4 <= nbase; k += 4) {
                     float x0[V], x1[V], x2[V], x3[V];
-                    read_vec<V>(bp, x0); read_vec<V>(bp + KB_TC, x1); read_vec<V>(bp + 2 * KB_TC, x2); read_vec<V>(bp + 3 * KB_TC, x3);
+                    read_row<V, H16>(bp, dtype, x0); read_row<V, H16>(bp + KB_ROW_BYTES, dtype, x1);
+                    read_row<V, H16>(bp + 2 * KB_ROW_BYTES, dtype, x2); read_row<V, H16>(bp + 3 * KB_ROW_BYTES, dtype, x3);
 #pragma unroll
                     for (int v = 0; v < V; ++v) { T[v] += x0[v]; T[v] += x1[v]; T[v] += x2[v]; T[v] += x3[v]; }
-                    bp += 4 * KB_TC;
+                    bp += 4 * KB_ROW_BYTES;
                 }
                 for (; k < nbase; ++k) {
                     float x0[V];
-                    read_vec<V>(bp, x0);
+                    read_row<V, H16>(bp, dtype, x0);
 #pragma unroll
                     for (int v = 0; v < V; ++v) T[v] += x0[v];
-                    bp += KB_TC;
+                    bp += KB_ROW_BYTES;
                 }
                 {                                        // column 0: zero (its row's value has been used)
                     float z[V];
@@ -284,7 +308,7 @@ k3_bulk(const float* __restrict__ g, int n, int theta_arg, int64_t ntiles, int64
                     const int kend = kadd + plan.corr_nadd[j];
                     for (; kadd < kend; ++kadd) {
                         float x[V];
-                        read_vec<V>(sv + int(add_row[kadd]) * KB_TC, x);
+                        read_row<V, H16>(svb + int(add_row[kadd]) * KB_ROW_BYTES, dtype, x);
 #pragma unroll
                         for (int v = 0; v < V; ++v) C[v] += x[v];
                     }

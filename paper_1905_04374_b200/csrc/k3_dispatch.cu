@@ -47,8 +47,10 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
     // memory and wins while the slot count is a compile-time constant, up to 32 slots.
     const int bulk_from = preagg ? 1 : 33;
     // (a few hundred thousand coordinates amortise its set-up: the plan, the barriers, the first tiles)
-    // (16-bit gradients go through the register kernel, which widens them as it loads)
-    const bool bulk = dtype == GAR_F32 && vec_max == 4 && theta >= bulk_from && d >= 400000;
+    // (16-bit gradients: staged for the pre-aggregating rules when the rows are 16-byte aligned,
+    // else through the register kernel, which widens them as it loads)
+    const bool rows16 = dtype != GAR_F32 && preagg && reinterpret_cast<uintptr_t>(grads) % 16 == 0 && ld % 8 == 0 && o % 16 == 0;
+    const bool bulk = (dtype == GAR_F32 ? vec_max == 4 : rows16) && theta >= bulk_from && d >= 400000;
 #define K3_TRY(P)                                                                                              \
     if (theta <= P) {                                                                                          \
         const int ctas = bulk ? bulk_ctas_for<P>(n, theta, preagg) : 0;                                        \

@@ -41,9 +41,9 @@ static int bulk_ctas(int n, int theta) {
 }
 
 // Full tiles [0, *covered) through the staged kernel, `ctas` CTAs per SM.
-template <int P, bool PREAGG>
+template <int P, bool PREAGG, bool H16>
 static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta,
-                            int ctas, const K3Out& out, int sm_count, cudaStream_t stream, int64_t* covered) {
+                            int ctas, const K3Out& out, int sm_count, cudaStream_t stream, int64_t* covered, int dtype) {
     constexpr bool EXACT = (K3_EXACT != 0);
     constexpr int V = BulkV<PREAGG>::V;
     using S = KBShape<V>;
@@ -60,16 +60,16 @@ static cudaError_t run_bulk(const float* g, int n, int64_t d, int64_t ld, gar_se
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (dev < 0 || dev >= 64 || configured[dev] < pool) {
-        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(pool));
+        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG, V, H16>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(pool));
         if (err != cudaSuccess) return err;
-        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG, V>, cudaFuncAttributePreferredSharedMemoryCarveout,
+        err = cudaFuncSetAttribute(k3_bulk<P, EXACT, PREAGG, V, H16>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                    cudaSharedmemCarveoutMaxShared);
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = pool;
     }
     int64_t grid = int64_t(sm_count) * ctas;
     if (grid > ntiles) grid = ntiles;
-    k3_bulk<P, EXACT, PREAGG, V><<<unsigned(grid), S::THREADS, pool, stream>>>(g, n, theta, ntiles, ld, sel, out, int(pool));
+    k3_bulk<P, EXACT, PREAGG, V, H16><<<unsigned(grid), S::THREADS, pool, stream>>>(g, n, theta, ntiles, ld, sel, out, int(pool), dtype);
     *covered = ntiles * S::TC;
     return cudaGetLastError();
 }
@@ -122,8 +122,11 @@ cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_
                               int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream, int dtype) {
     int64_t t0 = 0;
     if (bulk_ctas > 0) {                         // whole tiles staged through shared memory, the rest below
-        const cudaError_t err = preagg ? run_bulk<K3_P, true>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0)
-                                       : run_bulk<K3_P, false>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0);
+        // 16-bit gradients: the staged kernel is compiled for the pre-aggregating rules only
+        const cudaError_t err =
+            dtype != GAR_F32 ? run_bulk<K3_P, true, true>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0, dtype)
+            : preagg         ? run_bulk<K3_P, true, false>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0, dtype)
+                             : run_bulk<K3_P, false, false>(g, n, d, ld, sel, theta, bulk_ctas, out, sm_count, stream, &t0, dtype);
         if (err != cudaSuccess) return err;
         if (t0 == d) return cudaSuccess;
     }

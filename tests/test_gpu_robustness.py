@@ -346,7 +346,8 @@ def test_fused_sgd_leaves_the_model_alone_on_failure(pkg):
 
 # ------------------------------------------------------------ 16-bit gradient inputs
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
-@pytest.mark.parametrize("cfg,d", [(5, 4099), (5, 450_048), (5, 450_051), (2, 70_001), (3, 262_148), (1, 200_003)])
+@pytest.mark.parametrize("cfg,d", [(5, 4099), (5, 450_048), (5, 450_051), (2, 70_001), (3, 262_148), (1, 200_003),
+                                   (3, 262_144), (4, 401_408), (2, 1_048_576)])
 def test_sixteen_bit_gradients(pkg, dtype, cfg, d):
     """bfloat16 / binary16 gradients: every value is widened to fp32 exactly when it is loaded, so
     the oracle, fed the same 16-bit values promoted to fp64, is the reference at the usual bars
