@@ -57,7 +57,7 @@ extern "C" {
 #endif
 
 #define GAR_MAX_N 64
-#define GAR_VERSION 101
+#define GAR_VERSION 102
 
 typedef enum {
     GAR_AVERAGE      = 0, /* (1/n) sum_i G_i                       (Introduction)            */
@@ -213,6 +213,13 @@ int gar_version(void);
 
 /* Static description of a status code. */
 const char* gar_status_string(int status);
+
+/* The CUDA runtime error (a cudaError_t value; 0 = none yet) behind the calling thread's latest
+ * GAR_ERR_CUDA return, and the runtime's own name for it (a static string; "cudaSuccess" when
+ * there was none).  Kept per host thread; a later successful call does not clear it.  The paper
+ * has no counterpart. */
+int gar_last_cuda_error(void);
+const char* gar_last_cuda_error_name(void);
 
 /* theta (number of extraction rounds) and beta (values kept per coordinate) of a
  * rule: multi-Bulyan n-2f-2 and theta-2f (Algorithm 1); Bulyan n-2f and theta-2f

@@ -20,6 +20,7 @@ GRAD_DTYPES = {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}
 # gar_workspace control block, word 4: how the last distance call ran
 DISTANCE_PATHS = {0: "difference", 1: "gram", 2: "gram_rejected"}
 GAR_OK = 0
+GAR_ERR_CUDA = 5
 STATUS_NAMES = {0: "GAR_OK", 1: "GAR_ERR_INVALID_ARG", 2: "GAR_ERR_PRECONDITION", 3: "GAR_ERR_UNSUPPORTED",
                 4: "GAR_ERR_WORKSPACE", 5: "GAR_ERR_CUDA", 6: "GAR_ERR_TIMEOUT"}
 
@@ -68,6 +69,8 @@ class GarError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         msg = lib().gar_status_string(status).decode()
+        if status == GAR_ERR_CUDA:
+            msg += f": {gar_last_cuda_error()[1]}"
         super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({msg})")
 
 
@@ -82,6 +85,8 @@ def lib():
         L.gar_version.restype = C.c_int
         L.gar_status_string.restype = C.c_char_p
         L.gar_status_string.argtypes = [C.c_int]
+        L.gar_last_cuda_error.restype = C.c_int
+        L.gar_last_cuda_error_name.restype = C.c_char_p
         L.gar_theta.argtypes = [C.c_int, C.c_int, C.c_int]
         L.gar_beta.argtypes = [C.c_int, C.c_int, C.c_int]
         L.gar_workspace_bytes.restype = C.c_size_t
@@ -141,6 +146,11 @@ def gar_version() -> int:
 
 def gar_status_string(status: int) -> str:
     return lib().gar_status_string(status).decode()
+
+
+def gar_last_cuda_error():
+    """(cudaError_t value, the runtime's name for it) behind this thread's latest GAR_ERR_CUDA."""
+    return lib().gar_last_cuda_error(), lib().gar_last_cuda_error_name().decode()
 
 
 def gar_theta(rule, n: int, f: int) -> int:

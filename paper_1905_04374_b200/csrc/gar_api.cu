@@ -27,6 +27,20 @@ struct DeviceState {
 DeviceState g_dev[kMaxDevices];
 std::mutex  g_mutex;
 
+// The CUDA error behind this thread's latest GAR_ERR_CUDA (gar_last_cuda_error).
+thread_local cudaError_t t_last_cuda_error = cudaSuccess;
+using gar::cuda_status;
+
+}  // namespace
+
+int gar::cuda_status(cudaError_t err) {
+    if (err == cudaSuccess) return GAR_OK;
+    t_last_cuda_error = err;
+    return GAR_ERR_CUDA;
+}
+
+namespace {
+
 bool rule_ok(int rule) { return rule >= GAR_AVERAGE && rule <= GAR_MULTI_BULYAN; }
 
 int precondition(int rule, int n, int f) {
@@ -59,23 +73,24 @@ int basic_checks(int rule, int n, int f, int64_t d) {
 // Current device's state; creates the cached pieces that were asked for.
 int device_state(DeviceState** out, bool need_workspace) {
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return GAR_ERR_CUDA;
+    if (int rc_ = cuda_status(cudaGetDevice(&dev))) return rc_;
     if (dev < 0 || dev >= kMaxDevices) return GAR_ERR_UNSUPPORTED;
     std::lock_guard<std::mutex> lock(g_mutex);
     DeviceState& st = g_dev[dev];
     if (!st.known) {
-        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return GAR_ERR_CUDA;
+        if (int rc_ = cuda_status(cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev))) return rc_;
         st.known = true;
     }
     if (need_workspace && !st.workspace) {
-        if (cudaMalloc(&st.workspace, gar::kWorkspaceBytes) != cudaSuccess) return GAR_ERR_CUDA;
+        if (int rc_ = cuda_status(cudaMalloc(&st.workspace, gar::kWorkspaceBytes))) return rc_;
         // the control block must read zero before the first kernel of ANY stream touches it (a
         // memset on the legacy stream is not ordered before work on a non-blocking stream)
-        if (cudaMemset(st.workspace, 0, gar::kCtrlBytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaError_t err = cudaMemset(st.workspace, 0, gar::kCtrlBytes);
+        if (err == cudaSuccess) err = cudaDeviceSynchronize();
+        if (err != cudaSuccess) {
             cudaFree(st.workspace);
             st.workspace = nullptr;
-            return GAR_ERR_CUDA;
+            return cuda_status(err);
         }
     }
     *out = &st;
@@ -112,13 +127,13 @@ int enqueue(int rule, const float* grads, int n, int f, int64_t d, int64_t ld, c
     if (needs_dist) {
         err = dtype == GAR_F32 ? gar::launch_distances(grads, n, d, ld, dist, ws, sm_count, distance_mode, stream)
                                : gar::launch_distances_16(grads, dtype, n, d, ld, dist, ws, sm_count, stream);
-        if (err != cudaSuccess) return GAR_ERR_CUDA;
+        if (err != cudaSuccess) return cuda_status(err);
     }
     err = gar::launch_select(rule, dist, n, f, m, theta, beta, median_of_agr, even_median, sel, stream);
-    if (err != cudaSuccess) return GAR_ERR_CUDA;
+    if (err != cudaSuccess) return cuda_status(err);
     const int preagg = (rule == GAR_MULTI_BULYAN || rule == GAR_MULTI_KRUM || rule == GAR_AVERAGE) ? 1 : 0;
     err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg, out, sm_count, stream, dtype);
-    if (err != cudaSuccess) return GAR_ERR_CUDA;
+    if (err != cudaSuccess) return cuda_status(err);
     return GAR_OK;
 }
 
@@ -167,6 +182,9 @@ cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t
 extern "C" {
 
 int gar_version(void) { return GAR_VERSION; }
+
+int gar_last_cuda_error(void) { return int(t_last_cuda_error); }
+const char* gar_last_cuda_error_name(void) { return cudaGetErrorName(t_last_cuda_error); }
 
 const char* gar_status_string(int status) {
     switch (status) {
@@ -263,7 +281,7 @@ int gar_pairwise_distances_mode(const float* grads, int n, int64_t d, int64_t ld
     if (rc != GAR_OK) return rc;
     cudaError_t err = gar::launch_distances(grads, n, d, ld, dist, ws, st->sm_count, distance_mode,
                                             static_cast<cudaStream_t>(stream));
-    return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return cuda_status(err);
 }
 
 int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int median_of_agr, int even_median,
@@ -283,13 +301,13 @@ int gar_select(int rule, const double* dist, int n, int f, int m, int theta, int
     if (!even_median_ok(even_median)) return GAR_ERR_INVALID_ARG;
     cudaError_t err = gar::launch_select(rule, dist, n, f, m, th, beta_for(rule, th, f), median_of_agr, even_median, sel,
                                          static_cast<cudaStream_t>(stream));
-    return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return cuda_status(err);
 }
 
 int gar_schedule_from_tables(gar_selection_t* sel, void* stream) {
     if (!sel) return GAR_ERR_INVALID_ARG;
     cudaError_t err = gar::launch_schedule_only(sel, static_cast<cudaStream_t>(stream));
-    return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return cuda_status(err);
 }
 
 int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta,
@@ -304,7 +322,7 @@ int gar_coordinate_phase(const float* grads, int n, int64_t d, int64_t ld, gar_s
     const gar::K3Out o{out, nullptr, nullptr, 0.0f, 0.0f};
     cudaError_t err = gar::launch_coordinate(grads, n, d, ld, sel, theta, preagg ? 1 : 0, o, st->sm_count,
                                              static_cast<cudaStream_t>(stream));
-    return err == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return cuda_status(err);
 }
 
 int gar_reduce_partials(const double* parts, int count, int n, double* dist, void* stream) {
@@ -312,12 +330,12 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
     if (n > GAR_MAX_N) return GAR_ERR_UNSUPPORTED;
     const int nn = n * n;
     reduce_partials_kernel<<<(nn + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(parts, count, nn, dist);
-    return cudaGetLastError() == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return cuda_status(cudaGetLastError());
 }
 
 int gar_selftest_bounded_wait(unsigned int limit, long long* result, void* stream) {
     if (!result || limit < 1u || limit > 65536u) return GAR_ERR_INVALID_ARG;
-    return gar::launch_selftest_wait(limit, result, static_cast<cudaStream_t>(stream)) == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return cuda_status(gar::launch_selftest_wait(limit, result, static_cast<cudaStream_t>(stream)));
 }
 
 int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, float* out) {
@@ -335,34 +353,32 @@ int gar_aggregate_host(int rule, const float* grads, int n, int f, int64_t d, fl
         if (st->stage_grads_elems < need) {
             if (st->stage_grads) cudaFree(st->stage_grads);
             st->stage_grads = nullptr; st->stage_grads_elems = 0;
-            if (cudaMalloc(&st->stage_grads, need * sizeof(float)) != cudaSuccess) return GAR_ERR_CUDA;
+            if (int rc_ = cuda_status(cudaMalloc(&st->stage_grads, need * sizeof(float)))) return rc_;
             st->stage_grads_elems = need;
         }
         if (st->stage_out_elems < size_t(d)) {
             if (st->stage_out) cudaFree(st->stage_out);
             st->stage_out = nullptr; st->stage_out_elems = 0;
-            if (cudaMalloc(&st->stage_out, size_t(d) * sizeof(float)) != cudaSuccess) return GAR_ERR_CUDA;
+            if (int rc_ = cuda_status(cudaMalloc(&st->stage_out, size_t(d) * sizeof(float)))) return rc_;
             st->stage_out_elems = size_t(d);
         }
-        if (!st->host_stream && cudaStreamCreateWithFlags(&st->host_stream, cudaStreamNonBlocking) != cudaSuccess)
-            return GAR_ERR_CUDA;
+        if (!st->host_stream) {
+            if (int rc_ = cuda_status(cudaStreamCreateWithFlags(&st->host_stream, cudaStreamNonBlocking))) return rc_;
+        }
     }
     // rows in (one contiguous copy), the three kernels, the result and the selection's status out
     cudaStream_t s = st->host_stream;
-    if (cudaMemcpyAsync(st->stage_grads, grads, need * sizeof(float), cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return GAR_ERR_CUDA;
+    if (int rc_ = cuda_status(cudaMemcpyAsync(st->stage_grads, grads, need * sizeof(float), cudaMemcpyHostToDevice, s))) return rc_;
     Workspace ws{st->workspace};
     const int theta = default_theta(rule, n, f);
     const gar::K3Out stage_out{st->stage_out, nullptr, nullptr, 0.0f, 0.0f};
     rc = enqueue(rule, st->stage_grads, n, f, d, d, stage_out, 0, theta, 0, GAR_EVEN_MEDIAN_LOWER, GAR_DISTANCES_AUTO,
                  ws, nullptr, nullptr, st->sm_count, s);
     if (rc != GAR_OK) return rc;
-    if (cudaMemcpyAsync(out, st->stage_out, size_t(d) * sizeof(float), cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return GAR_ERR_CUDA;
+    if (int rc_ = cuda_status(cudaMemcpyAsync(out, st->stage_out, size_t(d) * sizeof(float), cudaMemcpyDeviceToHost, s))) return rc_;
     int32_t status = GAR_OK;
-    if (cudaMemcpyAsync(&status, &ws.selection()->status, sizeof(status), cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return GAR_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return GAR_ERR_CUDA;
+    if (int rc_ = cuda_status(cudaMemcpyAsync(&status, &ws.selection()->status, sizeof(status), cudaMemcpyDeviceToHost, s))) return rc_;
+    if (int rc_ = cuda_status(cudaStreamSynchronize(s))) return rc_;
     return status;
 }
 

@@ -98,4 +98,7 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
 // One warp waits, bounded, on a barrier nobody arrives on; result[0] = status, result[1] = ns.
 cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t stream);
 
+// cudaSuccess -> GAR_OK; anything else is remembered for gar_last_cuda_error and becomes GAR_ERR_CUDA
+int cuda_status(cudaError_t err);
+
 }  // namespace gar

@@ -10,11 +10,13 @@
 // symmetric matrix.  No floating-point atomics: results are bit-reproducible
 // and D_ij == D_ji by construction.
 //
-// Two kernels:
-//  * n <= 16 ("direct"): a thread loads its V coordinates of all n rows straight
-//    from global memory (software-prefetched one iteration ahead) and updates
-//    all n(n-1)/2 accumulators in registers.  No shared-memory staging, no
-//    barrier in the loop; HBM-bound.
+// Three kernels:
+//  * n <= 16, 16-byte aligned rows, d of at least one tile per SM ("direct, staged"): tiles of
+//    1024 coordinates of all n rows arrive in shared memory by one bulk copy per row; a thread
+//    reads its four coordinates of every row and updates all n(n-1)/2 accumulators in registers
+//    with packed two-lane fp32 instructions.  HBM-bound.
+//  * n <= 16 otherwise ("direct"): a thread fetches its V coordinates of all n rows through its
+//    own ring of cp.async copies and updates the accumulators with scalar instructions.
 //  * n > 16 ("tiled"): rows are grouped in blocks of 8; a column slab of all rows
 //    is staged in shared memory through a cp.async ring.  A half-warp owns either
 //    one off-diagonal 8x8 tile (64 pairs) or two diagonal tiles (2 x 28 pairs);
@@ -150,6 +152,7 @@ template <int N> __device__ __forceinline__ void direct_pair_rows(int p, int& i,
 constexpr int K1R_THREADS = 128;
 constexpr int K1R_FLUSH = 64;       // iterations between fp64 flushes
 constexpr int K1R_STAGES = 4;       // depth of the per-thread cp.async ring
+constexpr int K1B_V = 4;            // staged kernel: coordinates per thread and tile (two: 35 % slower, the per-tile barrier shows) // staged kernel: rows from which a thread owns two coordinates instead of four
 
 template <int BYTES>
 __device__ __forceinline__ void cp_async_small(void* smem_dst, const void* gsrc) {
@@ -259,122 +262,237 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
 }
 
 // ================================================ direct kernel, n <= 16, rows staged by bulk copies
-// Same arithmetic as k1_direct with V = 4; the rows travel differently.  A tile is K1B_TC
-// consecutive coordinates of all N rows; a producer warp fetches it with one bulk copy per row
-// (4 KB, contiguous) into a ring of shared-memory stages whose mbarriers count the bytes in, and
-// the compute threads read their four coordinates of every row at fixed offsets.  Copies of that
-// size keep HBM busier than 16-byte requests per thread do.  Needs 16-byte aligned rows
-// (base address and row stride); coordinates after the last whole tile are added by CTA 0 with
-// plain loads.  A wait that gives up (bounded) raises the CTA's error slot: the last CTA then
-// fills the matrix, diagonal included, with NaN and sets the workspace's error word.
-constexpr int K1B_CT = 256;                    // compute threads
-constexpr int K1B_THREADS = K1B_CT + 32;       // + the producer warp
-constexpr int K1B_TC = K1B_CT * 4;             // coordinates per tile
-constexpr int K1B_ROW_BYTES = K1B_TC * 4;
-constexpr int K1B_STAGES = 3;
+// Same differences and sums as k1_direct; the rows travel and the arithmetic issues differently.
+//
+// Staging.  A tile is TC consecutive coordinates of all N rows; warp 0 fetches it with one bulk
+// copy per row (contiguous, 2 or 4 KB of fp32) into a ring of shared-memory stages whose mbarriers
+// count the bytes in.  Copies of that size keep HBM busier than 16-byte requests per thread do.
+// All eight warps compute, so that every thread may hold up to 255 registers (a ninth warp would
+// put three warps on one scheduler, whose 16 K registers then allow 168 per thread: too few for the
+// 105 to 120 accumulators of 15 or 16 rows next to the rows themselves).  The warps meet in a named
+// barrier once per tile; a warp that has passed it has finished the previous tile, so warp 0 refills
+// that tile's stage right behind the barrier and no second set of mbarriers is needed.
+//
+// Arithmetic.  Rows are taken two at a time: R_a = (x_2a, x_2a+1) sits in one 64-bit register pair,
+// and one packed subtract plus one packed multiply-add (sub.f32x2, fma.rn.f32x2: two IEEE fp32
+// operations each, one issue slot) serve two pairs at once --
+//     R_a - R_b          -> pairs (2a, 2b), (2a+1, 2b+1)
+//     R_a - swap(R_b)    -> pairs (2a, 2b+1), (2a+1, 2b)
+//     R_a - (x_N-1, x_N-1) for the unpaired last row of an odd N
+// and the pair (2a, 2a+1) inside a row pair takes scalar instructions.  That is 112 issue slots per
+// coordinate for 15 rows instead of 210, which is what lets eight warps keep up with HBM.
+//
+// Needs 16-byte aligned rows (base address and row stride); coordinates after the last whole tile
+// are added by CTA 0 with plain loads.  A wait that gives up (bounded) raises the CTA's error slot:
+// the last CTA then fills the matrix, diagonal included, with NaN and sets the workspace's error word.
+template <int N> struct K1BShape {
+    static constexpr int V = K1B_V;                                // coordinates per thread and tile
+    static constexpr int THREADS = 256;
+    static constexpr int WARPS = THREADS / 32;
+    static constexpr int TC = THREADS * V;                         // coordinates per tile
+    static constexpr int ROW_BYTES = TC * 4;                       // one fp32 row of a tile
+    static constexpr int STAGE_BYTES = N * ROW_BYTES;
+    static constexpr int NP = N * (N - 1) / 2;
+    static constexpr int NPAD = (NP + 31) / 32 * 32;
+    static constexpr int SUM_BYTES = WARPS * NPAD * 8;
+    static constexpr int STAGES_FIT = (200 * 1024 - SUM_BYTES) / STAGE_BYTES;
+    static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT; // depth of the ring
+    static constexpr int NF = N / 2;                               // whole row pairs
+    static constexpr int NBLK = NF * (NF - 1) / 2;                 // blocks of two row pairs
+    static constexpr int NPK = 2 * NBLK + (N % 2 ? NF : 0);        // packed accumulators
+    static_assert(2 * NPK + NF == NP, "accumulator slots");
+    static_assert(STAGES >= 3, "ring depth");
+};
+constexpr int K1B_MIN_TC = 256 * K1B_V;        // coordinates per tile (dispatch threshold)
 constexpr int K1B_BAR_COMPUTE = 1;
 
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long p, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+// acc += (a - b)^2 in both lanes
+__device__ __forceinline__ void sqdiff2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+    unsigned long long df;
+    asm("sub.f32x2 %0, %1, %2;" : "=l"(df) : "l"(a), "l"(b));
+    asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc) : "l"(df));
+}
+
+// The accumulators of one thread.  Slot order (the order of the CTA's partial sums):
+//   for a < b < NF:   4 * blk(a, b) + {0: (2a, 2b), 1: (2a+1, 2b+1), 2: (2a, 2b+1), 3: (2a+1, 2b)}
+//   odd N, a < NF:    4 * NBLK + 2a + {0: (2a, N-1), 1: (2a+1, N-1)}
+//   a < NF:           2 * NPK + a: (2a, 2a+1)
+template <int N> struct K1BAcc {
+    using S = K1BShape<N>;
+    unsigned long long pk[S::NPK > 0 ? S::NPK : 1];
+    float dg[S::NF > 0 ? S::NF : 1];
+
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < S::NPK; ++i) pk[i] = 0ull;
+#pragma unroll
+        for (int i = 0; i < S::NF; ++i) dg[i] = 0.0f;
+    }
+    // one coordinate of all rows
+    __device__ __forceinline__ void add(const float (&x)[N]) {
+        unsigned long long R[S::NF > 0 ? S::NF : 1];
+#pragma unroll
+        for (int a = 0; a < S::NF; ++a) R[a] = pack2(x[2 * a], x[2 * a + 1]);
+        int k = 0;
+#pragma unroll
+        for (int a = 0; a < S::NF; ++a) {
+#pragma unroll
+            for (int b = a + 1; b < S::NF; ++b) {
+                sqdiff2(pk[k], R[a], R[b]);
+                sqdiff2(pk[k + 1], R[a], pack2(x[2 * b + 1], x[2 * b]));
+                k += 2;
+            }
+        }
+        if constexpr (N % 2 == 1) {
+            const unsigned long long last = pack2(x[N - 1], x[N - 1]);
+#pragma unroll
+            for (int a = 0; a < S::NF; ++a) sqdiff2(pk[2 * S::NBLK + a], R[a], last);
+        }
+#pragma unroll
+        for (int a = 0; a < S::NF; ++a) { const float df = x[2 * a] - x[2 * a + 1]; dg[a] = fmaf(df, df, dg[a]); }
+    }
+    // the warp's fp32 accumulators -> its fp64 sums in shared memory (fixed shuffle tree), then zero
+    __device__ __forceinline__ void flush(double* warp_sums, int lane, int sbase) {
+        float flat[S::NPAD];
+#pragma unroll
+        for (int i = 0; i < S::NPK; ++i) unpack2(pk[i], flat[2 * i], flat[2 * i + 1]);
+#pragma unroll
+        for (int i = 0; i < S::NF; ++i) flat[2 * S::NPK + i] = dg[i];
+#pragma unroll
+        for (int i = S::NP; i < S::NPAD; ++i) flat[i] = 0.0f;
+        reduce_scatter<S::NPAD, 32>(flat, lane);
+#pragma unroll
+        for (int i = 0; i < S::NPAD / 32; ++i) warp_sums[sbase + i] += double(flat[i]);
+        zero();
+    }
+};
+// slot of K1BAcc -> the pair of rows (i < j)
+template <int N> __device__ __forceinline__ void k1b_slot_rows(int slot, int& i, int& j) {
+    using S = K1BShape<N>;
+    if (slot >= 2 * S::NPK) { i = 2 * (slot - 2 * S::NPK); j = i + 1; return; }
+    if (slot >= 4 * S::NBLK) { i = slot - 4 * S::NBLK; j = N - 1; return; }
+    int blk = slot >> 2, a = 0;
+    while (blk >= S::NF - 1 - a) { blk -= S::NF - 1 - a; ++a; }
+    const int b = a + 1 + blk, which = slot & 3;
+    i = 2 * a + (which & 1);
+    j = 2 * b + ((which == 1 || which == 2) ? 1 : 0);
+}
+
 // dtype: the gradients' element type (gar_dtype_t).  16-bit elements are staged as they are (a row of
-// a tile is then 2 KB instead of 4) and widened to fp32 when the compute threads read them.
+// a tile is then half as long) and widened to fp32 when the compute threads read them.
 template <int N>
-__global__ void __launch_bounds__(K1B_THREADS)
+__global__ void __launch_bounds__(K1BShape<N>::THREADS, 1)
 k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, double* __restrict__ dist,
                double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
                unsigned int* __restrict__ path_word) {
-    constexpr int NP = N * (N - 1) / 2;
-    constexpr int NPAD = (NP + 31) / 32 * 32;
-    constexpr int WARPS = K1B_CT / 32;
+    using S = K1BShape<N>;
+    constexpr int NP = S::NP, NPAD = S::NPAD, V = S::V, THREADS = S::THREADS, WARPS = S::WARPS, TC = S::TC, STAGES = S::STAGES;
     const int esize = dtype == GAR_F32 ? 4 : 2;
-    const unsigned row_bytes = unsigned(K1B_TC) * unsigned(esize);
-    const unsigned STAGE_BYTES = unsigned(N) * row_bytes;
-    extern __shared__ __align__(128) unsigned char stages[];          // [stage][row][K1B_TC floats]
+    const unsigned row_bytes = unsigned(TC) * unsigned(esize);
+    const unsigned stage_bytes = unsigned(N) * row_bytes;
+    extern __shared__ __align__(128) unsigned char stages[];          // [stage][row][TC elements]
     __shared__ double sums[WARPS][NPAD];
-    __shared__ unsigned long long full[K1B_STAGES], empty[K1B_STAGES];
+    __shared__ unsigned long long full[STAGES];
     __shared__ int error_flag;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    for (int i = tid; i < WARPS * NPAD; i += K1B_THREADS) (&sums[0][0])[i] = 0.0;
+    for (int i = tid; i < WARPS * NPAD; i += THREADS) (&sums[0][0])[i] = 0.0;
     if (tid == 0) {
-        for (int st = 0; st < K1B_STAGES; ++st) { kb_init(&full[st], 1u); kb_init(&empty[st], unsigned(WARPS)); }
+        for (int st = 0; st < STAGES; ++st) kb_init(&full[st], 1u);
         error_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        kb_fence_init();
     }
     __syncthreads();
     volatile int* error = &error_flag;
 
-    const int64_t ntiles = d / K1B_TC;
+    const int64_t ntiles = d / TC;
     const int64_t first = blockIdx.x, step = gridDim.x;
     const int64_t mine = first < ntiles ? (ntiles - first + step - 1) / step : 0;
 
-    if (warp == WARPS) {
-        // ================================================================ producer: lane r fetches row r
-        int st = 0;
-        unsigned parity = 1;                         // the phase before the first one: the first waits pass
-        int64_t i = 0;
-        for (; i < mine; ++i) {
-            if (!__all_sync(0xffffffffu, kb_wait(kb_smem_u32(&empty[st]), parity, error))) break;
-            const unsigned bar = kb_smem_u32(&full[st]);
-            if (lane == 0) kb_expect_tx(bar, STAGE_BYTES);
-            __syncwarp();
-            if (lane < N)
-                kb_bulk_load(kb_smem_u32(stages) + unsigned(st) * STAGE_BYTES + unsigned(lane) * row_bytes,
-                             static_cast<const char*>(g) + (int64_t(lane) * ld + (first + i * step) * K1B_TC) * esize, row_bytes, bar);
-            if (++st == K1B_STAGES) { st = 0; parity ^= 1u; }
-        }
-        // no copy may be in flight when the CTA leaves: wait (bounded) for the last tiles issued
-        for (int64_t j = i > K1B_STAGES ? i - K1B_STAGES : 0; j < i; ++j)
-            kb_wait(kb_smem_u32(&full[j % K1B_STAGES]), unsigned(j / K1B_STAGES) & 1u, error, true);
-    } else {
-        // ================================================================ compute: four coordinates per thread
-        float acc[NPAD];
-#pragma unroll
-        for (int i = 0; i < NPAD; ++i) acc[i] = 0.0f;
-        const int sbase = scatter_base<NPAD, 32>(lane);
-        auto flush = [&]() { direct_flush<NPAD>(acc, sums[warp], lane, sbase); };
-        int st = 0, since = 0;
-        unsigned parity = 0;
-        for (int64_t it = 0; it < mine; ++it) {
-            // one warp waits on the stage's barrier, the others sleep in a hardware barrier meanwhile
-            if (warp == 0) kb_wait(kb_smem_u32(&full[st]), parity, error);
-            unsigned failed;                      // the same answer in every compute thread
-            asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
-                         : "=r"(failed) : "r"(*error), "r"(K1B_BAR_COMPUTE), "r"(K1B_CT) : "memory");
-            if (failed) break;
-            float x[N][4];
-            if (dtype == GAR_F32) {
-                const float4* src = reinterpret_cast<const float4*>(stages + size_t(st) * STAGE_BYTES) + tid;
-#pragma unroll
-                for (int r = 0; r < N; ++r) {
-                    const float4 q = src[r * (K1B_TC / 4)];
-                    x[r][0] = q.x; x[r][1] = q.y; x[r][2] = q.z; x[r][3] = q.w;
-                }
-            } else {
-                const uint2* src = reinterpret_cast<const uint2*>(stages + size_t(st) * STAGE_BYTES) + tid;
-#pragma unroll
-                for (int r = 0; r < N; ++r) {
-                    const uint2 q = src[r * (K1B_TC / 4)];
-                    x[r][0] = widen16(static_cast<unsigned short>(q.x & 0xffffu), dtype);
-                    x[r][1] = widen16(static_cast<unsigned short>(q.x >> 16), dtype);
-                    x[r][2] = widen16(static_cast<unsigned short>(q.y & 0xffffu), dtype);
-                    x[r][3] = widen16(static_cast<unsigned short>(q.y >> 16), dtype);
-                }
-            }
-            __syncwarp();                         // the rows are in registers: hand the stage back
-            if (lane == 0) kb_arrive(&empty[st]);
-            direct_pairs<N, 4, NPAD>(x, acc);
-            if (++since == K1R_FLUSH) { flush(); since = 0; }
-            if (++st == K1B_STAGES) { st = 0; parity ^= 1u; }
-        }
-        // coordinates after the last whole tile: CTA 0, plain loads
-        if (blockIdx.x == 0) {
-            for (int64_t t = ntiles * K1B_TC + tid; t < d; t += K1B_CT) direct_tail_coordinate<N, NPAD>(g, ld, t, acc, dtype);
-        }
+    // warp 0, lane r fetches row r of this CTA's tile number i into stage i % STAGES
+    auto fetch = [&](int64_t i) {
+        const int st = int(i % STAGES);
+        const unsigned bar = kb_smem_u32(&full[st]);
+        if (lane == 0) kb_expect_tx(bar, stage_bytes);
         __syncwarp();
-        flush();
+        if (lane < N)
+            kb_bulk_load(kb_smem_u32(stages) + unsigned(st) * stage_bytes + unsigned(lane) * row_bytes,
+                         static_cast<const char*>(g) + (int64_t(lane) * ld + (first + i * step) * TC) * esize, row_bytes, bar);
+    };
+    int64_t issued = 0;                              // warp 0: tiles requested so far
+    if (warp == 0) {
+        for (; issued < STAGES - 1 && issued < mine; ++issued) fetch(issued);
     }
+
+    K1BAcc<N> acc;
+    acc.zero();
+    const int sbase = scatter_base<NPAD, 32>(lane);
+    int st = 0, since = 0;
+    unsigned parity = 0;
+    int64_t it = 0;
+    for (; it < mine; ++it) {
+        // one warp waits on the stage's barrier, the others sleep in a hardware barrier meanwhile
+        if (warp == 0) kb_wait(kb_smem_u32(&full[st]), parity, error);
+        unsigned failed;                          // the same answer in every thread
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %1, 0;\n\tbar.red.or.pred p, %2, %3, q;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                     : "=r"(failed) : "r"(*error), "r"(K1B_BAR_COMPUTE), "r"(THREADS) : "memory");
+        if (failed) break;
+        // every warp is past tile it - 1: its stage takes tile it + STAGES - 1
+        if (warp == 0 && issued < mine) { fetch(issued); ++issued; }
+        const unsigned char* tile = stages + size_t(st) * stage_bytes;
+        if (dtype == GAR_F32) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                float x[N];
+#pragma unroll
+                for (int r = 0; r < N; ++r) x[r] = reinterpret_cast<const float*>(tile + size_t(r) * row_bytes)[v * THREADS + tid];
+                acc.add(x);
+            }
+        } else {
+#pragma unroll
+            for (int v = 0; v < V; v += 2) {
+                float x0[N], x1[N];
+#pragma unroll
+                for (int r = 0; r < N; ++r) {
+                    const unsigned q = reinterpret_cast<const unsigned*>(tile + size_t(r) * row_bytes)[(v / 2) * THREADS + tid];
+                    x0[r] = widen16(static_cast<unsigned short>(q & 0xffffu), dtype);
+                    x1[r] = widen16(static_cast<unsigned short>(q >> 16), dtype);
+                }
+                acc.add(x0);
+                acc.add(x1);
+            }
+        }
+        if (++since == K1R_FLUSH) { acc.flush(sums[warp], lane, sbase); since = 0; }
+        if (++st == STAGES) { st = 0; parity ^= 1u; }
+    }
+    // no copy may be in flight when the CTA leaves: after a failure, wait (bounded) for the tiles
+    // that were requested and not consumed
+    if (warp == 0) {
+        for (int64_t j = it; j < issued; ++j)
+            kb_wait(kb_smem_u32(&full[j % STAGES]), unsigned(j / STAGES) & 1u, error, true);
+    }
+    // coordinates after the last whole tile: CTA 0, plain loads
+    if (blockIdx.x == 0) {
+        for (int64_t t = ntiles * TC + tid; t < d; t += THREADS) {
+            float x[N];
+#pragma unroll
+            for (int r = 0; r < N; ++r) x[r] = load_elem(g, int64_t(r) * ld + t, dtype);
+            acc.add(x);
+        }
+    }
+    __syncwarp();
+    acc.flush(sums[warp], lane, sbase);
     __syncthreads();
 
     double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
-    for (int i = tid; i < NP; i += K1B_THREADS) {
+    for (int i = tid; i < NP; i += THREADS) {
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) s += sums[w][i];
@@ -392,15 +510,15 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
     __syncthreads();
     const bool failed = any_error != 0;
     const double nan = __longlong_as_double(0x7ff8000000000000ll);
-    reduce_partials(partials, NP, K1B_THREADS, [&](int p, double s) {
+    reduce_partials(partials, NP, THREADS, [&](int p, double s) {
         int i, j;
-        direct_pair_rows<N>(p, i, j);
+        k1b_slot_rows<N>(p, i, j);
         if (failed) s = nan;
         dist[i * N + j] = s;
         dist[j * N + i] = s;
     });
     // a NaN diagonal tells the selection kernel that the matrix is not to be used
-    for (int i = tid; i < N; i += K1B_THREADS) dist[i * N + i] = failed ? nan : 0.0;
+    for (int i = tid; i < N; i += THREADS) dist[i * N + i] = failed ? nan : 0.0;
     if (tid == 0) { *ticket = 0u; *path_word = kPathDifference; }   // ready for the next call
 }
 
@@ -726,11 +844,12 @@ template <int N>
 cudaError_t launch_direct_bulk(const void* g, int dtype, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                                cudaStream_t stream) {
     static int per_sm_cache[64] = {0};
-    const size_t smem = size_t(K1B_STAGES) * N * K1B_ROW_BYTES;      // sized for fp32 rows; 16-bit rows use half of it
+    using S = K1BShape<N>;
+    const size_t smem = size_t(S::STAGES) * S::STAGE_BYTES;          // sized for fp32 rows; 16-bit rows use half of it
     int64_t grid = 0;
-    cudaError_t err = persistent_grid(k1_direct_bulk<N>, K1B_THREADS, smem, sm_count, per_sm_cache, d / K1B_TC, &grid);
+    cudaError_t err = persistent_grid(k1_direct_bulk<N>, S::THREADS, smem, sm_count, per_sm_cache, d / S::TC, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct_bulk<N><<<unsigned(grid), K1B_THREADS, smem, stream>>>(g, dtype, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
+    k1_direct_bulk<N><<<unsigned(grid), S::THREADS, smem, stream>>>(g, dtype, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
                                                                      ws.k1_path());
     return cudaGetLastError();
 }
@@ -739,7 +858,7 @@ template <int N>
 cudaError_t launch_direct_n(const float* g, int64_t d, int64_t ld, double* dist, const Workspace& ws, int sm_count,
                             cudaStream_t stream, int vec) {
     // 16-byte aligned rows and enough whole tiles for every SM: rows staged by bulk copies
-    if (vec >= 4 && d >= int64_t(sm_count) * K1B_TC)
+    if (vec >= 4 && d >= int64_t(sm_count) * K1B_MIN_TC)
         return launch_direct_bulk<N>(g, GAR_F32, d, ld, dist, ws, sm_count, stream);
     // few rows: wide vectors keep enough bytes in flight; many rows: narrow ones keep the registers in check
     if constexpr (N <= 8) {
@@ -795,7 +914,7 @@ cudaError_t launch_distances_16(const void* grads, int dtype, int n, int64_t d, 
                                 const Workspace& ws, int sm_count, cudaStream_t stream) {
     if (n == 1) return cudaMemsetAsync(dist, 0, sizeof(double), stream);
     const uintptr_t addr = reinterpret_cast<uintptr_t>(grads);
-    if (n <= 16 && addr % 16 == 0 && ld % 8 == 0 && d >= int64_t(sm_count) * K1B_TC) {
+    if (n <= 16 && addr % 16 == 0 && ld % 8 == 0 && d >= int64_t(sm_count) * K1B_MIN_TC) {
 #define GAR_K1_BULK16(NV) case NV: return launch_direct_bulk<NV>(grads, dtype, d, ld, dist, ws, sm_count, stream);
         switch (n) {
             GAR_K1_BULK16(2) GAR_K1_BULK16(3) GAR_K1_BULK16(4) GAR_K1_BULK16(5) GAR_K1_BULK16(6) GAR_K1_BULK16(7)
@@ -863,7 +982,7 @@ extern "C" int gar_pairwise_distances_static(const float* grads, int n, int64_t 
     if (ld == 0) ld = d;
     if (ld < d) return GAR_ERR_INVALID_ARG;
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return GAR_ERR_CUDA;
+    if (int rc = gar::cuda_status(cudaGetDevice(&dev))) return rc;
     if (dev < 0 || dev >= 64) return GAR_ERR_UNSUPPORTED;
     gar::StaticScratchState& st = gar::g_static_state[dev];
     std::unique_lock<std::mutex> lock(gar::g_static_mutex);
@@ -871,9 +990,9 @@ extern "C" int gar_pairwise_distances_static(const float* grads, int n, int64_t 
         // Once per device, with that device current: in host code the array's name is only a
         // stand-in; the address the kernels need comes from the runtime.
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, gar::g_static_scratch) != cudaSuccess || p == nullptr) return GAR_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            return GAR_ERR_CUDA;
+        if (int rc = gar::cuda_status(cudaGetSymbolAddress(&p, gar::g_static_scratch))) return rc;
+        if (p == nullptr) return gar::cuda_status(cudaErrorInvalidSymbol);
+        if (int rc = gar::cuda_status(cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev))) return rc;
         st.ptr = static_cast<char*>(p);
         st.ready = true;
     }
@@ -881,7 +1000,7 @@ extern "C" int gar_pairwise_distances_static(const float* grads, int n, int64_t 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // the array keeps the previous call's contents: the ticket counter must start at zero
     // (the partial sums are overwritten before they are read)
-    if (cudaMemsetAsync(st.ptr, 0, gar::kCtrlBytes, s) != cudaSuccess) return GAR_ERR_CUDA;
+    if (int rc = gar::cuda_status(cudaMemsetAsync(st.ptr, 0, gar::kCtrlBytes, s))) return rc;
     gar::Workspace ws{st.ptr};
-    return gar::launch_distances(grads, n, d, ld, dist, ws, st.sm_count, GAR_DISTANCES_AUTO, s) == cudaSuccess ? GAR_OK : GAR_ERR_CUDA;
+    return gar::cuda_status(gar::launch_distances(grads, n, d, ld, dist, ws, st.sm_count, GAR_DISTANCES_AUTO, s));
 }

@@ -54,8 +54,9 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
 
 
 def test_version_and_strings(pkg):
-    assert pkg.gar_version() == 101
+    assert pkg.gar_version() == 102
     assert pkg.gar_status_string(0) == "ok"
+    assert pkg.gar_last_cuda_error() == (0, "cudaSuccess")      # nothing has failed in this thread yet
     assert "4f+3" in pkg.gar_status_string(2)
 
 
