@@ -271,7 +271,9 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
 // put three warps on one scheduler, whose 16 K registers then allow 168 per thread: too few for the
 // 105 to 120 accumulators of 15 or 16 rows next to the rows themselves).  The warps meet in a named
 // barrier once per tile; a warp that has passed it has finished the previous tile, so warp 0 refills
-// that tile's stage right behind the barrier and no second set of mbarriers is needed.
+// that tile's stage right behind the barrier and no second set of mbarriers is needed.  (Letting
+// every warp wait on the tiles' mbarriers by itself, with a second set to hand stages back, so that
+// the warps may drift apart, measured 8 % slower.)
 //
 // Arithmetic.  Rows are taken two at a time: R_a = (x_2a, x_2a+1) sits in one 64-bit register pair,
 // and one packed subtract plus one packed multiply-add (sub.f32x2, fma.rn.f32x2: two IEEE fp32
