@@ -57,7 +57,7 @@ extern "C" {
 #endif
 
 #define GAR_MAX_N 64
-#define GAR_VERSION 102
+#define GAR_VERSION 103
 
 typedef enum {
     GAR_AVERAGE      = 0, /* (1/n) sum_i G_i                       (Introduction)            */
@@ -282,6 +282,55 @@ int gar_pairwise_distances_mode(const float* grads, int n, int64_t d, int64_t ld
  *   parts dev [count][n*n] fp64, dist dev [n*n] (may be parts[0]); 1 <= count <= 1024.
  */
 int gar_reduce_partials(const double* parts, int count, int n, double* dist, void* stream);
+
+/*
+ * Many small tensors in one launch sequence.  A model's gradient usually sits in memory as one
+ * tensor per layer; aggregating those one call at a time costs three kernel launches per tensor,
+ * which dominates below about 10^6 coordinates.  This call takes `count` tensors that share rule,
+ * n and f -- tensor t is an n x d[t] block of fp32 gradients, row i from worker i -- and runs each
+ * stage once over all of them: three to seven launches whatever the count (tensors whose addresses
+ * allow wide accesses and those that do not are launched separately).
+ *   joint = 0: every tensor is a problem of its own: own distance matrix, own selection, own
+ *              coordinate phase (Algorithm 1 applied per tensor; the paper has no counterpart).
+ *   joint = 1: the tensors are the pieces of ONE gradient in R^d, d = sum of d[t] (Section 2.1: the
+ *              rule acts on the whole gradient): the per-tensor distance matrices are added in the
+ *              order given (squared distances add over disjoint coordinates), one selection is
+ *              made, and every tensor's coordinate phase uses it.  The result equals
+ *              gar_aggregate on the concatenation up to the summation order of the distances.
+ * Distances use the fp32 difference form (Eq. 4's ||G_i - G_j||^2 term by term).  The work is
+ * split over CTAs in proportion to the tensors' lengths, so a few long tensors among many short
+ * ones are fine, but a batch of long tensors (above about 10^7 coordinates each) is served better
+ * by one gar_aggregate_ex per tensor.
+ *   tensors    HOST array of `count` entries, read before the call returns; grads / out device
+ *              pointers, ld = 0 means d; `out` must not overlap any tensor's gradients.
+ *   workspace  device, 256-byte aligned, >= gar_multi_workspace_bytes(rule, n, f, count); it may
+ *              hold anything on entry and must not be shared by calls in flight on other streams.
+ *   dist_out   optional, device: joint ? n*n : count*n*n doubles (tensor t's matrix at t*n*n).
+ *   selection_out  optional, device: joint ? 1 : count entries; its status field reports a
+ *              selection that could not be made (the outputs are then NaN), as for gar_aggregate_ex.
+ * Returns GAR_OK once everything is enqueued on `stream`.
+ */
+typedef struct gar_tensor_t {
+    const float* grads;
+    float*       out;
+    int64_t      d;
+    int64_t      ld;
+} gar_tensor_t;
+
+typedef struct gar_multi_params_t {
+    int32_t  rule, n, f, count;
+    int32_t  joint;
+    int32_t  even_median;            /* gar_even_median_t */
+    const gar_tensor_t* tensors;
+    void*    workspace;
+    size_t   workspace_bytes;
+    double*  dist_out;
+    gar_selection_t* selection_out;
+    void*    stream;
+} gar_multi_params_t;
+
+size_t gar_multi_workspace_bytes(int rule, int n, int f, int count);
+int gar_aggregate_multi(const gar_multi_params_t* params);
 
 /*
  * Step 1 alone, for callers that must not allocate: the same distance kernels, but

@@ -65,6 +65,21 @@ class GarParams(C.Structure):
     ]
 
 
+class GarTensor(C.Structure):
+    """Mirror of gar_tensor_t."""
+    _fields_ = [("grads", C.c_void_p), ("out", C.c_void_p), ("d", C.c_int64), ("ld", C.c_int64)]
+
+
+class GarMultiParams(C.Structure):
+    """Mirror of gar_multi_params_t."""
+    _fields_ = [
+        ("rule", C.c_int32), ("n", C.c_int32), ("f", C.c_int32), ("count", C.c_int32),
+        ("joint", C.c_int32), ("even_median", C.c_int32),
+        ("tensors", C.POINTER(GarTensor)), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+        ("dist_out", C.c_void_p), ("selection_out", C.c_void_p), ("stream", C.c_void_p),
+    ]
+
+
 class GarError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -99,6 +114,9 @@ def lib():
         L.gar_pairwise_distances_mode.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                                   C.c_size_t, C.c_int, C.c_void_p]
         L.gar_reduce_partials.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p]
+        L.gar_multi_workspace_bytes.restype = C.c_size_t
+        L.gar_multi_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int]
+        L.gar_aggregate_multi.argtypes = [C.POINTER(GarMultiParams)]
         L.gar_selftest_bounded_wait.argtypes = [C.c_uint, C.c_void_p, C.c_void_p]
         L.gar_pairwise_distances_static.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p]
         L.gar_select.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
@@ -227,6 +245,53 @@ def gar_aggregate_ex(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None
         st = lib().gar_aggregate_ex(C.byref(p))
     _check(st, "gar_aggregate_ex")
     return out
+
+
+def gar_multi_workspace_bytes(rule, n: int, f: int, count: int) -> int:
+    return lib().gar_multi_workspace_bytes(_rule(rule), n, f, count)
+
+
+def gar_aggregate_multi(rule, grads, f: int, outs=None, joint: bool = False, even_median=0, workspace=None,
+                        dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None, stream=None):
+    """gar_aggregate_multi: `grads` is a list of CUDA float32 tensors [n, d_t] (one per layer, the
+    same n, unit column stride); returns the list of aggregates [d_t].  joint=False: every tensor
+    is a problem of its own; joint=True: the tensors are the pieces of one gradient (one selection).
+    Optional: workspace (uint8 CUDA tensor of gar_multi_workspace_bytes), dist_out float64
+    [count, n, n] ([n, n] when joint), selection_out uint8 CUDA tensor of count (1 when joint)
+    times sizeof(gar_selection_t)."""
+    grads = list(grads)
+    if not grads:
+        raise ValueError("grads is empty")
+    dev = grads[0].device
+    n = grads[0].shape[0]
+    count = len(grads)
+    if outs is None:
+        outs = [torch.empty(g.shape[1], dtype=torch.float32, device=dev) for g in grads]
+    tensors = (GarTensor * count)()
+    for t, (g, o) in enumerate(zip(grads, outs)):
+        _dev_f32(g, "grads[%d]" % t)
+        gn, d, ld = _rows(g)
+        if gn != n or g.device != dev:
+            raise ValueError("every tensor must have the same number of rows and sit on the same device")
+        if not (o.is_cuda and o.dtype == torch.float32 and o.is_contiguous() and o.numel() == d):
+            raise TypeError("outs[%d] must be a contiguous CUDA float32 tensor of d elements" % t)
+        tensors[t].grads, tensors[t].out, tensors[t].d, tensors[t].ld = g.data_ptr(), o.data_ptr(), d, ld
+    if workspace is None:
+        workspace = torch.empty(gar_multi_workspace_bytes(rule, n, f, count), dtype=torch.uint8, device=dev)
+    p = GarMultiParams()
+    p.rule, p.n, p.f, p.count = _rule(rule), n, f, count
+    p.joint, p.even_median = 1 if joint else 0, _even(even_median)
+    p.tensors = tensors
+    p.workspace, p.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+    if dist_out is not None:
+        p.dist_out = dist_out.data_ptr()
+    if selection_out is not None:
+        p.selection_out = selection_out.data_ptr()
+    p.stream = _stream(stream)
+    with torch.cuda.device(dev):
+        st = lib().gar_aggregate_multi(C.byref(p))
+    _check(st, "gar_aggregate_multi")
+    return outs
 
 
 def gar_aggregate_host(rule, grads: torch.Tensor, f: int, out: torch.Tensor | None = None) -> torch.Tensor:

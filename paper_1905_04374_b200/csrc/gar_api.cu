@@ -1,7 +1,9 @@
 // C ABI of libgar: argument validation, workspace handling and the enqueue of
 // the three kernels (distances -> selection -> coordinate phase).
+#include <algorithm>
 #include <cstdio>
 #include <mutex>
+#include <vector>
 
 #include "gar_internal.cuh"
 #include "mbar.cuh"
@@ -170,6 +172,43 @@ __global__ void reduce_partials_kernel(const double* __restrict__ parts, int cou
     dist[idx] = s;
 }
 
+// ---- gar_aggregate_multi: workspace layout and the split of the work over CTAs
+// CTAs beyond one per tensor that a batched launch may spend, shared out by length.
+constexpr int kMultiK1Budget = 1024, kMultiK3Budget = 2048;
+
+struct MultiLayout {
+    size_t tickets, table, dist, sel, partials, total;     // byte offsets; `table` = the host-built arrays
+    size_t table_bytes;
+    // inside the table
+    size_t desc1, desc3, cta1, cta3;
+};
+
+MultiLayout multi_layout(int n, int count) {
+    MultiLayout L{};
+    size_t off = 0;
+    L.tickets = off;  off += gar::align256(size_t(count) * sizeof(unsigned int));
+    L.table = off;
+    size_t t = 0;
+    L.desc1 = t;  t += gar::align256(size_t(count) * sizeof(gar::MultiDesc));
+    L.desc3 = t;  t += gar::align256(size_t(count) * sizeof(gar::MultiDesc));
+    L.cta1 = t;   t += gar::align256(size_t(count + kMultiK1Budget) * sizeof(int));
+    L.cta3 = t;   t += gar::align256(size_t(count + kMultiK3Budget) * sizeof(int));
+    L.table_bytes = t;
+    off += t;
+    L.dist = off;     off += gar::align256(size_t(count + 1) * n * n * sizeof(double));
+    L.sel = off;      off += gar::align256(size_t(count) * sizeof(gar_selection_t));
+    L.partials = off; off += size_t(count + kMultiK1Budget) * gar::kPairSlots * sizeof(double);
+    L.total = off;
+    return L;
+}
+
+// CTAs of one tensor: one, plus its share (by length) of the budget, at most `useful`.
+int multi_ctas(int64_t d, double total_d, int budget, int64_t useful) {
+    int64_t c = 1 + int64_t(double(budget) * double(d) / total_d);
+    if (c > useful) c = useful;
+    return c < 1 ? 1 : int(c);
+}
+
 }  // namespace
 
 namespace gar {
@@ -331,6 +370,153 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
     const int nn = n * n;
     reduce_partials_kernel<<<(nn + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(parts, count, nn, dist);
     return cuda_status(cudaGetLastError());
+}
+
+size_t gar_multi_workspace_bytes(int rule, int n, int f, int count) {
+    if (basic_checks(rule, n, f, 1) != GAR_OK || count < 1) return 0;
+    return multi_layout(n, count).total;
+}
+
+int gar_aggregate_multi(const gar_multi_params_t* p) {
+    if (!p) return GAR_ERR_INVALID_ARG;
+    int rc = basic_checks(p->rule, p->n, p->f, 1);
+    if (rc != GAR_OK) return rc;
+    if (p->count < 1 || !p->tensors || (p->joint != 0 && p->joint != 1) || !even_median_ok(p->even_median))
+        return GAR_ERR_INVALID_ARG;
+    const int n = p->n, count = p->count;
+    for (int t = 0; t < count; ++t) {
+        const gar_tensor_t& x = p->tensors[t];
+        const int64_t ld = x.ld ? x.ld : x.d;
+        if (!x.grads || !x.out || x.d < 1 || ld < x.d) return GAR_ERR_INVALID_ARG;
+        if (overlaps(x.grads, (size_t(n - 1) * ld + x.d) * sizeof(float), x.out, size_t(x.d) * sizeof(float)))
+            return GAR_ERR_INVALID_ARG;
+    }
+    const MultiLayout L = multi_layout(n, count);
+    if (!p->workspace || reinterpret_cast<uintptr_t>(p->workspace) % 256 != 0 || p->workspace_bytes < L.total)
+        return GAR_ERR_WORKSPACE;
+    DeviceState* st = nullptr;
+    rc = device_state(&st, false);
+    if (rc != GAR_OK) return rc;
+    char* const ws = static_cast<char*>(p->workspace);
+    cudaStream_t stream = static_cast<cudaStream_t>(p->stream);
+    const int rule = p->rule, f = p->f;
+    const int theta = default_theta(rule, n, f), beta = beta_for(rule, theta, f);
+    const int preagg = (rule == GAR_MULTI_BULYAN || rule == GAR_MULTI_KRUM || rule == GAR_AVERAGE) ? 1 : 0;
+    const bool needs_dist = !(rule == GAR_AVERAGE || rule == GAR_MEDIAN);
+
+    // ---- the host-built table: descriptors in launch order (wide-access tensors first) and the CTA lists
+    double total_d = 0.0;
+    for (int t = 0; t < count; ++t) total_d += double(p->tensors[t].d);
+    std::vector<char> table(L.table_bytes, 0);
+    gar::MultiDesc* desc1 = reinterpret_cast<gar::MultiDesc*>(table.data() + L.desc1);
+    gar::MultiDesc* desc3 = reinterpret_cast<gar::MultiDesc*>(table.data() + L.desc3);
+    int* cta1 = reinterpret_cast<int*>(table.data() + L.cta1);
+    int* cta3 = reinterpret_cast<int*>(table.data() + L.cta3);
+    auto fill = [&](gar::MultiDesc& m, int t) {
+        const gar_tensor_t& x = p->tensors[t];
+        m.grads = x.grads; m.out = x.out; m.d = x.d; m.ld = x.ld ? x.ld : x.d; m.index = t; m.ctas = 1; m.cta_first = 0; m.pad = 0;
+    };
+    // distances: class 0 = rows 16-byte aligned, class 1 = the rest
+    const int slab = gar::distances_multi_slab(n);
+    int first1[3] = {0, 0, 0}, ctas1[2] = {0, 0};
+    {
+        int pos = 0, cta_off = 0;
+        for (int cls = 0; cls < 2; ++cls) {
+            first1[cls] = pos;
+            int cta = 0;
+            for (int t = 0; t < count; ++t) {
+                const gar_tensor_t& x = p->tensors[t];
+                const int64_t ld = x.ld ? x.ld : x.d;
+                const bool wide = reinterpret_cast<uintptr_t>(x.grads) % 16 == 0 && ld % 4 == 0;
+                if ((wide ? 0 : 1) != cls) continue;
+                gar::MultiDesc& m = desc1[pos];
+                fill(m, t);
+                m.ctas = multi_ctas(x.d, total_d, kMultiK1Budget, (x.d + slab - 1) / slab);
+                m.cta_first = cta;
+                for (int c = 0; c < m.ctas; ++c) cta1[cta_off + cta + c] = pos - first1[cls];
+                cta += m.ctas;
+                ++pos;
+            }
+            ctas1[cls] = cta;
+            cta_off += cta;
+        }
+        first1[2] = pos;
+    }
+    // coordinate phase: classes by vector width 4, 2, 1
+    int first3[4] = {0, 0, 0, 0}, ctas3[3] = {0, 0, 0};
+    const int widths[3] = {4, 2, 1};
+    {
+        int pos = 0, cta_off = 0;
+        for (int cls = 0; cls < 3; ++cls) {
+            first3[cls] = pos;
+            const int threads = gar::coordinate_multi_threads(n, theta, preagg, widths[cls]);
+            int cta = 0;
+            for (int t = 0; t < count; ++t) {
+                const gar_tensor_t& x = p->tensors[t];
+                const int64_t ld = x.ld ? x.ld : x.d;
+                if (gar::coordinate_multi_vec(x.grads, x.out, x.d, ld, theta, preagg) != widths[cls]) continue;
+                gar::MultiDesc& m = desc3[pos];
+                fill(m, t);
+                const int64_t per_cta = int64_t(threads) * widths[cls];
+                m.ctas = multi_ctas(x.d, total_d, kMultiK3Budget, (x.d + per_cta - 1) / per_cta);
+                m.cta_first = cta;
+                for (int c = 0; c < m.ctas; ++c) cta3[cta_off + cta + c] = pos - first3[cls];
+                cta += m.ctas;
+                ++pos;
+            }
+            ctas3[cls] = cta;
+            cta_off += cta;
+        }
+        first3[3] = pos;
+    }
+    if (int e = cuda_status(cudaMemcpyAsync(ws + L.table, table.data(), L.table_bytes, cudaMemcpyHostToDevice, stream))) return e;
+    // the pageable source has been staged when the copy call returns; `table` may go out of scope
+
+    const gar::MultiDesc* d_desc1 = reinterpret_cast<const gar::MultiDesc*>(ws + L.table + L.desc1);
+    const gar::MultiDesc* d_desc3 = reinterpret_cast<const gar::MultiDesc*>(ws + L.table + L.desc3);
+    const int* d_cta1 = reinterpret_cast<const int*>(ws + L.table + L.cta1);
+    const int* d_cta3 = reinterpret_cast<const int*>(ws + L.table + L.cta3);
+    double* ws_dist = reinterpret_cast<double*>(ws + L.dist);
+    gar_selection_t* sel = p->selection_out ? p->selection_out : reinterpret_cast<gar_selection_t*>(ws + L.sel);
+    // independent problems: the matrices go where the caller wants them; joint: the pieces stay in
+    // the workspace and their sum goes there
+    double* dist_each = (!p->joint && p->dist_out) ? p->dist_out : ws_dist;
+    double* dist_joint = p->dist_out ? p->dist_out : ws_dist + size_t(count) * n * n;
+
+    if (needs_dist) {
+        if (int e = cuda_status(cudaMemsetAsync(ws + L.tickets, 0, size_t(count) * sizeof(unsigned int), stream))) return e;
+        double* partials = reinterpret_cast<double*>(ws + L.partials);
+        unsigned int* tickets = reinterpret_cast<unsigned int*>(ws + L.tickets);
+        int cta_off = 0;
+        for (int cls = 0; cls < 2; ++cls) {
+            if (ctas1[cls] == 0) continue;
+            const cudaError_t err = gar::launch_distances_multi(d_desc1 + first1[cls], d_cta1 + cta_off, ctas1[cls], n, cls == 0,
+                                                                dist_each, partials + size_t(cta_off) * gar::kPairSlots, tickets, stream);
+            if (err != cudaSuccess) return cuda_status(err);
+            cta_off += ctas1[cls];
+        }
+        if (p->joint) {
+            const int nn = n * n;
+            reduce_partials_kernel<<<(nn + 255) / 256, 256, 0, stream>>>(dist_each, count, nn, dist_joint);
+            if (int e = cuda_status(cudaGetLastError())) return e;
+        }
+    }
+    {
+        const cudaError_t err = gar::launch_select(rule, p->joint ? dist_joint : dist_each, n, f, 0, theta, beta, 0, p->even_median,
+                                                   sel, stream, p->joint ? 1 : count);
+        if (err != cudaSuccess) return cuda_status(err);
+    }
+    {
+        int cta_off = 0;
+        for (int cls = 0; cls < 3; ++cls) {
+            if (ctas3[cls] == 0) continue;
+            const cudaError_t err = gar::launch_coordinate_multi(d_desc3 + first3[cls], d_cta3 + cta_off, ctas3[cls], n, theta, preagg,
+                                                                 widths[cls], sel, p->joint ? 0 : 1, stream);
+            if (err != cudaSuccess) return cuda_status(err);
+            cta_off += ctas3[cls];
+        }
+    }
+    return GAR_OK;
 }
 
 int gar_selftest_bounded_wait(unsigned int limit, long long* result, void* stream) {

@@ -47,6 +47,19 @@ constexpr int kSlotRowExp    = 2100;    // .. +63: the tensor-core kernel's fina
 constexpr int kSlotNonfinite = 2300;    // 2300, 2301: masks of rows that hold Inf or NaN
 constexpr int kSlotError     = 2302;    // a bounded wait gave up
 
+// One tensor of a batched call (gar_aggregate_multi): the device copy of a gar_tensor_t, the
+// tensor's place in the caller's array (it addresses the tensor's distance matrix, selection and
+// ticket) and its share of the launch: CTAs cta_first .. cta_first + ctas - 1 of a one-dimensional
+// grid, sized by the tensor's length.  A second array maps every CTA to its descriptor.
+struct MultiDesc {
+    const void* grads;
+    float*      out;
+    int64_t     d, ld;
+    int         index;
+    int         ctas, cta_first;
+    int         pad;
+};
+
 // Where the coordinate kernel puts a coordinate's result: the aggregate itself (out, may be null
 // when a step is fused) and/or an SGD step on x with optional momentum buffer v (Eq. 2).
 struct K3Out {
@@ -87,7 +100,7 @@ cudaError_t launch_distances_umma(const float* grads, int n, int64_t d, int64_t 
 
 // Scoring + iterative selection (and schedule construction) into *sel.
 cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,
-                          int median_of_agr, int even_median, gar_selection_t* sel, cudaStream_t stream);
+                          int median_of_agr, int even_median, gar_selection_t* sel, cudaStream_t stream, int count = 1);
 cudaError_t launch_schedule_only(gar_selection_t* sel, cudaStream_t stream);
 
 // Coordinate phase.
@@ -97,6 +110,21 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
 
 // One warp waits, bounded, on a barrier nobody arrives on; result[0] = status, result[1] = ns.
 cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t stream);
+
+// Batched launches over device arrays of descriptors: `total_ctas` CTAs, cta_desc[b] = the
+// descriptor CTA b works on.  Distances of every tensor into dist + index * n * n (difference-form
+// tiled kernel; `vec`: every tensor's rows are 16-byte aligned; partial sums at partials + b *
+// kPairSlots, tickets + index); coordinate phase of every tensor with the selection
+// sel + index * sel_stride (register kernel, `vec` coordinates per thread).
+cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, bool vec, double* dist,
+                                   double* partials, unsigned int* tickets, cudaStream_t stream);
+cudaError_t launch_coordinate_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
+                                    int vec, gar_selection_t* sel, int sel_stride, cudaStream_t stream);
+// Coordinates a CTA of the batched launches covers per pass over its tensor (to size `ctas`).
+int distances_multi_slab(int n);
+int coordinate_multi_threads(int n, int theta, int preagg, int vec);
+// The vector width launch_coordinate_multi may be given for a tensor of these addresses and sizes.
+int coordinate_multi_vec(const void* grads, const void* out, int64_t d, int64_t ld, int theta, int preagg);
 
 // cudaSuccess -> GAR_OK; anything else is remembered for gar_last_cuda_error and becomes GAR_ERR_CUDA
 int cuda_status(cudaError_t err);

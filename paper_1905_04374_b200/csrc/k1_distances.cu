@@ -78,32 +78,37 @@ template <int COUNT, int LANES> __device__ __forceinline__ int scatter_base(int 
 
 // Last-CTA reduction of the per-CTA partial sums (fixed order) -> `combine(slot, sum)`.
 template <typename F>
-__device__ __forceinline__ void reduce_partials(const double* partials, int nslots, int nthreads, F combine) {
+__device__ __forceinline__ void reduce_partials(const double* partials, int nslots, int nthreads, unsigned nctas, F combine) {
     for (int i = threadIdx.x; i < nslots; i += nthreads) {
         double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
         unsigned b = 0;
-        for (; b + 4 <= gridDim.x; b += 4) {
+        for (; b + 4 <= nctas; b += 4) {
             s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
             s1 += __ldcg(partials + size_t(b + 1) * kPairSlots + i);
             s2 += __ldcg(partials + size_t(b + 2) * kPairSlots + i);
             s3 += __ldcg(partials + size_t(b + 3) * kPairSlots + i);
         }
-        for (; b < gridDim.x; ++b) s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
+        for (; b < nctas; ++b) s0 += __ldcg(partials + size_t(b) * kPairSlots + i);
         combine(i, (s0 + s1) + (s2 + s3));
     }
 }
+template <typename F>
+__device__ __forceinline__ void reduce_partials(const double* partials, int nslots, int nthreads, F combine) {
+    reduce_partials(partials, nslots, nthreads, gridDim.x, combine);
+}
 
-// Returns true in exactly one CTA: the last one to arrive.  All of this CTA's
-// partial sums must have been written before the call.
-__device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) {
+// Returns true in exactly one of the `nctas` CTAs that share the ticket: the last one to arrive.
+// All of this CTA's partial sums must have been written before the call.
+__device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket, unsigned nctas) {
     __shared__ int is_last;
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    if (threadIdx.x == 0) is_last = (atomicAdd(ticket, 1u) == nctas - 1);
     __syncthreads();
     if (is_last) __threadfence();
     return is_last != 0;
 }
+__device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) { return last_cta_ticket(ticket, gridDim.x); }
 
 // ---- pieces the two direct kernels (n <= 16) share
 // acc[p] += sum_v (x[i][v] - x[j][v])^2 over the pairs p = (0,1), (0,2), .., (0,N-1), (1,2), ..
@@ -611,10 +616,23 @@ template <int NB, bool VEC, int ES = 4>
 __global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
 k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
-         const unsigned int* __restrict__ gate, int dtype) {
+         const unsigned int* __restrict__ gate, int dtype, const MultiDesc* __restrict__ multi,
+         const int* __restrict__ cta_desc) {
     // launched behind the tensor-core kernel, this one only runs if that kernel rejected its own
     // result (the gate word is written before this grid starts: same stream)
     if (gate != nullptr && *gate == 0u) return;
+    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
+    if (multi != nullptr) {                       // a batch: CTA b works on the tensor of descriptor cta_desc[b]
+        const MultiDesc t = multi[cta_desc[blockIdx.x]];
+        g = static_cast<const float*>(t.grads);
+        d = t.d;
+        ld = t.ld;
+        dist += size_t(t.index) * n * n;
+        partials += size_t(t.cta_first) * kPairSlots;
+        ticket += t.index;
+        bx = blockIdx.x - unsigned(t.cta_first);
+        gx = unsigned(t.ctas);
+    }
     using D = K1Dims<NB>;
     constexpr int NSTAGE = D::NSTAGE;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -651,7 +669,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
     for (int i = 0; i < 64; ++i) acc[i] = 0.0f;
 
     const int64_t nslabs = (d + D::TK - 1) / D::TK;
-    const int64_t first = blockIdx.x, step = gridDim.x;
+    const int64_t first = bx, step = gx;
     const int64_t mine = first < nslabs ? (nslabs - first + step - 1) / step : 0;
 
     auto flush = [&]() {
@@ -746,15 +764,15 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
     __syncthreads();
 
     // CTA partial: sum the groups in order, one fp64 per (tile, pair)
-    double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
+    double* my_partial = partials + size_t(bx) * kPairSlots;
     for (int i = tid; i < D::TILES * 64; i += D::THREADS) {
         double s = 0.0;
 #pragma unroll 1
         for (int gq = 0; gq < D::G; ++gq) s += sums[size_t(gq) * D::TILES * 64 + i];
         my_partial[i] = s;
     }
-    if (!last_cta_ticket(ticket)) return;
-    reduce_partials(partials, D::TILES * 64, D::THREADS, [&](int i, double s) {
+    if (!last_cta_ticket(ticket, gx)) return;
+    reduce_partials(partials, D::TILES * 64, D::THREADS, gx, [&](int i, double s) {
         const int t = i >> 6, hi = (i & 63) >> 3, lo = i & 7;
         int ra, rb;
         if (t < D::OFFJ) {
@@ -779,7 +797,7 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
     for (int i = tid; i < n; i += D::THREADS) dist[i * n + i] = 0.0;
     if (tid == 0) {
         *ticket = 0u;                           // ready for the next call
-        if (gate == nullptr) *path_word = kPathDifference;
+        if (gate == nullptr && multi == nullptr) *path_word = kPathDifference;
     }
 }
 
@@ -824,7 +842,26 @@ cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* d
                                       (d + D::TK - 1) / D::TK, &grid);
     if (err != cudaSuccess) return err;
     k1_tiled<NB, VEC, ES><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket(),
-                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr, dtype);
+                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr, dtype, nullptr, nullptr);
+    return cudaGetLastError();
+}
+
+// A batch of tensors (fp32): one CTA per entry of cta_desc.
+template <int NB, bool VEC>
+cudaError_t launch_tiled_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, double* dist, double* partials,
+                               unsigned int* tickets, cudaStream_t stream) {
+    using D = K1Dims<NB>;
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (!(dev >= 0 && dev < 64 && configured[dev])) {
+        err = cudaFuncSetAttribute(k1_tiled<NB, VEC, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(D::SMEM_BYTES));
+        if (err != cudaSuccess) return err;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    k1_tiled<NB, VEC, 4><<<unsigned(total_ctas), D::THREADS, D::SMEM_BYTES, stream>>>(
+        nullptr, n, 0, 0, dist, partials, tickets, nullptr, nullptr, GAR_F32, desc, cta_desc);
     return cudaGetLastError();
 }
 
@@ -907,6 +944,27 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
 #undef GAR_K1_DIRECT
 #undef GAR_K1_TILED
     return cudaErrorInvalidValue;
+}
+
+cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, bool vec, double* dist,
+                                   double* partials, unsigned int* tickets, cudaStream_t stream) {
+#define GAR_K1_MULTI(NBV)                                                                                              \
+    case NBV:                                                                                                          \
+        return vec ? launch_tiled_multi<NBV, true>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream)      \
+                   : launch_tiled_multi<NBV, false>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream);
+    switch ((n + 7) / 8) {
+        GAR_K1_MULTI(1) GAR_K1_MULTI(2) GAR_K1_MULTI(3) GAR_K1_MULTI(4) GAR_K1_MULTI(5) GAR_K1_MULTI(6)
+        GAR_K1_MULTI(7) GAR_K1_MULTI(8)
+    }
+#undef GAR_K1_MULTI
+    return cudaErrorInvalidValue;
+}
+
+int distances_multi_slab(int n) {
+    switch ((n + 7) / 8) {
+        case 1: return K1Dims<1>::TK; case 2: return K1Dims<2>::TK; case 3: return K1Dims<3>::TK; case 4: return K1Dims<4>::TK;
+        case 5: return K1Dims<5>::TK; case 6: return K1Dims<6>::TK; case 7: return K1Dims<7>::TK; default: return K1Dims<8>::TK;
+    }
 }
 
 // 16-bit gradients (bfloat16 / binary16): the staged direct kernel for n <= 16 when the rows are

@@ -195,6 +195,8 @@ __device__ void build_schedule(gar_selection_t* sel, PlanSmem& ps) {
 __global__ void __launch_bounds__(K2_THREADS)
 k2_select(const double* __restrict__ dist, gar_selection_t* __restrict__ sel, int rule, int n, int f,
           int m_user, int theta, int beta, int median_of_agr, int even_median) {
+    dist += size_t(blockIdx.x) * n * n;           // a batch: CTA b takes the b-th matrix and selection
+    sel += blockIdx.x;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     K2Smem& sm = *reinterpret_cast<K2Smem*>(smem_raw);
     __shared__ PlanSmem plan_smem;
@@ -342,7 +344,7 @@ __global__ void __launch_bounds__(64) k2_schedule_only(gar_selection_t* sel) {
 }  // namespace
 
 cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int theta, int beta,
-                          int median_of_agr, int even_median, gar_selection_t* sel, cudaStream_t stream) {
+                          int median_of_agr, int even_median, gar_selection_t* sel, cudaStream_t stream, int count) {
     static bool configured[64] = {false};
     int dev = 0;
     cudaError_t err = cudaGetDevice(&dev);
@@ -352,7 +354,7 @@ cudaError_t launch_select(int rule, const double* dist, int n, int f, int m, int
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k2_select<<<1, K2_THREADS, sizeof(K2Smem), stream>>>(dist, sel, rule, n, f, m, theta, beta, median_of_agr, even_median);
+    k2_select<<<unsigned(count), K2_THREADS, sizeof(K2Smem), stream>>>(dist, sel, rule, n, f, m, theta, beta, median_of_agr, even_median);
     return cudaGetLastError();
 }
 

@@ -365,17 +365,33 @@ __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* _
 // Coordinates [t_begin, t_end), V per thread; (t_end - t_begin) % V == 0 and the
 // V-vectors at g + row*ld + t and out + t are naturally aligned.
 // Dynamic shared memory (PREAGG only): (loose_cap + GAR_MAX_SAVED) * blockDim * V floats.
+// A batch (multi != nullptr): CTA b takes its tensor (gradients, output, d, row stride) from the
+// descriptor multi[cta_desc[b]], the selection sel + index * sel_stride, and is one of the
+// descriptor's `ctas` CTAs.
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(K3_THREADS)
 k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin, int64_t t_end, int64_t ld,
-              gar_selection_t* __restrict__ sel, const K3Out out, int loose_cap, int dtype) {
+              gar_selection_t* __restrict__ sel, K3Out out, int loose_cap, int dtype,
+              const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, int sel_stride) {
     __shared__ K3Plan plan;
     extern __shared__ __align__(16) float k3_dyn[];
+    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
+    if (multi != nullptr) {
+        const MultiDesc t = multi[cta_desc[blockIdx.x]];
+        g = static_cast<const float*>(t.grads);
+        t_begin = 0;
+        t_end = t.d;
+        ld = t.ld;
+        out.out = t.out;
+        sel += size_t(t.index) * sel_stride;
+        bx = blockIdx.x - unsigned(t.cta_first);
+        gx = unsigned(t.ctas);
+    }
     const int status = k3_check(sel, n, theta_arg, PREAGG);
     if (status != GAR_OK) {                       // nothing usable: the output says so
-        for (int64_t t = t_begin + int64_t(blockIdx.x) * blockDim.x + threadIdx.x; t < t_end; t += int64_t(gridDim.x) * blockDim.x)
+        for (int64_t t = t_begin + int64_t(bx) * blockDim.x + threadIdx.x; t < t_end; t += int64_t(gx) * blockDim.x)
             k3_store_nan(out, t);
-        if (blockIdx.x == 0 && threadIdx.x == 0 && sel->status == GAR_OK) sel->status = status;
+        if (bx == 0 && threadIdx.x == 0 && sel->status == GAR_OK) sel->status = status;
         return;
     }
     load_plan(plan, sel, ld, P, PREAGG, loose_cap);
@@ -394,8 +410,8 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
     const unsigned long long chain_mask = plan.chain_mask, corr_mask = plan.corr_mask;
 
     const int64_t nvec = (t_end - t_begin) / V;
-    for (int64_t vi = int64_t(blockIdx.x) * nthreads + threadIdx.x; vi < nvec;
-         vi += int64_t(gridDim.x) * nthreads) {
+    for (int64_t vi = int64_t(bx) * nthreads + threadIdx.x; vi < nvec;
+         vi += int64_t(gx) * nthreads) {
         const int64_t t = t_begin + vi * V;
         const int esh = dtype == GAR_F32 ? 2 : 1;             // log2 of the element size
         float e[P][V], a[P][V];
@@ -410,7 +426,7 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
         }
         // few slots: the kernel waits on memory more than it computes, so pull the next
         // iteration's lines into L1 meanwhile (with many slots the extra instructions cost more)
-        const int64_t vnext = vi + int64_t(gridDim.x) * nthreads;
+        const int64_t vnext = vi + int64_t(gx) * nthreads;
         if (P <= 12 && vnext < nvec) {
             const char* gn = reinterpret_cast<const char*>(g) + ((t_begin + vnext * V) << esh);
 #pragma unroll
@@ -521,5 +537,9 @@ template <int P>
 cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_selection_t* sel, int theta, int preagg,
                         int vec, int bulk_ctas, const K3Out& out, int sm_count, cudaStream_t stream, int dtype);
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
+template <int P>
+cudaError_t launch_k3_multi_p(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg, int vec,
+                              gar_selection_t* sel, int sel_stride, cudaStream_t stream);
+template <int P> int k3_multi_threads(int n, int preagg, int vec);
 
 }  // namespace gar

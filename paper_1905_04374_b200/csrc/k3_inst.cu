@@ -109,10 +109,10 @@ static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, 
         const int64_t cap = int64_t(sm_count) * 8;
         if (blocks > cap) blocks = cap;
         k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, n, theta, t0, d_vec, ld, sel, out,
-                                                                                         loose_cap, dtype);
+                                                                                         loose_cap, dtype, nullptr, nullptr, 0);
     }
     if (d_vec < d) {   // ragged tail (only when ld > d): scalar kernel on the last d % V coordinates
-        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap, dtype);
+        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap, dtype, nullptr, nullptr, 0);
     }
     return cudaGetLastError();
 }
@@ -141,6 +141,63 @@ cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_
     if constexpr (kWide) if (vec == 4) return run<K3_P, false, 4>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
     if (vec == 2) return run<K3_P, false, 2>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
     return run<K3_P, false, 1>(g, n, theta, t0, d, ld, sel, out, sm_count, stream, dtype);
+}
+
+// A batch of tensors through the register kernel, V coordinates per thread (every tensor's d, row
+// stride and addresses allow V-wide accesses): one CTA per entry of cta_desc.
+template <int P, bool PREAGG, int V>
+static cudaError_t run_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, gar_selection_t* sel,
+                             int sel_stride, cudaStream_t stream) {
+    constexpr bool EXACT = (K3_EXACT != 0);
+    int threads = K3_THREADS;
+    size_t smem = 0;
+    const int loose_cap = n < K3_LOOSE_CAP ? n : K3_LOOSE_CAP;
+    if (PREAGG) {
+        preagg_shape(loose_cap, V, &threads, &smem);
+        static bool configured[64] = {false};      // per device, for this instantiation
+        int dev = 0;
+        cudaError_t err = cudaGetDevice(&dev);
+        if (err != cudaSuccess) return err;
+        if (!(dev >= 0 && dev < 64 && configured[dev])) {
+            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+            if (err != cudaSuccess) return err;
+            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, V>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                       cudaSharedmemCarveoutMaxShared);
+            if (err != cudaSuccess) return err;
+            if (dev >= 0 && dev < 64) configured[dev] = true;
+        }
+    }
+    const K3Out none{nullptr, nullptr, nullptr, 0.0f, 0.0f};
+    k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(total_ctas), threads, smem, stream>>>(
+        nullptr, n, theta, 0, 0, 0, sel, none, loose_cap, GAR_F32, desc, cta_desc, sel_stride);
+    return cudaGetLastError();
+}
+
+// 4-wide vectors are only compiled for small slot counts (register budget)
+static inline int multi_vec(int vec) { return (vec == 4 && K3_P > 8) ? 2 : vec; }
+
+template <>
+cudaError_t launch_k3_multi_p<K3_P>(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
+                                    int vec, gar_selection_t* sel, int sel_stride, cudaStream_t stream) {
+    constexpr bool kWide = (K3_P <= 8);
+    vec = multi_vec(vec);
+    if (preagg) {
+        if constexpr (kWide) if (vec == 4) return run_multi<K3_P, true, 4>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, stream);
+        if (vec == 2) return run_multi<K3_P, true, 2>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, stream);
+        return run_multi<K3_P, true, 1>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, stream);
+    }
+    if constexpr (kWide) if (vec == 4) return run_multi<K3_P, false, 4>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, stream);
+    if (vec == 2) return run_multi<K3_P, false, 2>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, stream);
+    return run_multi<K3_P, false, 1>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, stream);
+}
+
+// Threads per CTA of that launch.
+template <>
+int k3_multi_threads<K3_P>(int n, int preagg, int vec) {
+    int threads = K3_THREADS;
+    size_t smem = 0;
+    if (preagg) preagg_shape(n < K3_LOOSE_CAP ? n : K3_LOOSE_CAP, multi_vec(vec), &threads, &smem);
+    return threads;
 }
 
 // CTAs per SM the staged kernel would get for n gradients and theta slots (0: it cannot run).

@@ -42,7 +42,9 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
                    'offsetof(gar_selection_t,add_pos), offsetof(gar_selection_t,scores), sizeof(gar_params_t),'
                    'offsetof(gar_selection_t,even_median), offsetof(gar_selection_t,winners),'
                    'offsetof(gar_params_t,even_median), offsetof(gar_params_t,distance_mode));'
-                   'printf("%zu %zu\\n", offsetof(gar_params_t,sgd_params), offsetof(gar_params_t,sgd_lr));}')
+                   'printf("%zu %zu\\n", offsetof(gar_params_t,sgd_params), offsetof(gar_params_t,sgd_lr));'
+                   'printf("%zu %zu %zu %zu\\n", sizeof(gar_tensor_t), sizeof(gar_multi_params_t),'
+                   'offsetof(gar_multi_params_t,tensors), offsetof(gar_multi_params_t,stream));}')
     exe = tmp_path / "sz"
     subprocess.check_call(["g++", "-I" + os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(v) for v in subprocess.check_output([str(exe)]).split()]
@@ -50,11 +52,13 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
     P = pkg.GarParams
     assert got == [C.sizeof(S), S.sets.offset, S.nu.offset, S.add_pos.offset, S.scores.offset,
                    C.sizeof(P), S.even_median.offset, S.winners.offset, P.even_median.offset, P.distance_mode.offset,
-                   P.sgd_params.offset, P.sgd_lr.offset]
+                   P.sgd_params.offset, P.sgd_lr.offset,
+                   C.sizeof(pkg.GarTensor), C.sizeof(pkg.GarMultiParams), pkg.GarMultiParams.tensors.offset,
+                   pkg.GarMultiParams.stream.offset]
 
 
 def test_version_and_strings(pkg):
-    assert pkg.gar_version() == 102
+    assert pkg.gar_version() == 103
     assert pkg.gar_status_string(0) == "ok"
     assert pkg.gar_last_cuda_error() == (0, "cudaSuccess")      # nothing has failed in this thread yet
     assert "4f+3" in pkg.gar_status_string(2)
@@ -118,6 +122,31 @@ def test_errors_before_any_launch(pkg):
     p.sgd_params = (1 << 30) + 40                                          # parameters overlapping the output
     assert L.gar_aggregate_ex(C.byref(p)) == 1
     assert L.gar_pairwise_distances_mode(fake, 11, 100, 100, fake, None, 0, 5, None) == 1
+    # the batched call: argument and workspace errors come before any CUDA call
+    assert L.gar_aggregate_multi(None) == 1
+    assert pkg.gar_multi_workspace_bytes("multi_bulyan", 11, 2, 3) > 0
+    assert pkg.gar_multi_workspace_bytes("multi_bulyan", 10, 2, 3) == 0
+    assert pkg.gar_multi_workspace_bytes("multi_bulyan", 11, 2, 0) == 0
+    tensors = (pkg.GarTensor * 2)()
+    tensors[0].grads, tensors[0].out, tensors[0].d, tensors[0].ld = 4096, 1 << 30, 100, 100
+    tensors[1].grads, tensors[1].out, tensors[1].d, tensors[1].ld = 1 << 20, 1 << 31, 7, 0
+    q = pkg.GarMultiParams()
+    q.rule, q.n, q.f, q.count, q.tensors = 5, 11, 2, 2, tensors
+    assert L.gar_aggregate_multi(C.byref(q)) == 4                          # no workspace
+    q.workspace, q.workspace_bytes = 1 << 32, 1024                         # too small
+    assert L.gar_aggregate_multi(C.byref(q)) == 4
+    q.n = 10
+    assert L.gar_aggregate_multi(C.byref(q)) == 2                          # n < 4f + 3
+    q.n, q.count = 11, 0
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
+    q.count, q.joint = 2, 2
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
+    q.joint = 0
+    tensors[1].ld = 5                                                      # ld < d
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
+    tensors[1].ld = 0
+    tensors[0].out = 4096 + 400                                            # out overlaps its own gradients
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
     assert L.gar_reduce_partials(fake, 0, 11, fake, None) == 1 and L.gar_reduce_partials(fake, 2, 65, fake, None) == 3
     assert L.gar_select(5, fake, 11, 2, 0, 0, 0, 3, fake, None) == 1       # unknown even-median mode
     assert L.gar_selftest_bounded_wait(0, fake, None) == 1
