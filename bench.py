@@ -331,6 +331,77 @@ def measure_workload(pkg, cfg, dev, steps, warmup, world, local, d=None, variant
     return res, G
 
 
+def resnet18_lengths():
+    """Parameter-tensor lengths of an 18-layer residual network with 1000 outputs (62 tensors,
+    11,689,512 parameters): convolution weights, the two vectors of every normalisation layer,
+    the final linear layer."""
+    out = [64 * 3 * 7 * 7, 64, 64]
+    cin = 64
+    for cout in (64, 128, 256, 512):
+        for block in range(2):
+            first = block == 0 and cout != 64
+            out += [cout * cin * 9, cout, cout, cout * cout * 9, cout, cout]
+            if first:
+                out += [cout * cin, cout, cout]
+            cin = cout
+    return out + [512 * 1000, 1000]
+
+
+# Per-layer mixes the batched call is timed on: (n, f, tensor lengths).
+LAYER_MIXES = {
+    # a network of two convolutions and two linear layers with d = 431,080 parameters (the size of
+    # the model in Section 5), as weight and bias tensors: 5x5 kernels, 1 -> 20 -> 50 channels,
+    # 800 -> 500 -> 10 units
+    "cnn_d431080": (11, 2, [500, 20, 25_000, 50, 400_000, 500, 5_000, 10]),
+    "resnet18_lengths": (15, 3, resnet18_lengths()),
+}
+
+
+def measure_multi(pkg, dev, reps=20):
+    """gar_aggregate_multi (independent problems, and the tensors as one gradient) against one
+    gar_aggregate_ex per tensor, on per-layer tensors; CUDA events, inputs resident."""
+    import torch
+    results = []
+    for name, (n, f, dims) in LAYER_MIXES.items():
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(workloads_seed(name))
+        parts = [torch.randn(n, d, generator=gen, device=dev, dtype=torch.float32) for d in dims]
+        for g in parts:
+            g[n - f:] += 20.0
+        count = len(parts)
+        outs = [torch.empty(d, dtype=torch.float32, device=dev) for d in dims]
+        ws = torch.empty(pkg.gar_multi_workspace_bytes("multi_bulyan", n, f, count), dtype=torch.uint8, device=dev)
+        entry = {"mix": name, "n": n, "f": f, "tensors": count, "d_total": int(sum(dims)), "rule": "multi_bulyan"}
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        entry["ms_multi_independent"] = timed(lambda: pkg.gar_aggregate_multi("multi_bulyan", parts, f, outs=outs, workspace=ws))
+        entry["ms_multi_joint"] = timed(lambda: pkg.gar_aggregate_multi("multi_bulyan", parts, f, outs=outs, workspace=ws, joint=True))
+        entry["ms_one_call_per_tensor"] = timed(lambda: [pkg.gar_aggregate_ex("multi_bulyan", g, f, out=o) for g, o in zip(parts, outs)])
+        flat = torch.cat(parts, dim=1).contiguous()
+        flat_out = torch.empty(flat.shape[1], dtype=torch.float32, device=dev)
+        entry["ms_one_call_on_the_concatenation"] = timed(lambda: pkg.gar_aggregate_ex("multi_bulyan", flat, f, out=flat_out))
+        entry["hbm_floor_ms"] = 4.0 * sum(dims) * (2 * n + 1) / (measured_hbm_peak()[0] * 1e9) * 1e3
+        results.append(entry)
+        del parts, outs, flat, flat_out, ws
+        torch.cuda.empty_cache()
+    return results
+
+
+def workloads_seed(name):
+    return 20_190_509 + sum(ord(c) for c in name)
+
+
 def run_e2e(pkg, cfg, G, steps):
     """The same aggregation through the host entry point: pinned host buffers, both copies inside
     the timed region."""
@@ -453,6 +524,10 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     cfg = args.config
+    if args.multi_only:
+        if rank == 0:
+            print(json.dumps({"multi_tensor": measure_multi(pkg, dev)}), flush=True)
+        return
     if world > 1 or args.force_sharded:
         run_sharded(pkg, args, dev, world, rank, local)
         dist.destroy_process_group()
@@ -493,6 +568,7 @@ def run_ours(args):
                 entry.pop("elapsed_ms")
             per_config.append(entry)
 
+    multi = None if args.no_multi else measure_multi(pkg, dev)
     cpu = None if args.no_cpu_baseline else cpu_baseline(cfg, args.cpu_sample or CPU_SAMPLE[cfg])
 
     line = {
@@ -506,7 +582,7 @@ def run_ours(args):
                    "l2": "input (%.2f GB) larger than L2; no flush" % (4e-9 * n * d) if 4 * n * d > 2.6e8
                    else "input fits L2; not flushed between steps"},
         "roofline": main["roofline"], "path": main["path"], "kernels": main["kernels"],
-        "variant_bulyan": main.get("variant_bulyan"), "per_config": per_config, "cpu_baseline": cpu, "e2e": e2e,
+        "variant_bulyan": main.get("variant_bulyan"), "per_config": per_config, "multi_tensor": multi, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": launches_per_aggregation(n, d, main["theta"]) * args.steps, "clocks": main["clocks"],
     }
     print(json.dumps(line), flush=True)
@@ -529,6 +605,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--no-multi", action="store_true", help="skip the timing of the batched per-layer call")
+    ap.add_argument("--multi-only", action="store_true", help="print the batched per-layer call's timings and exit")
     ap.add_argument("--quick", action="store_true", help="device-side numbers of the chosen workload only")
     ap.add_argument("--distance-mode", default="auto", choices=["auto", "difference"],
                     help="difference: the fp32 difference-form distance kernels instead of the tensor-core one")
@@ -540,7 +618,7 @@ def main():
     if args.dtype != "f32":
         args.quick = True
     if args.quick:
-        args.no_e2e = args.no_cpu_baseline = args.no_per_config = True
+        args.no_e2e = args.no_cpu_baseline = args.no_per_config = args.no_multi = True
     if args.impl == "reference":
         run_reference(args)
     else:

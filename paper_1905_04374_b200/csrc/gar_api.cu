@@ -173,7 +173,8 @@ __global__ void reduce_partials_kernel(const double* __restrict__ parts, int cou
 }
 
 // ---- gar_aggregate_multi: workspace layout and the split of the work over CTAs
-// CTAs beyond one per tensor that a batched launch may spend, shared out by length.
+// CTAs beyond one per tensor that a batched launch may spend, shared out by length: upper bounds
+// (they size the workspace); a call spends about one wave of resident CTAs, by the SM count.
 constexpr int kMultiK1Budget = 1024, kMultiK3Budget = 2048;
 
 struct MultiLayout {
@@ -404,6 +405,9 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     const int preagg = (rule == GAR_MULTI_BULYAN || rule == GAR_MULTI_KRUM || rule == GAR_AVERAGE) ? 1 : 0;
     const bool needs_dist = !(rule == GAR_AVERAGE || rule == GAR_MEDIAN);
 
+    // one wave: the ring kernel keeps three CTAs per SM resident, the tiled kernel two, the register kernel six
+    const int k1_budget = std::min(kMultiK1Budget, (n <= 16 ? 3 : 2) * st->sm_count);
+    const int k3_budget = std::min(kMultiK3Budget, 6 * st->sm_count);
     // ---- the host-built table: descriptors in launch order (wide-access tensors first) and the CTA lists
     double total_d = 0.0;
     for (int t = 0; t < count; ++t) total_d += double(p->tensors[t].d);
@@ -416,22 +420,24 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         const gar_tensor_t& x = p->tensors[t];
         m.grads = x.grads; m.out = x.out; m.d = x.d; m.ld = x.ld ? x.ld : x.d; m.index = t; m.ctas = 1; m.cta_first = 0; m.pad = 0;
     };
-    // distances: class 0 = rows 16-byte aligned, class 1 = the rest
-    const int slab = gar::distances_multi_slab(n);
-    int first1[3] = {0, 0, 0}, ctas1[2] = {0, 0};
+    // distances: classes by the alignment of the rows, 16 / 8 / 4 bytes
+    const int widths[3] = {4, 2, 1};
+    int first1[4] = {0, 0, 0, 0}, ctas1[3] = {0, 0, 0};
     {
         int pos = 0, cta_off = 0;
-        for (int cls = 0; cls < 2; ++cls) {
+        for (int cls = 0; cls < 3; ++cls) {
             first1[cls] = pos;
+            const int chunk = gar::distances_multi_chunk(n, widths[cls]);
             int cta = 0;
             for (int t = 0; t < count; ++t) {
                 const gar_tensor_t& x = p->tensors[t];
                 const int64_t ld = x.ld ? x.ld : x.d;
-                const bool wide = reinterpret_cast<uintptr_t>(x.grads) % 16 == 0 && ld % 4 == 0;
-                if ((wide ? 0 : 1) != cls) continue;
+                const uintptr_t addr = reinterpret_cast<uintptr_t>(x.grads);
+                const int mine = (addr % 16 == 0 && ld % 4 == 0) ? 0 : ((addr % 8 == 0 && ld % 2 == 0) ? 1 : 2);
+                if (mine != cls) continue;
                 gar::MultiDesc& m = desc1[pos];
                 fill(m, t);
-                m.ctas = multi_ctas(x.d, total_d, kMultiK1Budget, (x.d + slab - 1) / slab);
+                m.ctas = multi_ctas(x.d, total_d, k1_budget, (x.d + chunk - 1) / chunk);
                 m.cta_first = cta;
                 for (int c = 0; c < m.ctas; ++c) cta1[cta_off + cta + c] = pos - first1[cls];
                 cta += m.ctas;
@@ -440,11 +446,10 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
             ctas1[cls] = cta;
             cta_off += cta;
         }
-        first1[2] = pos;
+        first1[3] = pos;
     }
     // coordinate phase: classes by vector width 4, 2, 1
     int first3[4] = {0, 0, 0, 0}, ctas3[3] = {0, 0, 0};
-    const int widths[3] = {4, 2, 1};
     {
         int pos = 0, cta_off = 0;
         for (int cls = 0; cls < 3; ++cls) {
@@ -458,7 +463,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
                 gar::MultiDesc& m = desc3[pos];
                 fill(m, t);
                 const int64_t per_cta = int64_t(threads) * widths[cls];
-                m.ctas = multi_ctas(x.d, total_d, kMultiK3Budget, (x.d + per_cta - 1) / per_cta);
+                m.ctas = multi_ctas(x.d, total_d, k3_budget, (x.d + per_cta - 1) / per_cta);
                 m.cta_first = cta;
                 for (int c = 0; c < m.ctas; ++c) cta3[cta_off + cta + c] = pos - first3[cls];
                 cta += m.ctas;
@@ -488,9 +493,9 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         double* partials = reinterpret_cast<double*>(ws + L.partials);
         unsigned int* tickets = reinterpret_cast<unsigned int*>(ws + L.tickets);
         int cta_off = 0;
-        for (int cls = 0; cls < 2; ++cls) {
+        for (int cls = 0; cls < 3; ++cls) {
             if (ctas1[cls] == 0) continue;
-            const cudaError_t err = gar::launch_distances_multi(d_desc1 + first1[cls], d_cta1 + cta_off, ctas1[cls], n, cls == 0,
+            const cudaError_t err = gar::launch_distances_multi(d_desc1 + first1[cls], d_cta1 + cta_off, ctas1[cls], n, widths[cls],
                                                                 dist_each, partials + size_t(cta_off) * gar::kPairSlots, tickets, stream);
             if (err != cudaSuccess) return cuda_status(err);
             cta_off += ctas1[cls];

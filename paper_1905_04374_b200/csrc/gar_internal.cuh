@@ -112,16 +112,17 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld,
 cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t stream);
 
 // Batched launches over device arrays of descriptors: `total_ctas` CTAs, cta_desc[b] = the
-// descriptor CTA b works on.  Distances of every tensor into dist + index * n * n (difference-form
-// tiled kernel; `vec`: every tensor's rows are 16-byte aligned; partial sums at partials + b *
-// kPairSlots, tickets + index); coordinate phase of every tensor with the selection
+// descriptor CTA b works on.  Distances of every tensor into dist + index * n * n (difference
+// form: the ring kernel up to 16 rows, the tiled kernel beyond; `vec` = 4, 2, 1: every tensor's
+// rows are 16-byte / 8-byte / 4-byte aligned; partial sums at partials + b * kPairSlots, tickets +
+// index); coordinate phase of every tensor with the selection
 // sel + index * sel_stride (register kernel, `vec` coordinates per thread).
-cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, bool vec, double* dist,
+cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int vec, double* dist,
                                    double* partials, unsigned int* tickets, cudaStream_t stream);
 cudaError_t launch_coordinate_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
                                     int vec, gar_selection_t* sel, int sel_stride, cudaStream_t stream);
-// Coordinates a CTA of the batched launches covers per pass over its tensor (to size `ctas`).
-int distances_multi_slab(int n);
+// Sizes that decide how many CTAs a tensor gets in the batched launches.
+int distances_multi_chunk(int n, int vec);
 int coordinate_multi_threads(int n, int theta, int preagg, int vec);
 // The vector width launch_coordinate_multi may be given for a tensor of these addresses and sizes.
 int coordinate_multi_vec(const void* grads, const void* out, int64_t d, int64_t ld, int theta, int preagg);

@@ -111,6 +111,105 @@ __device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket, unsigned n
 __device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) { return last_cta_ticket(ticket, gridDim.x); }
 
 // ---- pieces the two direct kernels (n <= 16) share
+// The arithmetic.  Rows are taken two at a time: R_a = (x_2a, x_2a+1) sits in one 64-bit register
+// pair, and one packed subtract plus one packed multiply-add (sub.f32x2, fma.rn.f32x2: two IEEE
+// fp32 operations each, one issue slot) serve two pairs at once --
+//     R_a - R_b          -> pairs (2a, 2b), (2a+1, 2b+1)
+//     R_a - swap(R_b)    -> pairs (2a, 2b+1), (2a+1, 2b)
+//     R_a - (x_N-1, x_N-1) for the unpaired last row of an odd N
+// and the pair (2a, 2a+1) inside a row pair takes scalar instructions: 112 issue slots per
+// coordinate for 15 rows instead of 210.
+template <int N> struct K1Pairs {
+    static constexpr int NP = N * (N - 1) / 2;
+    static constexpr int NPAD = (NP + 31) / 32 * 32;
+    static constexpr int NF = N / 2;                               // whole row pairs
+    static constexpr int NBLK = NF * (NF - 1) / 2;                 // blocks of two row pairs
+    static constexpr int NPK = 2 * NBLK + (N % 2 ? NF : 0);        // packed accumulators
+    static_assert(2 * NPK + NF == NP, "accumulator slots");
+};
+
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long p, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+// acc += (a - b)^2 in both lanes
+__device__ __forceinline__ void sqdiff2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
+    unsigned long long df;
+    asm("sub.f32x2 %0, %1, %2;" : "=l"(df) : "l"(a), "l"(b));
+    asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc) : "l"(df));
+}
+
+// The accumulators of one thread.  Slot order (the order of the CTA's partial sums):
+//   for a < b < NF:   4 * blk(a, b) + {0: (2a, 2b), 1: (2a+1, 2b+1), 2: (2a, 2b+1), 3: (2a+1, 2b)}
+//   odd N, a < NF:    4 * NBLK + 2a + {0: (2a, N-1), 1: (2a+1, N-1)}
+//   a < NF:           2 * NPK + a: (2a, 2a+1)
+template <int N> struct K1BAcc {
+    using S = K1Pairs<N>;
+    unsigned long long pk[S::NPK > 0 ? S::NPK : 1];
+    float dg[S::NF > 0 ? S::NF : 1];
+
+    __device__ __forceinline__ void zero() {
+#pragma unroll
+        for (int i = 0; i < S::NPK; ++i) pk[i] = 0ull;
+#pragma unroll
+        for (int i = 0; i < S::NF; ++i) dg[i] = 0.0f;
+    }
+    // one coordinate of all rows
+    __device__ __forceinline__ void add(const float (&x)[N]) {
+        unsigned long long R[S::NF > 0 ? S::NF : 1];
+#pragma unroll
+        for (int a = 0; a < S::NF; ++a) R[a] = pack2(x[2 * a], x[2 * a + 1]);
+        int k = 0;
+#pragma unroll
+        for (int a = 0; a < S::NF; ++a) {
+#pragma unroll
+            for (int b = a + 1; b < S::NF; ++b) {
+                sqdiff2(pk[k], R[a], R[b]);
+                sqdiff2(pk[k + 1], R[a], pack2(x[2 * b + 1], x[2 * b]));
+                k += 2;
+            }
+        }
+        if constexpr (N % 2 == 1) {
+            const unsigned long long last = pack2(x[N - 1], x[N - 1]);
+#pragma unroll
+            for (int a = 0; a < S::NF; ++a) sqdiff2(pk[2 * S::NBLK + a], R[a], last);
+        }
+#pragma unroll
+        for (int a = 0; a < S::NF; ++a) { const float df = x[2 * a] - x[2 * a + 1]; dg[a] = fmaf(df, df, dg[a]); }
+    }
+    // the warp's fp32 accumulators -> its fp64 sums in shared memory (fixed shuffle tree), then zero
+    __device__ __forceinline__ void flush(double* warp_sums, int lane, int sbase) {
+        float flat[S::NPAD];
+#pragma unroll
+        for (int i = 0; i < S::NPK; ++i) unpack2(pk[i], flat[2 * i], flat[2 * i + 1]);
+#pragma unroll
+        for (int i = 0; i < S::NF; ++i) flat[2 * S::NPK + i] = dg[i];
+#pragma unroll
+        for (int i = S::NP; i < S::NPAD; ++i) flat[i] = 0.0f;
+        reduce_scatter<S::NPAD, 32>(flat, lane);
+#pragma unroll
+        for (int i = 0; i < S::NPAD / 32; ++i) warp_sums[sbase + i] += double(flat[i]);
+        zero();
+    }
+};
+// slot of K1BAcc -> the pair of rows (i < j)
+template <int N> __device__ __forceinline__ void k1b_slot_rows(int slot, int& i, int& j) {
+    using S = K1Pairs<N>;
+    if (slot >= 2 * S::NPK) { i = 2 * (slot - 2 * S::NPK); j = i + 1; return; }
+    if (slot >= 4 * S::NBLK) { i = slot - 4 * S::NBLK; j = N - 1; return; }
+    int blk = slot >> 2, a = 0;
+    while (blk >= S::NF - 1 - a) { blk -= S::NF - 1 - a; ++a; }
+    const int b = a + 1 + blk, which = slot & 3;
+    i = 2 * a + (which & 1);
+    j = 2 * b + ((which == 1 || which == 2) ? 1 : 0);
+}
+
+// ---- the ring kernel's scalar form of the same sums (it is bound by the latency of its copies, and
+// the packed form costs it registers it needs for three CTAs per SM: measured 2.5 times slower there)
 // acc[p] += sum_v (x[i][v] - x[j][v])^2 over the pairs p = (0,1), (0,2), .., (0,N-1), (1,2), ..
 template <int N, int V, int NPAD>
 __device__ __forceinline__ void direct_pairs(const float (&x)[N][V], float (&acc)[NPAD]) {
@@ -174,13 +273,27 @@ template <int N, int V> struct K1RDims {
 // through a ring of cp.async copies into shared-memory slots private to the
 // thread (K1R_STAGES - 1 iterations in flight, no barrier, no register staging),
 // so many bytes are in flight per SM while the registers hold the accumulators.
+// A batch (multi != nullptr): CTA b works on the tensor of descriptor multi[cta_desc[b]] as one of
+// that descriptor's `ctas` CTAs; distances to dist + index * N * N, ticket + index.
 template <int N, int V>
 __global__ void __launch_bounds__(K1R_THREADS)
 k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
-          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word) {
-    constexpr int NP = N * (N - 1) / 2;
-    constexpr int NPAD = (NP + 31) / 32 * 32;
+          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
+          const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc) {
+    constexpr int NP = K1Pairs<N>::NP, NPAD = K1Pairs<N>::NPAD;
     constexpr int WARPS = K1R_THREADS / 32;
+    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
+    if (multi != nullptr) {
+        const MultiDesc t = multi[cta_desc[blockIdx.x]];
+        g = static_cast<const float*>(t.grads);
+        d = t.d;
+        ld = t.ld;
+        dist += size_t(t.index) * N * N;
+        partials += size_t(t.cta_first) * kPairSlots;
+        ticket += t.index;
+        bx = blockIdx.x - unsigned(t.cta_first);
+        gx = unsigned(t.ctas);
+    }
     extern __shared__ __align__(16) float ring[];            // [stage][row][thread][V]
     __shared__ double sums[WARPS][NPAD];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -222,8 +335,8 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
 
     // the loop bound is per warp, so that the flush (warp-collective) is uniform
     const int64_t nvec = d / V;
-    const int64_t stride = int64_t(gridDim.x) * K1R_THREADS;
-    const int64_t wfirst = int64_t(blockIdx.x) * K1R_THREADS + warp * 32;
+    const int64_t stride = int64_t(gx) * K1R_THREADS;
+    const int64_t wfirst = int64_t(bx) * K1R_THREADS + warp * 32;
     const int64_t iters = wfirst < nvec ? (nvec - wfirst + stride - 1) / stride : 0;
 #pragma unroll
     for (int s = 0; s < K1R_STAGES - 1; ++s) {
@@ -241,29 +354,32 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     }
     cp_async_wait<0>();
     // ragged tail: the last d % V coordinates, one thread
-    if (V > 1 && blockIdx.x == 0 && tid == 0) {
+    if (V > 1 && bx == 0 && tid == 0) {
         for (int64_t t = nvec * V; t < d; ++t) direct_tail_coordinate<N, NPAD>(g, ld, t, acc);
     }
     __syncwarp();
     flush();
     __syncthreads();
 
-    double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
+    double* my_partial = partials + size_t(bx) * kPairSlots;
     for (int i = tid; i < NP; i += K1R_THREADS) {
         double s = 0.0;
 #pragma unroll
         for (int w = 0; w < WARPS; ++w) s += sums[w][i];
         my_partial[i] = s;
     }
-    if (!last_cta_ticket(ticket)) return;
-    reduce_partials(partials, NP, K1R_THREADS, [&](int p, double s) {
+    if (!last_cta_ticket(ticket, gx)) return;
+    reduce_partials(partials, NP, K1R_THREADS, gx, [&](int p, double s) {
         int i, j;
         direct_pair_rows<N>(p, i, j);
         dist[i * N + j] = s;
         dist[j * N + i] = s;
     });
     for (int i = tid; i < N; i += K1R_THREADS) dist[i * N + i] = 0.0;
-    if (tid == 0) { *ticket = 0u; *path_word = kPathDifference; }   // ready for the next call
+    if (tid == 0) {
+        *ticket = 0u;                             // ready for the next call
+        if (multi == nullptr) *path_word = kPathDifference;
+    }
 }
 
 // ================================================ direct kernel, n <= 16, rows staged by bulk copies
@@ -299,99 +415,14 @@ template <int N> struct K1BShape {
     static constexpr int TC = THREADS * V;                         // coordinates per tile
     static constexpr int ROW_BYTES = TC * 4;                       // one fp32 row of a tile
     static constexpr int STAGE_BYTES = N * ROW_BYTES;
-    static constexpr int NP = N * (N - 1) / 2;
-    static constexpr int NPAD = (NP + 31) / 32 * 32;
+    static constexpr int NP = K1Pairs<N>::NP, NPAD = K1Pairs<N>::NPAD;
     static constexpr int SUM_BYTES = WARPS * NPAD * 8;
     static constexpr int STAGES_FIT = (200 * 1024 - SUM_BYTES) / STAGE_BYTES;
     static constexpr int STAGES = STAGES_FIT > 8 ? 8 : STAGES_FIT; // depth of the ring
-    static constexpr int NF = N / 2;                               // whole row pairs
-    static constexpr int NBLK = NF * (NF - 1) / 2;                 // blocks of two row pairs
-    static constexpr int NPK = 2 * NBLK + (N % 2 ? NF : 0);        // packed accumulators
-    static_assert(2 * NPK + NF == NP, "accumulator slots");
     static_assert(STAGES >= 3, "ring depth");
 };
 constexpr int K1B_MIN_TC = 256 * K1B_V;        // coordinates per tile (dispatch threshold)
 constexpr int K1B_BAR_COMPUTE = 1;
-
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
-    unsigned long long r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void unpack2(unsigned long long p, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
-}
-// acc += (a - b)^2 in both lanes
-__device__ __forceinline__ void sqdiff2(unsigned long long& acc, unsigned long long a, unsigned long long b) {
-    unsigned long long df;
-    asm("sub.f32x2 %0, %1, %2;" : "=l"(df) : "l"(a), "l"(b));
-    asm("fma.rn.f32x2 %0, %1, %1, %0;" : "+l"(acc) : "l"(df));
-}
-
-// The accumulators of one thread.  Slot order (the order of the CTA's partial sums):
-//   for a < b < NF:   4 * blk(a, b) + {0: (2a, 2b), 1: (2a+1, 2b+1), 2: (2a, 2b+1), 3: (2a+1, 2b)}
-//   odd N, a < NF:    4 * NBLK + 2a + {0: (2a, N-1), 1: (2a+1, N-1)}
-//   a < NF:           2 * NPK + a: (2a, 2a+1)
-template <int N> struct K1BAcc {
-    using S = K1BShape<N>;
-    unsigned long long pk[S::NPK > 0 ? S::NPK : 1];
-    float dg[S::NF > 0 ? S::NF : 1];
-
-    __device__ __forceinline__ void zero() {
-#pragma unroll
-        for (int i = 0; i < S::NPK; ++i) pk[i] = 0ull;
-#pragma unroll
-        for (int i = 0; i < S::NF; ++i) dg[i] = 0.0f;
-    }
-    // one coordinate of all rows
-    __device__ __forceinline__ void add(const float (&x)[N]) {
-        unsigned long long R[S::NF > 0 ? S::NF : 1];
-#pragma unroll
-        for (int a = 0; a < S::NF; ++a) R[a] = pack2(x[2 * a], x[2 * a + 1]);
-        int k = 0;
-#pragma unroll
-        for (int a = 0; a < S::NF; ++a) {
-#pragma unroll
-            for (int b = a + 1; b < S::NF; ++b) {
-                sqdiff2(pk[k], R[a], R[b]);
-                sqdiff2(pk[k + 1], R[a], pack2(x[2 * b + 1], x[2 * b]));
-                k += 2;
-            }
-        }
-        if constexpr (N % 2 == 1) {
-            const unsigned long long last = pack2(x[N - 1], x[N - 1]);
-#pragma unroll
-            for (int a = 0; a < S::NF; ++a) sqdiff2(pk[2 * S::NBLK + a], R[a], last);
-        }
-#pragma unroll
-        for (int a = 0; a < S::NF; ++a) { const float df = x[2 * a] - x[2 * a + 1]; dg[a] = fmaf(df, df, dg[a]); }
-    }
-    // the warp's fp32 accumulators -> its fp64 sums in shared memory (fixed shuffle tree), then zero
-    __device__ __forceinline__ void flush(double* warp_sums, int lane, int sbase) {
-        float flat[S::NPAD];
-#pragma unroll
-        for (int i = 0; i < S::NPK; ++i) unpack2(pk[i], flat[2 * i], flat[2 * i + 1]);
-#pragma unroll
-        for (int i = 0; i < S::NF; ++i) flat[2 * S::NPK + i] = dg[i];
-#pragma unroll
-        for (int i = S::NP; i < S::NPAD; ++i) flat[i] = 0.0f;
-        reduce_scatter<S::NPAD, 32>(flat, lane);
-#pragma unroll
-        for (int i = 0; i < S::NPAD / 32; ++i) warp_sums[sbase + i] += double(flat[i]);
-        zero();
-    }
-};
-// slot of K1BAcc -> the pair of rows (i < j)
-template <int N> __device__ __forceinline__ void k1b_slot_rows(int slot, int& i, int& j) {
-    using S = K1BShape<N>;
-    if (slot >= 2 * S::NPK) { i = 2 * (slot - 2 * S::NPK); j = i + 1; return; }
-    if (slot >= 4 * S::NBLK) { i = slot - 4 * S::NBLK; j = N - 1; return; }
-    int blk = slot >> 2, a = 0;
-    while (blk >= S::NF - 1 - a) { blk -= S::NF - 1 - a; ++a; }
-    const int b = a + 1 + blk, which = slot & 3;
-    i = 2 * a + (which & 1);
-    j = 2 * b + ((which == 1 || which == 2) ? 1 : 0);
-}
 
 // dtype: the gradients' element type (gar_dtype_t).  16-bit elements are staged as they are (a row of
 // a tile is then half as long) and widened to fp32 when the compute threads read them.
@@ -875,8 +906,39 @@ cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, c
     cudaError_t err = persistent_grid(k1_direct<N, V>, K1R_THREADS, smem, sm_count, per_sm_cache,
                                       (nvec + K1R_THREADS - 1) / K1R_THREADS, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_path());
+    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_path(), nullptr, nullptr);
     return cudaGetLastError();
+}
+
+// A batch of tensors through the ring kernel: one CTA per entry of cta_desc.
+template <int N, int V>
+cudaError_t launch_direct_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, double* dist, double* partials,
+                                unsigned int* tickets, cudaStream_t stream) {
+    constexpr size_t smem = K1RDims<N, V>::RING_BYTES;
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (!(dev >= 0 && dev < 64 && configured[dev])) {
+        if (smem > 48 * 1024) {
+            err = cudaFuncSetAttribute(k1_direct<N, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+            if (err != cudaSuccess) return err;
+        }
+        err = cudaFuncSetAttribute(k1_direct<N, V>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (err != cudaSuccess) return err;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    k1_direct<N, V><<<unsigned(total_ctas), K1R_THREADS, smem, stream>>>(nullptr, 0, 0, dist, partials, tickets, nullptr, desc, cta_desc);
+    return cudaGetLastError();
+}
+template <int N>
+cudaError_t launch_direct_multi_n(const MultiDesc* desc, const int* cta_desc, int total_ctas, int vec, double* dist,
+                                  double* partials, unsigned int* tickets, cudaStream_t stream) {
+    if constexpr (N <= 8) {
+        if (vec >= 4) return launch_direct_multi<N, 4>(desc, cta_desc, total_ctas, dist, partials, tickets, stream);
+    }
+    if (vec >= 2) return launch_direct_multi<N, 2>(desc, cta_desc, total_ctas, dist, partials, tickets, stream);
+    return launch_direct_multi<N, 1>(desc, cta_desc, total_ctas, dist, partials, tickets, stream);
 }
 
 template <int N>
@@ -946,24 +1008,39 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
     return cudaErrorInvalidValue;
 }
 
-cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, bool vec, double* dist,
+cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int vec, double* dist,
                                    double* partials, unsigned int* tickets, cudaStream_t stream) {
+#define GAR_K1_MULTI_DIRECT(NV) \
+    case NV: return launch_direct_multi_n<NV>(desc, cta_desc, total_ctas, vec, dist, partials, tickets, stream);
 #define GAR_K1_MULTI(NBV)                                                                                              \
     case NBV:                                                                                                          \
-        return vec ? launch_tiled_multi<NBV, true>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream)      \
-                   : launch_tiled_multi<NBV, false>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream);
+        return vec == 4 ? launch_tiled_multi<NBV, true>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream) \
+                        : launch_tiled_multi<NBV, false>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream);
+    if (n <= 16) {
+        switch (n) {
+            GAR_K1_MULTI_DIRECT(2) GAR_K1_MULTI_DIRECT(3) GAR_K1_MULTI_DIRECT(4) GAR_K1_MULTI_DIRECT(5) GAR_K1_MULTI_DIRECT(6)
+            GAR_K1_MULTI_DIRECT(7) GAR_K1_MULTI_DIRECT(8) GAR_K1_MULTI_DIRECT(9) GAR_K1_MULTI_DIRECT(10) GAR_K1_MULTI_DIRECT(11)
+            GAR_K1_MULTI_DIRECT(12) GAR_K1_MULTI_DIRECT(13) GAR_K1_MULTI_DIRECT(14) GAR_K1_MULTI_DIRECT(15) GAR_K1_MULTI_DIRECT(16)
+        }
+    }
     switch ((n + 7) / 8) {
-        GAR_K1_MULTI(1) GAR_K1_MULTI(2) GAR_K1_MULTI(3) GAR_K1_MULTI(4) GAR_K1_MULTI(5) GAR_K1_MULTI(6)
-        GAR_K1_MULTI(7) GAR_K1_MULTI(8)
+        GAR_K1_MULTI(1) GAR_K1_MULTI(3) GAR_K1_MULTI(4) GAR_K1_MULTI(5) GAR_K1_MULTI(6) GAR_K1_MULTI(7) GAR_K1_MULTI(8)
     }
 #undef GAR_K1_MULTI
+#undef GAR_K1_MULTI_DIRECT
     return cudaErrorInvalidValue;
 }
 
-int distances_multi_slab(int n) {
+// Coordinates that are worth a CTA of its own in a batched distance launch (a few passes of the
+// kernel's loop), for tensors whose alignment class is `vec`.
+int distances_multi_chunk(int n, int vec) {
+    if (n <= 16) {
+        const int v = (vec >= 4 && n <= 8) ? 4 : (vec >= 2 ? 2 : 1);
+        return K1R_THREADS * v * 8;
+    }
     switch ((n + 7) / 8) {
-        case 1: return K1Dims<1>::TK; case 2: return K1Dims<2>::TK; case 3: return K1Dims<3>::TK; case 4: return K1Dims<4>::TK;
-        case 5: return K1Dims<5>::TK; case 6: return K1Dims<6>::TK; case 7: return K1Dims<7>::TK; default: return K1Dims<8>::TK;
+        case 3: return 4 * K1Dims<3>::TK; case 4: return 4 * K1Dims<4>::TK; case 5: return 4 * K1Dims<5>::TK;
+        case 6: return 4 * K1Dims<6>::TK; case 7: return 4 * K1Dims<7>::TK; default: return 4 * K1Dims<8>::TK;
     }
 }
 
