@@ -187,7 +187,7 @@ struct MultiLayout {
 MultiLayout multi_layout(int n, int count) {
     MultiLayout L{};
     size_t off = 0;
-    L.tickets = off;  off += gar::align256(size_t(count) * sizeof(unsigned int));
+    L.tickets = off;  off += gar::align256(size_t(count + 1) * sizeof(unsigned int));   // + the staged kernel's error word
     L.table = off;
     size_t t = 0;
     L.desc1 = t;  t += gar::align256(size_t(count) * sizeof(gar::MultiDesc));
@@ -389,8 +389,27 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         const gar_tensor_t& x = p->tensors[t];
         const int64_t ld = x.ld ? x.ld : x.d;
         if (!x.grads || !x.out || x.d < 1 || ld < x.d) return GAR_ERR_INVALID_ARG;
-        if (overlaps(x.grads, (size_t(n - 1) * ld + x.d) * sizeof(float), x.out, size_t(x.d) * sizeof(float)))
-            return GAR_ERR_INVALID_ARG;
+    }
+    {
+        // no output may overlap a gradient block or another output, of any tensor: sweep over the
+        // address ranges in order of their start
+        struct Range { uintptr_t begin, end; bool is_out; };
+        std::vector<Range> ranges;
+        ranges.reserve(2 * size_t(count));
+        for (int t = 0; t < count; ++t) {
+            const gar_tensor_t& x = p->tensors[t];
+            const int64_t ld = x.ld ? x.ld : x.d;
+            const uintptr_t g0 = reinterpret_cast<uintptr_t>(x.grads), o0 = reinterpret_cast<uintptr_t>(x.out);
+            ranges.push_back({g0, g0 + (size_t(n - 1) * ld + x.d) * sizeof(float), false});
+            ranges.push_back({o0, o0 + size_t(x.d) * sizeof(float), true});
+        }
+        std::sort(ranges.begin(), ranges.end(), [](const Range& a, const Range& b) { return a.begin < b.begin; });
+        uintptr_t end_any = 0, end_out = 0;
+        for (const Range& r : ranges) {
+            if (r.begin < (r.is_out ? end_any : end_out)) return GAR_ERR_INVALID_ARG;
+            if (r.end > end_any) end_any = r.end;
+            if (r.is_out && r.end > end_out) end_out = r.end;
+        }
     }
     const MultiLayout L = multi_layout(n, count);
     if (!p->workspace || reinterpret_cast<uintptr_t>(p->workspace) % 256 != 0 || p->workspace_bytes < L.total)
@@ -420,24 +439,40 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         const gar_tensor_t& x = p->tensors[t];
         m.grads = x.grads; m.out = x.out; m.d = x.d; m.ld = x.ld ? x.ld : x.d; m.index = t; m.ctas = 1; m.cta_first = 0; m.pad = 0;
     };
-    // distances: classes by the alignment of the rows, 16 / 8 / 4 bytes
+    // distances: classes by the alignment of the rows, 16 / 8 / 4 bytes; up to 16 rows, long
+    // tensors of the first class form a class of their own (the staged kernel, one CTA per SM)
     const int widths[3] = {4, 2, 1};
-    int first1[4] = {0, 0, 0, 0}, ctas1[3] = {0, 0, 0};
+    const int k1_class[4] = {gar::kMultiStaged, 4, 2, 1};
+    int first1[5] = {0, 0, 0, 0, 0}, ctas1[4] = {0, 0, 0, 0};
     {
         int pos = 0, cta_off = 0;
-        for (int cls = 0; cls < 3; ++cls) {
+        for (int cls = 0; cls < 4; ++cls) {
             first1[cls] = pos;
-            const int chunk = gar::distances_multi_chunk(n, widths[cls]);
+            const int chunk = gar::distances_multi_chunk(n, k1_class[cls]);
+            auto class_of = [&](const gar_tensor_t& x) {
+                const int64_t ld = x.ld ? x.ld : x.d;
+                const uintptr_t addr = reinterpret_cast<uintptr_t>(x.grads);
+                const int c = (addr % 16 == 0 && ld % 4 == 0) ? 1 : ((addr % 8 == 0 && ld % 2 == 0) ? 2 : 3);
+                return (c == 1 && n <= 16 && x.d >= gar::kMultiStagedMinDim) ? 0 : c;
+            };
+            // the staged kernel holds a whole SM: its CTAs, the one per tensor included, stay within one wave
+            int budget = k1_budget;
+            double class_d = total_d;
+            if (cls == 0) {
+                int members = 0;
+                class_d = 0.0;
+                for (int t = 0; t < count; ++t)
+                    if (class_of(p->tensors[t]) == 0) { ++members; class_d += double(p->tensors[t].d); }
+                budget = st->sm_count > members ? st->sm_count - members : 0;
+                if (class_d <= 0.0) class_d = 1.0;
+            }
             int cta = 0;
             for (int t = 0; t < count; ++t) {
                 const gar_tensor_t& x = p->tensors[t];
-                const int64_t ld = x.ld ? x.ld : x.d;
-                const uintptr_t addr = reinterpret_cast<uintptr_t>(x.grads);
-                const int mine = (addr % 16 == 0 && ld % 4 == 0) ? 0 : ((addr % 8 == 0 && ld % 2 == 0) ? 1 : 2);
-                if (mine != cls) continue;
+                if (class_of(x) != cls) continue;
                 gar::MultiDesc& m = desc1[pos];
                 fill(m, t);
-                m.ctas = multi_ctas(x.d, total_d, k1_budget, (x.d + chunk - 1) / chunk);
+                m.ctas = multi_ctas(x.d, class_d, budget, (x.d + chunk - 1) / chunk);
                 m.cta_first = cta;
                 for (int c = 0; c < m.ctas; ++c) cta1[cta_off + cta + c] = pos - first1[cls];
                 cta += m.ctas;
@@ -446,7 +481,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
             ctas1[cls] = cta;
             cta_off += cta;
         }
-        first1[3] = pos;
+        first1[4] = pos;
     }
     // coordinate phase: classes by vector width 4, 2, 1
     int first3[4] = {0, 0, 0, 0}, ctas3[3] = {0, 0, 0};
@@ -489,14 +524,15 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     double* dist_joint = p->dist_out ? p->dist_out : ws_dist + size_t(count) * n * n;
 
     if (needs_dist) {
-        if (int e = cuda_status(cudaMemsetAsync(ws + L.tickets, 0, size_t(count) * sizeof(unsigned int), stream))) return e;
+        if (int e = cuda_status(cudaMemsetAsync(ws + L.tickets, 0, size_t(count + 1) * sizeof(unsigned int), stream))) return e;
         double* partials = reinterpret_cast<double*>(ws + L.partials);
         unsigned int* tickets = reinterpret_cast<unsigned int*>(ws + L.tickets);
         int cta_off = 0;
-        for (int cls = 0; cls < 3; ++cls) {
+        for (int cls = 0; cls < 4; ++cls) {
             if (ctas1[cls] == 0) continue;
-            const cudaError_t err = gar::launch_distances_multi(d_desc1 + first1[cls], d_cta1 + cta_off, ctas1[cls], n, widths[cls],
-                                                                dist_each, partials + size_t(cta_off) * gar::kPairSlots, tickets, stream);
+            const cudaError_t err = gar::launch_distances_multi(d_desc1 + first1[cls], d_cta1 + cta_off, ctas1[cls], n, k1_class[cls],
+                                                                dist_each, partials + size_t(cta_off) * gar::kPairSlots, tickets,
+                                                                tickets + count, stream);
             if (err != cudaSuccess) return cuda_status(err);
             cta_off += ctas1[cls];
         }

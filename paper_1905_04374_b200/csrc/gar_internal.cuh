@@ -114,11 +114,15 @@ cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t
 // Batched launches over device arrays of descriptors: `total_ctas` CTAs, cta_desc[b] = the
 // descriptor CTA b works on.  Distances of every tensor into dist + index * n * n (difference
 // form: the ring kernel up to 16 rows, the tiled kernel beyond; `vec` = 4, 2, 1: every tensor's
-// rows are 16-byte / 8-byte / 4-byte aligned; partial sums at partials + b * kPairSlots, tickets +
+// rows are 16-byte / 8-byte / 4-byte aligned; kMultiStaged: the staged kernel; partial sums at partials + b * kPairSlots, tickets +
 // index); coordinate phase of every tensor with the selection
 // sel + index * sel_stride (register kernel, `vec` coordinates per thread).
 cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int vec, double* dist,
-                                   double* partials, unsigned int* tickets, cudaStream_t stream);
+                                   double* partials, unsigned int* tickets, unsigned int* error_word, cudaStream_t stream);
+// `vec` of the class of long tensors (n <= 16, 16-byte aligned rows) that go through the staged
+// kernel, one CTA per SM; and the length from which a tensor belongs to it
+constexpr int kMultiStaged = 8;
+constexpr int64_t kMultiStagedMinDim = 32768;
 cudaError_t launch_coordinate_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
                                     int vec, gar_selection_t* sel, int sel_stride, cudaStream_t stream);
 // Sizes that decide how many CTAs a tensor gets in the batched launches.

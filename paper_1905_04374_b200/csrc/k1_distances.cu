@@ -430,8 +430,20 @@ template <int N>
 __global__ void __launch_bounds__(K1BShape<N>::THREADS, 1)
 k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, double* __restrict__ dist,
                double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
-               unsigned int* __restrict__ path_word) {
+               unsigned int* __restrict__ path_word, const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc) {
     using S = K1BShape<N>;
+    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
+    if (multi != nullptr) {                       // a batch: CTA b works on the tensor of descriptor cta_desc[b]
+        const MultiDesc t = multi[cta_desc[blockIdx.x]];
+        g = t.grads;
+        d = t.d;
+        ld = t.ld;
+        dist += size_t(t.index) * N * N;
+        partials += size_t(t.cta_first) * kPairSlots;
+        ticket += t.index;
+        bx = blockIdx.x - unsigned(t.cta_first);
+        gx = unsigned(t.ctas);
+    }
     constexpr int NP = S::NP, NPAD = S::NPAD, V = S::V, THREADS = S::THREADS, WARPS = S::WARPS, TC = S::TC, STAGES = S::STAGES;
     const int esize = dtype == GAR_F32 ? 4 : 2;
     const unsigned row_bytes = unsigned(TC) * unsigned(esize);
@@ -451,7 +463,7 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
     volatile int* error = &error_flag;
 
     const int64_t ntiles = d / TC;
-    const int64_t first = blockIdx.x, step = gridDim.x;
+    const int64_t first = bx, step = gx;
     const int64_t mine = first < ntiles ? (ntiles - first + step - 1) / step : 0;
 
     // warp 0, lane r fetches row r of this CTA's tile number i into stage i % STAGES
@@ -517,7 +529,7 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
             kb_wait(kb_smem_u32(&full[j % STAGES]), unsigned(j / STAGES) & 1u, error, true);
     }
     // coordinates after the last whole tile: CTA 0, plain loads
-    if (blockIdx.x == 0) {
+    if (bx == 0) {
         for (int64_t t = ntiles * TC + tid; t < d; t += THREADS) {
             float x[N];
 #pragma unroll
@@ -529,7 +541,7 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
     acc.flush(sums[warp], lane, sbase);
     __syncthreads();
 
-    double* my_partial = partials + size_t(blockIdx.x) * kPairSlots;
+    double* my_partial = partials + size_t(bx) * kPairSlots;
     for (int i = tid; i < NP; i += THREADS) {
         double s = 0.0;
 #pragma unroll
@@ -537,18 +549,18 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
         my_partial[i] = s;
     }
     if (tid == 0) my_partial[kSlotError] = double(error_flag);
-    if (!last_cta_ticket(ticket)) return;
+    if (!last_cta_ticket(ticket, gx)) return;
     __shared__ int any_error;
     if (tid == 0) {
         unsigned err = 0u;
-        for (unsigned b = 0; b < gridDim.x; ++b) err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + kSlotError));
+        for (unsigned b = 0; b < gx; ++b) err |= unsigned(__ldcg(partials + size_t(b) * kPairSlots + kSlotError));
         any_error = int(err);
         if (err) *error_word = 1u;
     }
     __syncthreads();
     const bool failed = any_error != 0;
     const double nan = __longlong_as_double(0x7ff8000000000000ll);
-    reduce_partials(partials, NP, THREADS, [&](int p, double s) {
+    reduce_partials(partials, NP, THREADS, gx, [&](int p, double s) {
         int i, j;
         k1b_slot_rows<N>(p, i, j);
         if (failed) s = nan;
@@ -557,7 +569,10 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
     });
     // a NaN diagonal tells the selection kernel that the matrix is not to be used
     for (int i = tid; i < N; i += THREADS) dist[i * N + i] = failed ? nan : 0.0;
-    if (tid == 0) { *ticket = 0u; *path_word = kPathDifference; }   // ready for the next call
+    if (tid == 0) {
+        *ticket = 0u;                             // ready for the next call
+        if (multi == nullptr) *path_word = kPathDifference;
+    }
 }
 
 // ========================================================= tiled kernel, n > 16
@@ -951,7 +966,29 @@ cudaError_t launch_direct_bulk(const void* g, int dtype, int64_t d, int64_t ld, 
     cudaError_t err = persistent_grid(k1_direct_bulk<N>, S::THREADS, smem, sm_count, per_sm_cache, d / S::TC, &grid);
     if (err != cudaSuccess) return err;
     k1_direct_bulk<N><<<unsigned(grid), S::THREADS, smem, stream>>>(g, dtype, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
-                                                                     ws.k1_path());
+                                                                     ws.k1_path(), nullptr, nullptr);
+    return cudaGetLastError();
+}
+
+// A batch of long tensors with 16-byte aligned rows through the staged kernel: one CTA per entry of cta_desc.
+template <int N>
+cudaError_t launch_direct_bulk_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, double* dist, double* partials,
+                                     unsigned int* tickets, unsigned int* error_word, cudaStream_t stream) {
+    using S = K1BShape<N>;
+    const size_t smem = size_t(S::STAGES) * S::STAGE_BYTES;
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err != cudaSuccess) return err;
+    if (!(dev >= 0 && dev < 64 && configured[dev])) {
+        err = cudaFuncSetAttribute(k1_direct_bulk<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (err != cudaSuccess) return err;
+        err = cudaFuncSetAttribute(k1_direct_bulk<N>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        if (err != cudaSuccess) return err;
+        if (dev >= 0 && dev < 64) configured[dev] = true;
+    }
+    k1_direct_bulk<N><<<unsigned(total_ctas), S::THREADS, smem, stream>>>(nullptr, GAR_F32, 0, 0, dist, partials, tickets, error_word,
+                                                                           nullptr, desc, cta_desc);
     return cudaGetLastError();
 }
 
@@ -1009,9 +1046,12 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
 }
 
 cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int vec, double* dist,
-                                   double* partials, unsigned int* tickets, cudaStream_t stream) {
-#define GAR_K1_MULTI_DIRECT(NV) \
-    case NV: return launch_direct_multi_n<NV>(desc, cta_desc, total_ctas, vec, dist, partials, tickets, stream);
+                                   double* partials, unsigned int* tickets, unsigned int* error_word, cudaStream_t stream) {
+#define GAR_K1_MULTI_DIRECT(NV)                                                                                          \
+    case NV:                                                                                                             \
+        return vec == kMultiStaged                                                                                       \
+                   ? launch_direct_bulk_multi<NV>(desc, cta_desc, total_ctas, dist, partials, tickets, error_word, stream) \
+                   : launch_direct_multi_n<NV>(desc, cta_desc, total_ctas, vec, dist, partials, tickets, stream);
 #define GAR_K1_MULTI(NBV)                                                                                              \
     case NBV:                                                                                                          \
         return vec == 4 ? launch_tiled_multi<NBV, true>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream) \
@@ -1034,6 +1074,7 @@ cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, i
 // Coordinates that are worth a CTA of its own in a batched distance launch (a few passes of the
 // kernel's loop), for tensors whose alignment class is `vec`.
 int distances_multi_chunk(int n, int vec) {
+    if (n <= 16 && vec == kMultiStaged) return 4 * K1B_MIN_TC;
     if (n <= 16) {
         const int v = (vec >= 4 && n <= 8) ? 4 : (vec >= 2 ? 2 : 1);
         return K1R_THREADS * v * 8;

@@ -147,6 +147,12 @@ def test_errors_before_any_launch(pkg):
     tensors[1].ld = 0
     tensors[0].out = 4096 + 400                                            # out overlaps its own gradients
     assert L.gar_aggregate_multi(C.byref(q)) == 1
+    tensors[0].out = (1 << 20) + 8                                         # ... another tensor's gradients
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
+    tensors[0].out = (1 << 31) + 4                                         # ... another tensor's output
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
+    tensors[0].out = 1 << 30
+    assert L.gar_aggregate_multi(C.byref(q)) == 4                          # all well again: the workspace is what is missing
     assert L.gar_reduce_partials(fake, 0, 11, fake, None) == 1 and L.gar_reduce_partials(fake, 2, 65, fake, None) == 3
     assert L.gar_select(5, fake, 11, 2, 0, 0, 0, 3, fake, None) == 1       # unknown even-median mode
     assert L.gar_selftest_bounded_wait(0, fake, None) == 1
