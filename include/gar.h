@@ -308,7 +308,9 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
  *   dist_out   optional, device: joint ? n*n : count*n*n doubles (tensor t's matrix at t*n*n).
  *   selection_out  optional, device: joint ? 1 : count entries; its status field reports a
  *              selection that could not be made (the outputs are then NaN), as for gar_aggregate_ex.
- * Returns GAR_OK once everything is enqueued on `stream`.
+ * Returns GAR_OK once everything is enqueued on `stream`.  The call copies a table it builds from
+ * `tensors` out of a temporary host buffer, so it must not be recorded into a CUDA graph; calls
+ * from several host threads are fine as long as each uses its own workspace.
  */
 typedef struct gar_tensor_t {
     const float* grads;
