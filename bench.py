@@ -398,6 +398,45 @@ def measure_multi(pkg, dev, reps=20):
     return results
 
 
+def measure_small(pkg, dev, reps=200):
+    """Workloads 1 and 2 (d = 1e5, 1e6): three dependent launches, latency-bound.  Time per
+    aggregation of plain calls and of a CUDA graph of the same three launches replayed."""
+    import torch
+    out = []
+    for cfg in (1, 2):
+        wl = pkg.workloads.WORKLOADS[cfg]
+        G, _ = pkg.workloads.make_gradients(cfg, device=dev)
+        res = torch.empty(wl.d, dtype=torch.float32, device=dev)
+        ws = torch.zeros(pkg.gar_workspace_bytes("multi_bulyan", wl.n, wl.f, wl.d), dtype=torch.uint8, device=dev)
+        call = lambda: pkg.gar_aggregate_ex("multi_bulyan", G, wl.f, out=res, workspace=ws)
+        for _ in range(5):
+            call()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            call()
+
+        def timed(fn):
+            for _ in range(5):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        out.append({"workload": wl.name, "n": wl.n, "f": wl.f, "d": wl.d,
+                    "bound": "latency (three dependent launches)",
+                    "ms_per_aggregation": timed(call), "ms_per_aggregation_graph_replay": timed(graph.replay),
+                    "hbm_floor_ms": 4.0 * wl.d * (2 * wl.n + 1) / (measured_hbm_peak()[0] * 1e9) * 1e3})
+        del graph, G, res, ws
+        torch.cuda.empty_cache()
+    return out
+
+
 def workloads_seed(name):
     return 20_190_509 + sum(ord(c) for c in name)
 
@@ -526,7 +565,7 @@ def run_ours(args):
     cfg = args.config
     if args.multi_only:
         if rank == 0:
-            print(json.dumps({"multi_tensor": measure_multi(pkg, dev)}), flush=True)
+            print(json.dumps({"multi_tensor": measure_multi(pkg, dev), "small_d": measure_small(pkg, dev)}), flush=True)
         return
     if world > 1 or args.force_sharded:
         run_sharded(pkg, args, dev, world, rank, local)
@@ -569,6 +608,7 @@ def run_ours(args):
             per_config.append(entry)
 
     multi = None if args.no_multi else measure_multi(pkg, dev)
+    small = None if args.no_multi else measure_small(pkg, dev)
     cpu = None if args.no_cpu_baseline else cpu_baseline(cfg, args.cpu_sample or CPU_SAMPLE[cfg])
 
     line = {
@@ -582,7 +622,7 @@ def run_ours(args):
                    "l2": "input (%.2f GB) larger than L2; no flush" % (4e-9 * n * d) if 4 * n * d > 2.6e8
                    else "input fits L2; not flushed between steps"},
         "roofline": main["roofline"], "path": main["path"], "kernels": main["kernels"],
-        "variant_bulyan": main.get("variant_bulyan"), "per_config": per_config, "multi_tensor": multi, "cpu_baseline": cpu, "e2e": e2e,
+        "variant_bulyan": main.get("variant_bulyan"), "per_config": per_config, "small_d": small, "multi_tensor": multi, "cpu_baseline": cpu, "e2e": e2e,
         "gpu_launches": launches_per_aggregation(n, d, main["theta"]) * args.steps, "clocks": main["clocks"],
     }
     print(json.dumps(line), flush=True)

@@ -92,10 +92,6 @@ __device__ __forceinline__ void reduce_partials(const double* partials, int nslo
         combine(i, (s0 + s1) + (s2 + s3));
     }
 }
-template <typename F>
-__device__ __forceinline__ void reduce_partials(const double* partials, int nslots, int nthreads, F combine) {
-    reduce_partials(partials, nslots, nthreads, gridDim.x, combine);
-}
 
 // Returns true in exactly one of the `nctas` CTAs that share the ticket: the last one to arrive.
 // All of this CTA's partial sums must have been written before the call.
@@ -108,7 +104,6 @@ __device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket, unsigned n
     if (is_last) __threadfence();
     return is_last != 0;
 }
-__device__ __forceinline__ bool last_cta_ticket(unsigned int* ticket) { return last_cta_ticket(ticket, gridDim.x); }
 
 // ---- pieces the two direct kernels (n <= 16) share
 // The arithmetic.  Rows are taken two at a time: R_a = (x_2a, x_2a+1) sits in one 64-bit register
@@ -273,27 +268,14 @@ template <int N, int V> struct K1RDims {
 // through a ring of cp.async copies into shared-memory slots private to the
 // thread (K1R_STAGES - 1 iterations in flight, no barrier, no register staging),
 // so many bytes are in flight per SM while the registers hold the accumulators.
-// A batch (multi != nullptr): CTA b works on the tensor of descriptor multi[cta_desc[b]] as one of
-// that descriptor's `ctas` CTAs; distances to dist + index * N * N, ticket + index.
+// bx, gx: this CTA's place among the CTAs that share the problem (the ticket, the partial sums);
+// path_word may be null.
 template <int N, int V>
-__global__ void __launch_bounds__(K1R_THREADS)
-k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
-          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
-          const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc) {
+__device__ __forceinline__ void k1_direct_body(const float* __restrict__ g, const int64_t d, const int64_t ld, double* __restrict__ dist,
+                                               double* __restrict__ partials, unsigned int* __restrict__ ticket,
+                                               unsigned int* __restrict__ path_word, const unsigned bx, const unsigned gx) {
     constexpr int NP = K1Pairs<N>::NP, NPAD = K1Pairs<N>::NPAD;
     constexpr int WARPS = K1R_THREADS / 32;
-    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
-    if (multi != nullptr) {
-        const MultiDesc t = multi[cta_desc[blockIdx.x]];
-        g = static_cast<const float*>(t.grads);
-        d = t.d;
-        ld = t.ld;
-        dist += size_t(t.index) * N * N;
-        partials += size_t(t.cta_first) * kPairSlots;
-        ticket += t.index;
-        bx = blockIdx.x - unsigned(t.cta_first);
-        gx = unsigned(t.ctas);
-    }
     extern __shared__ __align__(16) float ring[];            // [stage][row][thread][V]
     __shared__ double sums[WARPS][NPAD];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -378,8 +360,25 @@ k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict
     for (int i = tid; i < N; i += K1R_THREADS) dist[i * N + i] = 0.0;
     if (tid == 0) {
         *ticket = 0u;                             // ready for the next call
-        if (multi == nullptr) *path_word = kPathDifference;
+        if (path_word != nullptr) *path_word = kPathDifference;
     }
+}
+
+template <int N, int V>
+__global__ void __launch_bounds__(K1R_THREADS)
+k1_direct(const float* __restrict__ g, int64_t d, int64_t ld, double* __restrict__ dist,
+          double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word) {
+    k1_direct_body<N, V>(g, d, ld, dist, partials, ticket, path_word, blockIdx.x, gridDim.x);
+}
+// Batch mode: CTA b works on the tensor of descriptor multi[cta_desc[b]].
+template <int N, int V>
+__global__ void __launch_bounds__(K1R_THREADS)
+k1_direct_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, double* __restrict__ dist,
+                double* __restrict__ partials, unsigned int* __restrict__ tickets) {
+    const MultiDesc t = multi[cta_desc[blockIdx.x]];
+    k1_direct_body<N, V>(static_cast<const float*>(t.grads), t.d, t.ld, dist + size_t(t.index) * N * N,
+                         partials + size_t(t.cta_first) * kPairSlots, tickets + t.index, nullptr,
+                         blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
 // ================================================ direct kernel, n <= 16, rows staged by bulk copies
@@ -426,24 +425,13 @@ constexpr int K1B_BAR_COMPUTE = 1;
 
 // dtype: the gradients' element type (gar_dtype_t).  16-bit elements are staged as they are (a row of
 // a tile is then half as long) and widened to fp32 when the compute threads read them.
+// bx, gx: this CTA's place among the CTAs that share the problem; path_word may be null.
 template <int N>
-__global__ void __launch_bounds__(K1BShape<N>::THREADS, 1)
-k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, double* __restrict__ dist,
-               double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
-               unsigned int* __restrict__ path_word, const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc) {
+__device__ __forceinline__ void k1_direct_bulk_body(const void* __restrict__ g, const int dtype, const int64_t d, const int64_t ld,
+                                                    double* __restrict__ dist, double* __restrict__ partials,
+                                                    unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
+                                                    unsigned int* __restrict__ path_word, const unsigned bx, const unsigned gx) {
     using S = K1BShape<N>;
-    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
-    if (multi != nullptr) {                       // a batch: CTA b works on the tensor of descriptor cta_desc[b]
-        const MultiDesc t = multi[cta_desc[blockIdx.x]];
-        g = t.grads;
-        d = t.d;
-        ld = t.ld;
-        dist += size_t(t.index) * N * N;
-        partials += size_t(t.cta_first) * kPairSlots;
-        ticket += t.index;
-        bx = blockIdx.x - unsigned(t.cta_first);
-        gx = unsigned(t.ctas);
-    }
     constexpr int NP = S::NP, NPAD = S::NPAD, V = S::V, THREADS = S::THREADS, WARPS = S::WARPS, TC = S::TC, STAGES = S::STAGES;
     const int esize = dtype == GAR_F32 ? 4 : 2;
     const unsigned row_bytes = unsigned(TC) * unsigned(esize);
@@ -571,8 +559,25 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
     for (int i = tid; i < N; i += THREADS) dist[i * N + i] = failed ? nan : 0.0;
     if (tid == 0) {
         *ticket = 0u;                             // ready for the next call
-        if (multi == nullptr) *path_word = kPathDifference;
+        if (path_word != nullptr) *path_word = kPathDifference;
     }
+}
+
+template <int N>
+__global__ void __launch_bounds__(K1BShape<N>::THREADS, 1)
+k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, double* __restrict__ dist,
+               double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ error_word,
+               unsigned int* __restrict__ path_word) {
+    k1_direct_bulk_body<N>(g, dtype, d, ld, dist, partials, ticket, error_word, path_word, blockIdx.x, gridDim.x);
+}
+// Batch mode (fp32): CTA b works on the tensor of descriptor multi[cta_desc[b]].
+template <int N>
+__global__ void __launch_bounds__(K1BShape<N>::THREADS, 1)
+k1_direct_bulk_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, double* __restrict__ dist,
+                     double* __restrict__ partials, unsigned int* __restrict__ tickets, unsigned int* __restrict__ error_word) {
+    const MultiDesc t = multi[cta_desc[blockIdx.x]];
+    k1_direct_bulk_body<N>(t.grads, GAR_F32, t.d, t.ld, dist + size_t(t.index) * N * N, partials + size_t(t.cta_first) * kPairSlots,
+                           tickets + t.index, error_word, nullptr, blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
 // ========================================================= tiled kernel, n > 16
@@ -658,27 +663,12 @@ template <int ES> __device__ __forceinline__ float4 tile_ld4(const float* tile, 
     }
 }
 
-template <int NB, bool VEC, int ES = 4>
-__global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
-k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
-         double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
-         const unsigned int* __restrict__ gate, int dtype, const MultiDesc* __restrict__ multi,
-         const int* __restrict__ cta_desc) {
-    // launched behind the tensor-core kernel, this one only runs if that kernel rejected its own
-    // result (the gate word is written before this grid starts: same stream)
-    if (gate != nullptr && *gate == 0u) return;
-    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
-    if (multi != nullptr) {                       // a batch: CTA b works on the tensor of descriptor cta_desc[b]
-        const MultiDesc t = multi[cta_desc[blockIdx.x]];
-        g = static_cast<const float*>(t.grads);
-        d = t.d;
-        ld = t.ld;
-        dist += size_t(t.index) * n * n;
-        partials += size_t(t.cta_first) * kPairSlots;
-        ticket += t.index;
-        bx = blockIdx.x - unsigned(t.cta_first);
-        gx = unsigned(t.ctas);
-    }
+// bx, gx: this CTA's place among the CTAs that share the problem; path_word may be null.
+template <int NB, bool VEC, int ES>
+__device__ __forceinline__ void k1_tiled_body(const float* __restrict__ g, const int n, const int64_t d, const int64_t ld,
+                                              double* __restrict__ dist, double* __restrict__ partials,
+                                              unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
+                                              const int dtype, const unsigned bx, const unsigned gx) {
     using D = K1Dims<NB>;
     constexpr int NSTAGE = D::NSTAGE;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -843,8 +833,30 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
     for (int i = tid; i < n; i += D::THREADS) dist[i * n + i] = 0.0;
     if (tid == 0) {
         *ticket = 0u;                           // ready for the next call
-        if (gate == nullptr && multi == nullptr) *path_word = kPathDifference;
+        if (path_word != nullptr) *path_word = kPathDifference;
     }
+}
+
+template <int NB, bool VEC, int ES = 4>
+__global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
+k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __restrict__ dist,
+         double* __restrict__ partials, unsigned int* __restrict__ ticket, unsigned int* __restrict__ path_word,
+         const unsigned int* __restrict__ gate, int dtype) {
+    // launched behind the tensor-core kernel, this one only runs if that kernel rejected its own
+    // result (the gate word is written before this grid starts: same stream); the path word is
+    // then that kernel's to write
+    if (gate != nullptr && *gate == 0u) return;
+    k1_tiled_body<NB, VEC, ES>(g, n, d, ld, dist, partials, ticket, gate == nullptr ? path_word : nullptr, dtype, blockIdx.x, gridDim.x);
+}
+// Batch mode (fp32): CTA b works on the tensor of descriptor multi[cta_desc[b]].
+template <int NB, bool VEC>
+__global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
+k1_tiled_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, int n, double* __restrict__ dist,
+               double* __restrict__ partials, unsigned int* __restrict__ tickets) {
+    const MultiDesc t = multi[cta_desc[blockIdx.x]];
+    k1_tiled_body<NB, VEC, 4>(static_cast<const float*>(t.grads), n, t.d, t.ld, dist + size_t(t.index) * n * n,
+                              partials + size_t(t.cta_first) * kPairSlots, tickets + t.index, nullptr, GAR_F32,
+                              blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
 // ------------------------------------------------------------------ launchers
@@ -888,7 +900,7 @@ cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* d
                                       (d + D::TK - 1) / D::TK, &grid);
     if (err != cudaSuccess) return err;
     k1_tiled<NB, VEC, ES><<<unsigned(grid), D::THREADS, D::SMEM_BYTES, stream>>>(g, n, d, ld, dist, ws.partials(), ws.ticket(),
-                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr, dtype, nullptr, nullptr);
+                                                                          ws.k1_path(), gated ? ws.k1_gate() : nullptr, dtype);
     return cudaGetLastError();
 }
 
@@ -902,12 +914,11 @@ cudaError_t launch_tiled_multi(const MultiDesc* desc, const int* cta_desc, int t
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (!(dev >= 0 && dev < 64 && configured[dev])) {
-        err = cudaFuncSetAttribute(k1_tiled<NB, VEC, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(D::SMEM_BYTES));
+        err = cudaFuncSetAttribute(k1_tiled_multi<NB, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(D::SMEM_BYTES));
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k1_tiled<NB, VEC, 4><<<unsigned(total_ctas), D::THREADS, D::SMEM_BYTES, stream>>>(
-        nullptr, n, 0, 0, dist, partials, tickets, nullptr, nullptr, GAR_F32, desc, cta_desc);
+    k1_tiled_multi<NB, VEC><<<unsigned(total_ctas), D::THREADS, D::SMEM_BYTES, stream>>>(desc, cta_desc, n, dist, partials, tickets);
     return cudaGetLastError();
 }
 
@@ -921,7 +932,7 @@ cudaError_t launch_direct(const float* g, int64_t d, int64_t ld, double* dist, c
     cudaError_t err = persistent_grid(k1_direct<N, V>, K1R_THREADS, smem, sm_count, per_sm_cache,
                                       (nvec + K1R_THREADS - 1) / K1R_THREADS, &grid);
     if (err != cudaSuccess) return err;
-    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_path(), nullptr, nullptr);
+    k1_direct<N, V><<<unsigned(grid), K1R_THREADS, smem, stream>>>(g, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_path());
     return cudaGetLastError();
 }
 
@@ -936,14 +947,14 @@ cudaError_t launch_direct_multi(const MultiDesc* desc, const int* cta_desc, int 
     if (err != cudaSuccess) return err;
     if (!(dev >= 0 && dev < 64 && configured[dev])) {
         if (smem > 48 * 1024) {
-            err = cudaFuncSetAttribute(k1_direct<N, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+            err = cudaFuncSetAttribute(k1_direct_multi<N, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
             if (err != cudaSuccess) return err;
         }
-        err = cudaFuncSetAttribute(k1_direct<N, V>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        err = cudaFuncSetAttribute(k1_direct_multi<N, V>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k1_direct<N, V><<<unsigned(total_ctas), K1R_THREADS, smem, stream>>>(nullptr, 0, 0, dist, partials, tickets, nullptr, desc, cta_desc);
+    k1_direct_multi<N, V><<<unsigned(total_ctas), K1R_THREADS, smem, stream>>>(desc, cta_desc, dist, partials, tickets);
     return cudaGetLastError();
 }
 template <int N>
@@ -966,7 +977,7 @@ cudaError_t launch_direct_bulk(const void* g, int dtype, int64_t d, int64_t ld, 
     cudaError_t err = persistent_grid(k1_direct_bulk<N>, S::THREADS, smem, sm_count, per_sm_cache, d / S::TC, &grid);
     if (err != cudaSuccess) return err;
     k1_direct_bulk<N><<<unsigned(grid), S::THREADS, smem, stream>>>(g, dtype, d, ld, dist, ws.partials(), ws.ticket(), ws.k1_error(),
-                                                                     ws.k1_path(), nullptr, nullptr);
+                                                                     ws.k1_path());
     return cudaGetLastError();
 }
 
@@ -981,14 +992,13 @@ cudaError_t launch_direct_bulk_multi(const MultiDesc* desc, const int* cta_desc,
     cudaError_t err = cudaGetDevice(&dev);
     if (err != cudaSuccess) return err;
     if (!(dev >= 0 && dev < 64 && configured[dev])) {
-        err = cudaFuncSetAttribute(k1_direct_bulk<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        err = cudaFuncSetAttribute(k1_direct_bulk_multi<N>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (err != cudaSuccess) return err;
-        err = cudaFuncSetAttribute(k1_direct_bulk<N>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+        err = cudaFuncSetAttribute(k1_direct_bulk_multi<N>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k1_direct_bulk<N><<<unsigned(total_ctas), S::THREADS, smem, stream>>>(nullptr, GAR_F32, 0, 0, dist, partials, tickets, error_word,
-                                                                           nullptr, desc, cta_desc);
+    k1_direct_bulk_multi<N><<<unsigned(total_ctas), S::THREADS, smem, stream>>>(desc, cta_desc, dist, partials, tickets, error_word);
     return cudaGetLastError();
 }
 

@@ -365,28 +365,14 @@ __device__ __forceinline__ void load_plan(K3Plan& plan, const gar_selection_t* _
 // Coordinates [t_begin, t_end), V per thread; (t_end - t_begin) % V == 0 and the
 // V-vectors at g + row*ld + t and out + t are naturally aligned.
 // Dynamic shared memory (PREAGG only): (loose_cap + GAR_MAX_SAVED) * blockDim * V floats.
-// A batch (multi != nullptr): CTA b takes its tensor (gradients, output, d, row stride) from the
-// descriptor multi[cta_desc[b]], the selection sel + index * sel_stride, and is one of the
-// descriptor's `ctas` CTAs.
+// bx, gx: this CTA's place among the CTAs that work on the problem.
 template <int P, bool EXACT, bool PREAGG, int V>
-__global__ void __launch_bounds__(K3_THREADS)
-k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin, int64_t t_end, int64_t ld,
-              gar_selection_t* __restrict__ sel, K3Out out, int loose_cap, int dtype,
-              const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, int sel_stride) {
+__device__ __forceinline__ void k3_coordinate_body(const float* __restrict__ g, const int n, const int theta_arg, const int64_t t_begin,
+                                                   const int64_t t_end, const int64_t ld, gar_selection_t* __restrict__ sel,
+                                                   const K3Out& out, const int loose_cap, const int dtype, const unsigned bx,
+                                                   const unsigned gx) {
     __shared__ K3Plan plan;
     extern __shared__ __align__(16) float k3_dyn[];
-    unsigned bx = blockIdx.x, gx = gridDim.x;     // this CTA's place among those of its problem
-    if (multi != nullptr) {
-        const MultiDesc t = multi[cta_desc[blockIdx.x]];
-        g = static_cast<const float*>(t.grads);
-        t_begin = 0;
-        t_end = t.d;
-        ld = t.ld;
-        out.out = t.out;
-        sel += size_t(t.index) * sel_stride;
-        bx = blockIdx.x - unsigned(t.cta_first);
-        gx = unsigned(t.ctas);
-    }
     const int status = k3_check(sel, n, theta_arg, PREAGG);
     if (status != GAR_OK) {                       // nothing usable: the output says so
         for (int64_t t = t_begin + int64_t(bx) * blockDim.x + threadIdx.x; t < t_end; t += int64_t(gx) * blockDim.x)
@@ -531,6 +517,25 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
         k3_finish<P, V>(e, a, theta, beta, inv_beta, lo_pads, PREAGG && med_agr, even_mean, median_only, res);
         k3_store<V>(out, t, res);
     }
+}
+
+template <int P, bool EXACT, bool PREAGG, int V>
+__global__ void __launch_bounds__(K3_THREADS)
+k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin, int64_t t_end, int64_t ld,
+              gar_selection_t* __restrict__ sel, const K3Out out, int loose_cap, int dtype) {
+    k3_coordinate_body<P, EXACT, PREAGG, V>(g, n, theta_arg, t_begin, t_end, ld, sel, out, loose_cap, dtype, blockIdx.x, gridDim.x);
+}
+// Batch mode (fp32): CTA b takes its tensor (gradients, output, d, row stride) from the descriptor
+// multi[cta_desc[b]] and the selection sel + index * sel_stride.
+template <int P, bool EXACT, bool PREAGG, int V>
+__global__ void __launch_bounds__(K3_THREADS)
+k3_coordinate_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, int n, int theta_arg,
+                    gar_selection_t* __restrict__ sel, int sel_stride, int loose_cap) {
+    const MultiDesc t = multi[cta_desc[blockIdx.x]];
+    const K3Out out{t.out, nullptr, nullptr, 0.0f, 0.0f};
+    k3_coordinate_body<P, EXACT, PREAGG, V>(static_cast<const float*>(t.grads), n, theta_arg, 0, t.d, t.ld,
+                                            sel + size_t(t.index) * sel_stride, out, loose_cap, GAR_F32,
+                                            blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
 template <int P>

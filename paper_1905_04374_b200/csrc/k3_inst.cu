@@ -109,10 +109,10 @@ static cudaError_t run(const float* g, int n, int theta, int64_t t0, int64_t d, 
         const int64_t cap = int64_t(sm_count) * 8;
         if (blocks > cap) blocks = cap;
         k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(blocks), threads, smem, stream>>>(g, n, theta, t0, d_vec, ld, sel, out,
-                                                                                         loose_cap, dtype, nullptr, nullptr, 0);
+                                                                                         loose_cap, dtype);
     }
     if (d_vec < d) {   // ragged tail (only when ld > d): scalar kernel on the last d % V coordinates
-        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap, dtype, nullptr, nullptr, 0);
+        k3_coordinate<P, EXACT, PREAGG, 1><<<1, threads1, smem1, stream>>>(g, n, theta, d_vec, d, ld, sel, out, loose_cap, dtype);
     }
     return cudaGetLastError();
 }
@@ -159,17 +159,16 @@ static cudaError_t run_multi(const MultiDesc* desc, const int* cta_desc, int tot
         cudaError_t err = cudaGetDevice(&dev);
         if (err != cudaSuccess) return err;
         if (!(dev >= 0 && dev < 64 && configured[dev])) {
-            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+            err = cudaFuncSetAttribute(k3_coordinate_multi<P, EXACT, PREAGG, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
             if (err != cudaSuccess) return err;
-            err = cudaFuncSetAttribute(k3_coordinate<P, EXACT, PREAGG, V>, cudaFuncAttributePreferredSharedMemoryCarveout,
+            err = cudaFuncSetAttribute(k3_coordinate_multi<P, EXACT, PREAGG, V>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                        cudaSharedmemCarveoutMaxShared);
             if (err != cudaSuccess) return err;
             if (dev >= 0 && dev < 64) configured[dev] = true;
         }
     }
-    const K3Out none{nullptr, nullptr, nullptr, 0.0f, 0.0f};
-    k3_coordinate<P, EXACT, PREAGG, V><<<unsigned(total_ctas), threads, smem, stream>>>(
-        nullptr, n, theta, 0, 0, 0, sel, none, loose_cap, GAR_F32, desc, cta_desc, sel_stride);
+    k3_coordinate_multi<P, EXACT, PREAGG, V><<<unsigned(total_ctas), threads, smem, stream>>>(desc, cta_desc, n, theta, sel, sel_stride,
+                                                                                              loose_cap);
     return cudaGetLastError();
 }
 

@@ -395,3 +395,32 @@ def test_sixteen_bit_strided_views(pkg):
         out = pkg.gar_aggregate_ex("multi_bulyan", view, f).cpu().numpy()
         want, tab = rule_tables("multi_bulyan", vh, f)
         assert_outputs_match(out, want, G=vh, tables=tab, max_tie_frac=1e-2)
+
+
+def test_cuda_graph_capture_and_replay(pkg):
+    """The three launches of an aggregation are plain stream work: once a first call has set the
+    kernels' attributes they can be captured into a CUDA graph and replayed (the launch-bound
+    small-d regime), on new contents of the same buffers."""
+    cfg = 1
+    wl = pkg.workloads.WORKLOADS[cfg]
+    G, _ = pkg.workloads.make_gradients(cfg, d=100_000, device=DEV)
+    out = torch.empty(G.shape[1], dtype=torch.float32, device=DEV)
+    ws = torch.zeros(pkg.gar_workspace_bytes("multi_bulyan", wl.n, wl.f, G.shape[1]), dtype=torch.uint8, device=DEV)
+    pkg.gar_aggregate_ex("multi_bulyan", G, wl.f, out=out, workspace=ws)
+    torch.cuda.synchronize()
+    first = out.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        pkg.gar_aggregate_ex("multi_bulyan", G, wl.f, out=out, workspace=ws)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, first)
+    # new gradients in the captured buffer: the replay aggregates them
+    G2, _ = pkg.workloads.make_gradients(cfg, d=100_000, device=DEV, seed=4242)
+    G.copy_(G2)
+    graph.replay()
+    torch.cuda.synchronize()
+    Gh = G2.cpu().numpy()
+    want, osel, gap = O.multi_bulyan(Gh, wl.f)
+    assert_outputs_match(out.cpu().numpy(), want, G=Gh, tables=dict(winners=osel.winners, sets=osel.sets, beta=osel.beta, gap=gap))
