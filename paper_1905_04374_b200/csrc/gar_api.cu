@@ -428,8 +428,6 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     const int k1_budget = std::min(kMultiK1Budget, (n <= 16 ? 3 : 2) * st->sm_count);
     const int k3_budget = std::min(kMultiK3Budget, 6 * st->sm_count);
     // ---- the host-built table: descriptors in launch order (wide-access tensors first) and the CTA lists
-    double total_d = 0.0;
-    for (int t = 0; t < count; ++t) total_d += double(p->tensors[t].d);
     std::vector<char> table(L.table_bytes, 0);
     gar::MultiDesc* desc1 = reinterpret_cast<gar::MultiDesc*>(table.data() + L.desc1);
     gar::MultiDesc* desc3 = reinterpret_cast<gar::MultiDesc*>(table.data() + L.desc3);
@@ -455,17 +453,15 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
                 const int c = (addr % 16 == 0 && ld % 4 == 0) ? 1 : ((addr % 8 == 0 && ld % 2 == 0) ? 2 : 3);
                 return (c == 1 && n <= 16 && x.d >= gar::kMultiStagedMinDim) ? 0 : c;
             };
-            // the staged kernel holds a whole SM: its CTAs, the one per tensor included, stay within one wave
-            int budget = k1_budget;
-            double class_d = total_d;
-            if (cls == 0) {
-                int members = 0;
-                class_d = 0.0;
-                for (int t = 0; t < count; ++t)
-                    if (class_of(p->tensors[t]) == 0) { ++members; class_d += double(p->tensors[t].d); }
-                budget = st->sm_count > members ? st->sm_count - members : 0;
-                if (class_d <= 0.0) class_d = 1.0;
-            }
+            // the class's CTAs, the one per tensor included, stay within one wave of resident CTAs
+            // (the staged kernel holds a whole SM); the rest of the wave is shared out by length
+            int members = 0;
+            double class_d = 0.0;
+            for (int t = 0; t < count; ++t)
+                if (class_of(p->tensors[t]) == cls) { ++members; class_d += double(p->tensors[t].d); }
+            if (members == 0) continue;
+            const int wave = cls == 0 ? st->sm_count : k1_budget;
+            const int budget = wave > members ? wave - members : 0;
             int cta = 0;
             for (int t = 0; t < count; ++t) {
                 const gar_tensor_t& x = p->tensors[t];
@@ -490,15 +486,23 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         for (int cls = 0; cls < 3; ++cls) {
             first3[cls] = pos;
             const int threads = gar::coordinate_multi_threads(n, theta, preagg, widths[cls]);
+            auto class_of = [&](const gar_tensor_t& x) {
+                return gar::coordinate_multi_vec(x.grads, x.out, x.d, x.ld ? x.ld : x.d, theta, preagg);
+            };
+            int members = 0;
+            double class_d = 0.0;
+            for (int t = 0; t < count; ++t)
+                if (class_of(p->tensors[t]) == widths[cls]) { ++members; class_d += double(p->tensors[t].d); }
+            if (members == 0) continue;
+            const int budget = k3_budget > members ? k3_budget - members : 0;
             int cta = 0;
             for (int t = 0; t < count; ++t) {
                 const gar_tensor_t& x = p->tensors[t];
-                const int64_t ld = x.ld ? x.ld : x.d;
-                if (gar::coordinate_multi_vec(x.grads, x.out, x.d, ld, theta, preagg) != widths[cls]) continue;
+                if (class_of(x) != widths[cls]) continue;
                 gar::MultiDesc& m = desc3[pos];
                 fill(m, t);
                 const int64_t per_cta = int64_t(threads) * widths[cls];
-                m.ctas = multi_ctas(x.d, total_d, k3_budget, (x.d + per_cta - 1) / per_cta);
+                m.ctas = multi_ctas(x.d, class_d, budget, (x.d + per_cta - 1) / per_cta);
                 m.cta_first = cta;
                 for (int c = 0; c < m.ctas; ++c) cta3[cta_off + cta + c] = pos - first3[cls];
                 cta += m.ctas;
