@@ -35,7 +35,7 @@ NOMINAL_HBM_GBS = 8000.0
 NCU_DRAM_BYTES_PER_COORD = {
     ("k1_distances", 39): 1313.0e6 / 8388608, ("k3_coordinate", 39): 1041.5e6 / 8388608,     # k1_umma (packed) / k3_bulk<19, V=2>
     ("k1_distances", 51): 1718.0e6 / 8388608, ("k3_coordinate", 51): 1680.0e6 / 8388608,     # k1_umma (wide) / k3_bulk<25, V=2>
-    ("k1_distances", 15): 1010.4e6 / 16777216, ("k3_coordinate", 15): 731.8e6 / 16777216,    # k1_direct_bulk / k3_bulk<7, V=4>
+    ("k1_distances", 15): 1010.8e6 / 16777216, ("k3_coordinate", 15): 731.8e6 / 16777216,    # k1_direct_bulk / k3_bulk<7, V=4>
 }
 
 
