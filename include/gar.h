@@ -57,7 +57,7 @@ extern "C" {
 #endif
 
 #define GAR_MAX_N 64
-#define GAR_VERSION 103
+#define GAR_VERSION 104
 
 typedef enum {
     GAR_AVERAGE      = 0, /* (1/n) sum_i G_i                       (Introduction)            */
@@ -302,7 +302,8 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
  * ones are fine, but a batch of long tensors (above about 10^7 coordinates each) is served better
  * by one gar_aggregate_ex per tensor.
  *   tensors    HOST array of `count` entries, read before the call returns; grads / out device
- *              pointers, ld = 0 means d; `out` must not overlap any tensor's gradients.
+ *              pointers, ld = 0 means d; no output (out, sgd_params, sgd_momentum_buf) may
+ *              overlap any tensor's gradients or another output.
  *   workspace  device, 256-byte aligned, >= gar_multi_workspace_bytes(rule, n, f, count); it may
  *              hold anything on entry and must not be shared by calls in flight on other streams.
  *   dist_out   optional, device: joint ? n*n : count*n*n doubles (tensor t's matrix at t*n*n).
@@ -314,9 +315,14 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
  */
 typedef struct gar_tensor_t {
     const float* grads;
-    float*       out;
+    float*       out;              /* d values; may be NULL when sgd_params is given */
     int64_t      d;
     int64_t      ld;
+    /* Optional SGD step fused into the store of this tensor's aggregate g (Eq. 2), as in
+       gar_params_t, with the step size and momentum of gar_multi_params_t:
+           v <- sgd_momentum * v + g   (only if sgd_momentum_buf is given),   x <- x - sgd_lr * v   (or g) */
+    float*       sgd_params;       /* dev [d], x, updated in place; NULL: no step */
+    float*       sgd_momentum_buf; /* dev [d], v, updated in place; NULL: plain SGD */
 } gar_tensor_t;
 
 typedef struct gar_multi_params_t {
@@ -329,6 +335,8 @@ typedef struct gar_multi_params_t {
     double*  dist_out;
     gar_selection_t* selection_out;
     void*    stream;
+    float    sgd_lr;
+    float    sgd_momentum;
 } gar_multi_params_t;
 
 size_t gar_multi_workspace_bytes(int rule, int n, int f, int count);

@@ -67,7 +67,8 @@ class GarParams(C.Structure):
 
 class GarTensor(C.Structure):
     """Mirror of gar_tensor_t."""
-    _fields_ = [("grads", C.c_void_p), ("out", C.c_void_p), ("d", C.c_int64), ("ld", C.c_int64)]
+    _fields_ = [("grads", C.c_void_p), ("out", C.c_void_p), ("d", C.c_int64), ("ld", C.c_int64),
+                ("sgd_params", C.c_void_p), ("sgd_momentum_buf", C.c_void_p)]
 
 
 class GarMultiParams(C.Structure):
@@ -77,6 +78,7 @@ class GarMultiParams(C.Structure):
         ("joint", C.c_int32), ("even_median", C.c_int32),
         ("tensors", C.POINTER(GarTensor)), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("dist_out", C.c_void_p), ("selection_out", C.c_void_p), ("stream", C.c_void_p),
+        ("sgd_lr", C.c_float), ("sgd_momentum", C.c_float),
     ]
 
 
@@ -252,30 +254,41 @@ def gar_multi_workspace_bytes(rule, n: int, f: int, count: int) -> int:
 
 
 def gar_aggregate_multi(rule, grads, f: int, outs=None, joint: bool = False, even_median=0, workspace=None,
-                        dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None, stream=None):
+                        dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None, stream=None,
+                        sgd_params=None, sgd_momentum_bufs=None, sgd_lr: float = 0.0, sgd_momentum: float = 0.0,
+                        store_out: bool = True):
     """gar_aggregate_multi: `grads` is a list of CUDA float32 tensors [n, d_t] (one per layer, the
     same n, unit column stride); returns the list of aggregates [d_t].  joint=False: every tensor
     is a problem of its own; joint=True: the tensors are the pieces of one gradient (one selection).
     Optional: workspace (uint8 CUDA tensor of gar_multi_workspace_bytes), dist_out float64
     [count, n, n] ([n, n] when joint), selection_out uint8 CUDA tensor of count (1 when joint)
-    times sizeof(gar_selection_t)."""
+    times sizeof(gar_selection_t); a fused SGD step on the lists sgd_params / sgd_momentum_bufs
+    (CUDA float32 [d_t] each, updated in place; store_out=False then passes out = NULL and
+    returns None)."""
     grads = list(grads)
     if not grads:
         raise ValueError("grads is empty")
     dev = grads[0].device
     n = grads[0].shape[0]
     count = len(grads)
-    if outs is None:
+    if outs is None and (store_out or sgd_params is None):
         outs = [torch.empty(g.shape[1], dtype=torch.float32, device=dev) for g in grads]
     tensors = (GarTensor * count)()
-    for t, (g, o) in enumerate(zip(grads, outs)):
+    for t, g in enumerate(grads):
         _dev_f32(g, "grads[%d]" % t)
         gn, d, ld = _rows(g)
         if gn != n or g.device != dev:
             raise ValueError("every tensor must have the same number of rows and sit on the same device")
-        if not (o.is_cuda and o.dtype == torch.float32 and o.is_contiguous() and o.numel() == d):
-            raise TypeError("outs[%d] must be a contiguous CUDA float32 tensor of d elements" % t)
-        tensors[t].grads, tensors[t].out, tensors[t].d, tensors[t].ld = g.data_ptr(), o.data_ptr(), d, ld
+        tensors[t].grads, tensors[t].d, tensors[t].ld = g.data_ptr(), d, ld
+        vecs = {"out": outs[t] if outs is not None else None,
+                "sgd_params": sgd_params[t] if sgd_params is not None else None,
+                "sgd_momentum_buf": sgd_momentum_bufs[t] if sgd_momentum_bufs is not None else None}
+        for name, o in vecs.items():
+            if o is None:
+                continue
+            if not (o.is_cuda and o.dtype == torch.float32 and o.is_contiguous() and o.numel() == d):
+                raise TypeError("%s[%d] must be a contiguous CUDA float32 tensor of d elements" % (name, t))
+            setattr(tensors[t], name, o.data_ptr())
     if workspace is None:
         workspace = torch.empty(gar_multi_workspace_bytes(rule, n, f, count), dtype=torch.uint8, device=dev)
     p = GarMultiParams()
@@ -288,6 +301,7 @@ def gar_aggregate_multi(rule, grads, f: int, outs=None, joint: bool = False, eve
     if selection_out is not None:
         p.selection_out = selection_out.data_ptr()
     p.stream = _stream(stream)
+    p.sgd_lr, p.sgd_momentum = sgd_lr, sgd_momentum
     with torch.cuda.device(dev):
         st = lib().gar_aggregate_multi(C.byref(p))
     _check(st, "gar_aggregate_multi")

@@ -388,20 +388,26 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     for (int t = 0; t < count; ++t) {
         const gar_tensor_t& x = p->tensors[t];
         const int64_t ld = x.ld ? x.ld : x.d;
-        if (!x.grads || !x.out || x.d < 1 || ld < x.d) return GAR_ERR_INVALID_ARG;
+        if (!x.grads || (!x.out && !x.sgd_params) || x.d < 1 || ld < x.d) return GAR_ERR_INVALID_ARG;
+        if (x.sgd_momentum_buf && !x.sgd_params) return GAR_ERR_INVALID_ARG;
     }
     {
         // no output may overlap a gradient block or another output, of any tensor: sweep over the
         // address ranges in order of their start
         struct Range { uintptr_t begin, end; bool is_out; };
         std::vector<Range> ranges;
-        ranges.reserve(2 * size_t(count));
+        ranges.reserve(4 * size_t(count));
         for (int t = 0; t < count; ++t) {
             const gar_tensor_t& x = p->tensors[t];
             const int64_t ld = x.ld ? x.ld : x.d;
-            const uintptr_t g0 = reinterpret_cast<uintptr_t>(x.grads), o0 = reinterpret_cast<uintptr_t>(x.out);
+            const uintptr_t g0 = reinterpret_cast<uintptr_t>(x.grads);
             ranges.push_back({g0, g0 + (size_t(n - 1) * ld + x.d) * sizeof(float), false});
-            ranges.push_back({o0, o0 + size_t(x.d) * sizeof(float), true});
+            const float* outs[3] = {x.out, x.sgd_params, x.sgd_momentum_buf};
+            for (const float* o : outs) {
+                if (!o) continue;
+                const uintptr_t o0 = reinterpret_cast<uintptr_t>(o);
+                ranges.push_back({o0, o0 + size_t(x.d) * sizeof(float), true});
+            }
         }
         std::sort(ranges.begin(), ranges.end(), [](const Range& a, const Range& b) { return a.begin < b.begin; });
         uintptr_t end_any = 0, end_out = 0;
@@ -435,7 +441,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     int* cta3 = reinterpret_cast<int*>(table.data() + L.cta3);
     auto fill = [&](gar::MultiDesc& m, int t) {
         const gar_tensor_t& x = p->tensors[t];
-        m.grads = x.grads; m.out = x.out; m.d = x.d; m.ld = x.ld ? x.ld : x.d; m.index = t; m.ctas = 1; m.cta_first = 0; m.pad = 0;
+        m.grads = x.grads; m.out = x.out; m.x = x.sgd_params; m.v = x.sgd_momentum_buf; m.d = x.d; m.ld = x.ld ? x.ld : x.d; m.index = t; m.ctas = 1; m.cta_first = 0; m.pad = 0;
     };
     // distances: classes by the alignment of the rows, 16 / 8 / 4 bytes; up to 16 rows, long
     // tensors of the first class form a class of their own (the staged kernel, one CTA per SM)
@@ -487,7 +493,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
             first3[cls] = pos;
             const int threads = gar::coordinate_multi_threads(n, theta, preagg, widths[cls]);
             auto class_of = [&](const gar_tensor_t& x) {
-                return gar::coordinate_multi_vec(x.grads, x.out, x.d, x.ld ? x.ld : x.d, theta, preagg);
+                return gar::coordinate_multi_vec(x.grads, x.out, x.sgd_params, x.sgd_momentum_buf, x.d, x.ld ? x.ld : x.d, theta, preagg);
             };
             int members = 0;
             double class_d = 0.0;
@@ -556,7 +562,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         for (int cls = 0; cls < 3; ++cls) {
             if (ctas3[cls] == 0) continue;
             const cudaError_t err = gar::launch_coordinate_multi(d_desc3 + first3[cls], d_cta3 + cta_off, ctas3[cls], n, theta, preagg,
-                                                                 widths[cls], sel, p->joint ? 0 : 1, stream);
+                                                                 widths[cls], sel, p->joint ? 0 : 1, p->sgd_lr, p->sgd_momentum, stream);
             if (err != cudaSuccess) return cuda_status(err);
             cta_off += ctas3[cls];
         }

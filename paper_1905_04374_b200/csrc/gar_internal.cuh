@@ -54,6 +54,8 @@ constexpr int kSlotError     = 2302;    // a bounded wait gave up
 struct MultiDesc {
     const void* grads;
     float*      out;
+    float*      x;          // fused SGD step: parameters and momentum buffer (may be null)
+    float*      v;
     int64_t     d, ld;
     int         index;
     int         ctas, cta_first;
@@ -124,12 +126,13 @@ cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, i
 constexpr int kMultiStaged = 8;
 constexpr int64_t kMultiStagedMinDim = 32768;
 cudaError_t launch_coordinate_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
-                                    int vec, gar_selection_t* sel, int sel_stride, cudaStream_t stream);
+                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, cudaStream_t stream);
 // Sizes that decide how many CTAs a tensor gets in the batched launches.
 int distances_multi_chunk(int n, int vec);
 int coordinate_multi_threads(int n, int theta, int preagg, int vec);
 // The vector width launch_coordinate_multi may be given for a tensor of these addresses and sizes.
-int coordinate_multi_vec(const void* grads, const void* out, int64_t d, int64_t ld, int theta, int preagg);
+int coordinate_multi_vec(const void* grads, const void* out, const void* x, const void* v, int64_t d, int64_t ld, int theta,
+                         int preagg);
 
 // cudaSuccess -> GAR_OK; anything else is remembered for gar_last_cuda_error and becomes GAR_ERR_CUDA
 int cuda_status(cudaError_t err);

@@ -189,3 +189,41 @@ def test_argument_errors(pkg):
     assert e.value.status == 4
     with pytest.raises(ValueError):
         pkg.gar_aggregate_multi("multi_bulyan", [g, torch.zeros(n + 1, 8, dtype=torch.float32, device=DEV)], f)
+
+
+@pytest.mark.parametrize("joint", [False, True])
+@pytest.mark.parametrize("momentum", [False, True])
+def test_fused_sgd_step_per_tensor(pkg, joint, momentum):
+    """The SGD step of Eq. 2 fused into every tensor's store: x <- x - lr (mu v + g), with g the
+    aggregate the same call returns for the tensor when asked to store it."""
+    cfg = 1
+    wl = pkg.workloads.WORKLOADS[cfg]
+    dims = [7, 1000, 4099, 65_536, 30_001]
+    _, parts, _ = layers(pkg, cfg, dims, strided=True)
+    lr, mu = 0.1, 0.9
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(9)
+    xs = [torch.randn(d, generator=gen, device=DEV, dtype=torch.float32) for d in dims]
+    vs = [torch.randn(d, generator=gen, device=DEV, dtype=torch.float32) for d in dims] if momentum else None
+    x0 = [x.cpu().numpy().astype(np.float64) for x in xs]
+    v0 = [v.cpu().numpy().astype(np.float64) for v in vs] if momentum else None
+    # the aggregates alone, then the same call with the step and no stored aggregate
+    gs = [g.clone() for g in pkg.gar_aggregate_multi("multi_bulyan", parts, wl.f, joint=joint)]
+    res = pkg.gar_aggregate_multi("multi_bulyan", parts, wl.f, joint=joint, sgd_params=xs, sgd_momentum_bufs=vs,
+                                  sgd_lr=lr, sgd_momentum=mu if momentum else 0.0, store_out=False)
+    torch.cuda.synchronize()
+    assert res is None
+    for t in range(len(dims)):
+        g = gs[t].cpu().numpy().astype(np.float64)
+        want_x, want_v = O.sgd_step(x0[t], g, lr, momentum_buf=v0[t] if momentum else None, momentum=mu)
+        got_x = xs[t].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got_x - want_x) <= 1e-6 * (1.0 + np.abs(want_x)))
+        if momentum:
+            got_v = vs[t].cpu().numpy().astype(np.float64)
+            assert np.all(np.abs(got_v - want_v) <= 1e-6 * (1.0 + np.abs(want_v)))
+    # both at once: the stored aggregates are the ones the step used
+    outs = pkg.gar_aggregate_multi("multi_bulyan", parts, wl.f, joint=joint, sgd_params=xs, sgd_momentum_bufs=vs,
+                                   sgd_lr=lr, sgd_momentum=mu if momentum else 0.0)
+    torch.cuda.synchronize()
+    for a, b in zip(outs, gs):
+        assert torch.equal(a, b)
