@@ -57,7 +57,7 @@ extern "C" {
 #endif
 
 #define GAR_MAX_N 64
-#define GAR_VERSION 104
+#define GAR_VERSION 105
 
 typedef enum {
     GAR_AVERAGE      = 0, /* (1/n) sum_i G_i                       (Introduction)            */
@@ -287,9 +287,10 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
  * Many small tensors in one launch sequence.  A model's gradient usually sits in memory as one
  * tensor per layer; aggregating those one call at a time costs three kernel launches per tensor,
  * which dominates below about 10^6 coordinates.  This call takes `count` tensors that share rule,
- * n and f -- tensor t is an n x d[t] block of fp32 gradients, row i from worker i -- and runs each
+ * n and f -- tensor t is an n x d[t] block of gradients, row i from worker i -- and runs each
  * stage once over all of them: three to seven launches whatever the count (tensors whose addresses
- * allow wide accesses and those that do not are launched separately).
+ * allow wide accesses and those that do not are launched separately).  The gradients are fp32,
+ * or bfloat16 / binary16 for all tensors alike (grads_dtype), widened exactly as they are loaded.
  *   joint = 0: every tensor is a problem of its own: own distance matrix, own selection, own
  *              coordinate phase (Algorithm 1 applied per tensor; the paper has no counterpart).
  *   joint = 1: the tensors are the pieces of ONE gradient in R^d, d = sum of d[t] (Section 2.1: the
@@ -314,7 +315,7 @@ int gar_reduce_partials(const double* parts, int count, int n, double* dist, voi
  * from several host threads are fine as long as each uses its own workspace.
  */
 typedef struct gar_tensor_t {
-    const float* grads;
+    const void*  grads;            /* fp32, or 16-bit elements by gar_multi_params_t.grads_dtype */
     float*       out;              /* d values; may be NULL when sgd_params is given */
     int64_t      d;
     int64_t      ld;
@@ -337,6 +338,7 @@ typedef struct gar_multi_params_t {
     void*    stream;
     float    sgd_lr;
     float    sgd_momentum;
+    int32_t  grads_dtype;            /* gar_dtype_t: element type of every tensor's gradients (d, ld in elements) */
 } gar_multi_params_t;
 
 size_t gar_multi_workspace_bytes(int rule, int n, int f, int count);

@@ -78,7 +78,7 @@ class GarMultiParams(C.Structure):
         ("joint", C.c_int32), ("even_median", C.c_int32),
         ("tensors", C.POINTER(GarTensor)), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("dist_out", C.c_void_p), ("selection_out", C.c_void_p), ("stream", C.c_void_p),
-        ("sgd_lr", C.c_float), ("sgd_momentum", C.c_float),
+        ("sgd_lr", C.c_float), ("sgd_momentum", C.c_float), ("grads_dtype", C.c_int32),
     ]
 
 
@@ -257,8 +257,8 @@ def gar_aggregate_multi(rule, grads, f: int, outs=None, joint: bool = False, eve
                         dist_out: torch.Tensor | None = None, selection_out: torch.Tensor | None = None, stream=None,
                         sgd_params=None, sgd_momentum_bufs=None, sgd_lr: float = 0.0, sgd_momentum: float = 0.0,
                         store_out: bool = True):
-    """gar_aggregate_multi: `grads` is a list of CUDA float32 tensors [n, d_t] (one per layer, the
-    same n, unit column stride); returns the list of aggregates [d_t].  joint=False: every tensor
+    """gar_aggregate_multi: `grads` is a list of CUDA float32 (or all bfloat16 / all float16) tensors
+    [n, d_t] (one per layer, the same n, unit column stride); returns the list of aggregates [d_t].  joint=False: every tensor
     is a problem of its own; joint=True: the tensors are the pieces of one gradient (one selection).
     Optional: workspace (uint8 CUDA tensor of gar_multi_workspace_bytes), dist_out float64
     [count, n, n] ([n, n] when joint), selection_out uint8 CUDA tensor of count (1 when joint)
@@ -274,8 +274,12 @@ def gar_aggregate_multi(rule, grads, f: int, outs=None, joint: bool = False, eve
     if outs is None and (store_out or sgd_params is None):
         outs = [torch.empty(g.shape[1], dtype=torch.float32, device=dev) for g in grads]
     tensors = (GarTensor * count)()
+    dtype = grads[0].dtype
+    if dtype not in GRAD_DTYPES:
+        raise TypeError("grads must be float32, bfloat16 or float16 tensors")
     for t, g in enumerate(grads):
-        _dev_f32(g, "grads[%d]" % t)
+        if not (g.is_cuda and g.dtype == dtype):
+            raise TypeError("grads[%d] must be a CUDA tensor of the same element type as grads[0]" % t)
         gn, d, ld = _rows(g)
         if gn != n or g.device != dev:
             raise ValueError("every tensor must have the same number of rows and sit on the same device")
@@ -302,6 +306,7 @@ def gar_aggregate_multi(rule, grads, f: int, outs=None, joint: bool = False, eve
         p.selection_out = selection_out.data_ptr()
     p.stream = _stream(stream)
     p.sgd_lr, p.sgd_momentum = sgd_lr, sgd_momentum
+    p.grads_dtype = GRAD_DTYPES[dtype]
     with torch.cuda.device(dev):
         st = lib().gar_aggregate_multi(C.byref(p))
     _check(st, "gar_aggregate_multi")

@@ -384,6 +384,9 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     if (rc != GAR_OK) return rc;
     if (p->count < 1 || !p->tensors || (p->joint != 0 && p->joint != 1) || !even_median_ok(p->even_median))
         return GAR_ERR_INVALID_ARG;
+    if (p->grads_dtype != GAR_F32 && p->grads_dtype != GAR_BF16 && p->grads_dtype != GAR_F16) return GAR_ERR_INVALID_ARG;
+    const int dtype = p->grads_dtype;
+    const size_t esize = dtype == GAR_F32 ? sizeof(float) : 2;
     const int n = p->n, count = p->count;
     for (int t = 0; t < count; ++t) {
         const gar_tensor_t& x = p->tensors[t];
@@ -401,7 +404,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
             const gar_tensor_t& x = p->tensors[t];
             const int64_t ld = x.ld ? x.ld : x.d;
             const uintptr_t g0 = reinterpret_cast<uintptr_t>(x.grads);
-            ranges.push_back({g0, g0 + (size_t(n - 1) * ld + x.d) * sizeof(float), false});
+            ranges.push_back({g0, g0 + (size_t(n - 1) * ld + x.d) * esize, false});
             const float* outs[3] = {x.out, x.sgd_params, x.sgd_momentum_buf};
             for (const float* o : outs) {
                 if (!o) continue;
@@ -431,7 +434,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
     const bool needs_dist = !(rule == GAR_AVERAGE || rule == GAR_MEDIAN);
 
     // one wave: the ring kernel keeps three CTAs per SM resident, the tiled kernel two, the register kernel six
-    const int k1_budget = std::min(kMultiK1Budget, (n <= 16 ? 3 : 2) * st->sm_count);
+    const int k1_budget = std::min(kMultiK1Budget, ((n <= 16 && p->grads_dtype == GAR_F32) ? 3 : 2) * st->sm_count);
     const int k3_budget = std::min(kMultiK3Budget, 6 * st->sm_count);
     // ---- the host-built table: descriptors in launch order (wide-access tensors first) and the CTA lists
     std::vector<char> table(L.table_bytes, 0);
@@ -452,10 +455,12 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         int pos = 0, cta_off = 0;
         for (int cls = 0; cls < 4; ++cls) {
             first1[cls] = pos;
-            const int chunk = gar::distances_multi_chunk(n, k1_class[cls]);
+            const int chunk = gar::distances_multi_chunk(n, k1_class[cls], dtype);
             auto class_of = [&](const gar_tensor_t& x) {
                 const int64_t ld = x.ld ? x.ld : x.d;
                 const uintptr_t addr = reinterpret_cast<uintptr_t>(x.grads);
+                if (dtype != GAR_F32)     // 16-bit: the staged kernel (rows 16-byte aligned), else element by element
+                    return (n <= 16 && addr % 16 == 0 && ld % 8 == 0 && x.d >= gar::kMultiStagedMinDim) ? 0 : 3;
                 const int c = (addr % 16 == 0 && ld % 4 == 0) ? 1 : ((addr % 8 == 0 && ld % 2 == 0) ? 2 : 3);
                 return (c == 1 && n <= 16 && x.d >= gar::kMultiStagedMinDim) ? 0 : c;
             };
@@ -493,7 +498,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
             first3[cls] = pos;
             const int threads = gar::coordinate_multi_threads(n, theta, preagg, widths[cls]);
             auto class_of = [&](const gar_tensor_t& x) {
-                return gar::coordinate_multi_vec(x.grads, x.out, x.sgd_params, x.sgd_momentum_buf, x.d, x.ld ? x.ld : x.d, theta, preagg);
+                return gar::coordinate_multi_vec(x.grads, x.out, x.sgd_params, x.sgd_momentum_buf, x.d, x.ld ? x.ld : x.d, theta, preagg, dtype);
             };
             int members = 0;
             double class_d = 0.0;
@@ -542,7 +547,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
             if (ctas1[cls] == 0) continue;
             const cudaError_t err = gar::launch_distances_multi(d_desc1 + first1[cls], d_cta1 + cta_off, ctas1[cls], n, k1_class[cls],
                                                                 dist_each, partials + size_t(cta_off) * gar::kPairSlots, tickets,
-                                                                tickets + count, stream);
+                                                                tickets + count, dtype, stream);
             if (err != cudaSuccess) return cuda_status(err);
             cta_off += ctas1[cls];
         }
@@ -562,7 +567,7 @@ int gar_aggregate_multi(const gar_multi_params_t* p) {
         for (int cls = 0; cls < 3; ++cls) {
             if (ctas3[cls] == 0) continue;
             const cudaError_t err = gar::launch_coordinate_multi(d_desc3 + first3[cls], d_cta3 + cta_off, ctas3[cls], n, theta, preagg,
-                                                                 widths[cls], sel, p->joint ? 0 : 1, p->sgd_lr, p->sgd_momentum, stream);
+                                                                 widths[cls], sel, p->joint ? 0 : 1, p->sgd_lr, p->sgd_momentum, dtype, stream);
             if (err != cudaSuccess) return cuda_status(err);
             cta_off += ctas3[cls];
         }

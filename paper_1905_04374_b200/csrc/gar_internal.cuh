@@ -120,19 +120,19 @@ cudaError_t launch_selftest_wait(unsigned limit, long long* result, cudaStream_t
 // index); coordinate phase of every tensor with the selection
 // sel + index * sel_stride (register kernel, `vec` coordinates per thread).
 cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int vec, double* dist,
-                                   double* partials, unsigned int* tickets, unsigned int* error_word, cudaStream_t stream);
+                                   double* partials, unsigned int* tickets, unsigned int* error_word, int dtype, cudaStream_t stream);
 // `vec` of the class of long tensors (n <= 16, 16-byte aligned rows) that go through the staged
 // kernel, one CTA per SM; and the length from which a tensor belongs to it
 constexpr int kMultiStaged = 8;
 constexpr int64_t kMultiStagedMinDim = 32768;
 cudaError_t launch_coordinate_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
-                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, cudaStream_t stream);
+                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, int dtype, cudaStream_t stream);
 // Sizes that decide how many CTAs a tensor gets in the batched launches.
-int distances_multi_chunk(int n, int vec);
+int distances_multi_chunk(int n, int vec, int dtype);
 int coordinate_multi_threads(int n, int theta, int preagg, int vec);
 // The vector width launch_coordinate_multi may be given for a tensor of these addresses and sizes.
 int coordinate_multi_vec(const void* grads, const void* out, const void* x, const void* v, int64_t d, int64_t ld, int theta,
-                         int preagg);
+                         int preagg, int dtype);
 
 // cudaSuccess -> GAR_OK; anything else is remembered for gar_last_cuda_error and becomes GAR_ERR_CUDA
 int cuda_status(cudaError_t err);

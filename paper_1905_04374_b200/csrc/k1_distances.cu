@@ -570,13 +570,14 @@ k1_direct_bulk(const void* __restrict__ g, int dtype, int64_t d, int64_t ld, dou
                unsigned int* __restrict__ path_word) {
     k1_direct_bulk_body<N>(g, dtype, d, ld, dist, partials, ticket, error_word, path_word, blockIdx.x, gridDim.x);
 }
-// Batch mode (fp32): CTA b works on the tensor of descriptor multi[cta_desc[b]].
+// Batch mode: CTA b works on the tensor of descriptor multi[cta_desc[b]].
 template <int N>
 __global__ void __launch_bounds__(K1BShape<N>::THREADS, 1)
 k1_direct_bulk_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, double* __restrict__ dist,
-                     double* __restrict__ partials, unsigned int* __restrict__ tickets, unsigned int* __restrict__ error_word) {
+                     double* __restrict__ partials, unsigned int* __restrict__ tickets, unsigned int* __restrict__ error_word,
+                     int dtype) {
     const MultiDesc t = multi[cta_desc[blockIdx.x]];
-    k1_direct_bulk_body<N>(t.grads, GAR_F32, t.d, t.ld, dist + size_t(t.index) * N * N, partials + size_t(t.cta_first) * kPairSlots,
+    k1_direct_bulk_body<N>(t.grads, dtype, t.d, t.ld, dist + size_t(t.index) * N * N, partials + size_t(t.cta_first) * kPairSlots,
                            tickets + t.index, error_word, nullptr, blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
@@ -848,14 +849,15 @@ k1_tiled(const float* __restrict__ g, int n, int64_t d, int64_t ld, double* __re
     if (gate != nullptr && *gate == 0u) return;
     k1_tiled_body<NB, VEC, ES>(g, n, d, ld, dist, partials, ticket, gate == nullptr ? path_word : nullptr, dtype, blockIdx.x, gridDim.x);
 }
-// Batch mode (fp32): CTA b works on the tensor of descriptor multi[cta_desc[b]].
+// Batch mode: CTA b works on the tensor of descriptor multi[cta_desc[b]] (16-bit gradients: the
+// element-by-element staging, VEC = false, only).
 template <int NB, bool VEC>
 __global__ void __launch_bounds__(K1Dims<NB>::THREADS, K1Dims<NB>::MIN_CTAS)
 k1_tiled_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, int n, double* __restrict__ dist,
-               double* __restrict__ partials, unsigned int* __restrict__ tickets) {
+               double* __restrict__ partials, unsigned int* __restrict__ tickets, int dtype) {
     const MultiDesc t = multi[cta_desc[blockIdx.x]];
     k1_tiled_body<NB, VEC, 4>(static_cast<const float*>(t.grads), n, t.d, t.ld, dist + size_t(t.index) * n * n,
-                              partials + size_t(t.cta_first) * kPairSlots, tickets + t.index, nullptr, GAR_F32,
+                              partials + size_t(t.cta_first) * kPairSlots, tickets + t.index, nullptr, dtype,
                               blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
@@ -907,7 +909,7 @@ cudaError_t launch_tiled(const float* g, int n, int64_t d, int64_t ld, double* d
 // A batch of tensors (fp32): one CTA per entry of cta_desc.
 template <int NB, bool VEC>
 cudaError_t launch_tiled_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, double* dist, double* partials,
-                               unsigned int* tickets, cudaStream_t stream) {
+                               unsigned int* tickets, int dtype, cudaStream_t stream) {
     using D = K1Dims<NB>;
     static bool configured[64] = {false};
     int dev = 0;
@@ -918,7 +920,7 @@ cudaError_t launch_tiled_multi(const MultiDesc* desc, const int* cta_desc, int t
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k1_tiled_multi<NB, VEC><<<unsigned(total_ctas), D::THREADS, D::SMEM_BYTES, stream>>>(desc, cta_desc, n, dist, partials, tickets);
+    k1_tiled_multi<NB, VEC><<<unsigned(total_ctas), D::THREADS, D::SMEM_BYTES, stream>>>(desc, cta_desc, n, dist, partials, tickets, dtype);
     return cudaGetLastError();
 }
 
@@ -984,7 +986,7 @@ cudaError_t launch_direct_bulk(const void* g, int dtype, int64_t d, int64_t ld, 
 // A batch of long tensors with 16-byte aligned rows through the staged kernel: one CTA per entry of cta_desc.
 template <int N>
 cudaError_t launch_direct_bulk_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, double* dist, double* partials,
-                                     unsigned int* tickets, unsigned int* error_word, cudaStream_t stream) {
+                                     unsigned int* tickets, unsigned int* error_word, int dtype, cudaStream_t stream) {
     using S = K1BShape<N>;
     const size_t smem = size_t(S::STAGES) * S::STAGE_BYTES;
     static bool configured[64] = {false};
@@ -998,7 +1000,7 @@ cudaError_t launch_direct_bulk_multi(const MultiDesc* desc, const int* cta_desc,
         if (err != cudaSuccess) return err;
         if (dev >= 0 && dev < 64) configured[dev] = true;
     }
-    k1_direct_bulk_multi<N><<<unsigned(total_ctas), S::THREADS, smem, stream>>>(desc, cta_desc, dist, partials, tickets, error_word);
+    k1_direct_bulk_multi<N><<<unsigned(total_ctas), S::THREADS, smem, stream>>>(desc, cta_desc, dist, partials, tickets, error_word, dtype);
     return cudaGetLastError();
 }
 
@@ -1056,17 +1058,20 @@ cudaError_t launch_distances(const float* grads, int n, int64_t d, int64_t ld, d
 }
 
 cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int vec, double* dist,
-                                   double* partials, unsigned int* tickets, unsigned int* error_word, cudaStream_t stream) {
-#define GAR_K1_MULTI_DIRECT(NV)                                                                                          \
-    case NV:                                                                                                             \
-        return vec == kMultiStaged                                                                                       \
-                   ? launch_direct_bulk_multi<NV>(desc, cta_desc, total_ctas, dist, partials, tickets, error_word, stream) \
+                                   double* partials, unsigned int* tickets, unsigned int* error_word, int dtype, cudaStream_t stream) {
+#define GAR_K1_MULTI_DIRECT(NV)                                                                                                  \
+    case NV:                                                                                                                     \
+        return vec == kMultiStaged                                                                                               \
+                   ? launch_direct_bulk_multi<NV>(desc, cta_desc, total_ctas, dist, partials, tickets, error_word, dtype, stream)  \
                    : launch_direct_multi_n<NV>(desc, cta_desc, total_ctas, vec, dist, partials, tickets, stream);
-#define GAR_K1_MULTI(NBV)                                                                                              \
-    case NBV:                                                                                                          \
-        return vec == 4 ? launch_tiled_multi<NBV, true>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream) \
-                        : launch_tiled_multi<NBV, false>(desc, cta_desc, total_ctas, n, dist, partials, tickets, stream);
-    if (n <= 16) {
+#define GAR_K1_MULTI(NBV)                                                                                                        \
+    case NBV:                                                                                                                    \
+        return (vec == 4 && dtype == GAR_F32)                                                                                    \
+                   ? launch_tiled_multi<NBV, true>(desc, cta_desc, total_ctas, n, dist, partials, tickets, dtype, stream)          \
+                   : launch_tiled_multi<NBV, false>(desc, cta_desc, total_ctas, n, dist, partials, tickets, dtype, stream);
+    // up to 16 rows: the staged kernel (either element size) or, fp32, the ring kernel; 16-bit
+    // gradients that the staged kernel cannot take go through the tiled kernel
+    if (n <= 16 && (dtype == GAR_F32 || vec == kMultiStaged)) {
         switch (n) {
             GAR_K1_MULTI_DIRECT(2) GAR_K1_MULTI_DIRECT(3) GAR_K1_MULTI_DIRECT(4) GAR_K1_MULTI_DIRECT(5) GAR_K1_MULTI_DIRECT(6)
             GAR_K1_MULTI_DIRECT(7) GAR_K1_MULTI_DIRECT(8) GAR_K1_MULTI_DIRECT(9) GAR_K1_MULTI_DIRECT(10) GAR_K1_MULTI_DIRECT(11)
@@ -1074,7 +1079,8 @@ cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, i
         }
     }
     switch ((n + 7) / 8) {
-        GAR_K1_MULTI(1) GAR_K1_MULTI(3) GAR_K1_MULTI(4) GAR_K1_MULTI(5) GAR_K1_MULTI(6) GAR_K1_MULTI(7) GAR_K1_MULTI(8)
+        GAR_K1_MULTI(1) GAR_K1_MULTI(2) GAR_K1_MULTI(3) GAR_K1_MULTI(4) GAR_K1_MULTI(5) GAR_K1_MULTI(6) GAR_K1_MULTI(7)
+        GAR_K1_MULTI(8)
     }
 #undef GAR_K1_MULTI
 #undef GAR_K1_MULTI_DIRECT
@@ -1083,13 +1089,14 @@ cudaError_t launch_distances_multi(const MultiDesc* desc, const int* cta_desc, i
 
 // Coordinates that are worth a CTA of its own in a batched distance launch (a few passes of the
 // kernel's loop), for tensors whose alignment class is `vec`.
-int distances_multi_chunk(int n, int vec) {
+int distances_multi_chunk(int n, int vec, int dtype) {
     if (n <= 16 && vec == kMultiStaged) return 4 * K1B_MIN_TC;
-    if (n <= 16) {
+    if (n <= 16 && dtype == GAR_F32) {
         const int v = (vec >= 4 && n <= 8) ? 4 : (vec >= 2 ? 2 : 1);
         return K1R_THREADS * v * 8;
     }
     switch ((n + 7) / 8) {
+        case 1: return 4 * K1Dims<1>::TK; case 2: return 4 * K1Dims<2>::TK;
         case 3: return 4 * K1Dims<3>::TK; case 4: return 4 * K1Dims<4>::TK; case 5: return 4 * K1Dims<5>::TK;
         case 6: return 4 * K1Dims<6>::TK; case 7: return 4 * K1Dims<7>::TK; default: return 4 * K1Dims<8>::TK;
     }

@@ -525,16 +525,16 @@ k3_coordinate(const float* __restrict__ g, int n, int theta_arg, int64_t t_begin
               gar_selection_t* __restrict__ sel, const K3Out out, int loose_cap, int dtype) {
     k3_coordinate_body<P, EXACT, PREAGG, V>(g, n, theta_arg, t_begin, t_end, ld, sel, out, loose_cap, dtype, blockIdx.x, gridDim.x);
 }
-// Batch mode (fp32): CTA b takes its tensor (gradients, output, d, row stride) from the descriptor
+// Batch mode: CTA b takes its tensor (gradients, output, d, row stride) from the descriptor
 // multi[cta_desc[b]] and the selection sel + index * sel_stride.
 template <int P, bool EXACT, bool PREAGG, int V>
 __global__ void __launch_bounds__(K3_THREADS)
 k3_coordinate_multi(const MultiDesc* __restrict__ multi, const int* __restrict__ cta_desc, int n, int theta_arg,
-                    gar_selection_t* __restrict__ sel, int sel_stride, int loose_cap, float lr, float mu) {
+                    gar_selection_t* __restrict__ sel, int sel_stride, int loose_cap, float lr, float mu, int dtype) {
     const MultiDesc t = multi[cta_desc[blockIdx.x]];
     const K3Out out{t.out, t.x, t.v, lr, mu};
     k3_coordinate_body<P, EXACT, PREAGG, V>(static_cast<const float*>(t.grads), n, theta_arg, 0, t.d, t.ld,
-                                            sel + size_t(t.index) * sel_stride, out, loose_cap, GAR_F32,
+                                            sel + size_t(t.index) * sel_stride, out, loose_cap, dtype,
                                             blockIdx.x - unsigned(t.cta_first), unsigned(t.ctas));
 }
 
@@ -544,7 +544,7 @@ cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_select
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 template <int P>
 cudaError_t launch_k3_multi_p(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg, int vec,
-                              gar_selection_t* sel, int sel_stride, float lr, float mu, cudaStream_t stream);
+                              gar_selection_t* sel, int sel_stride, float lr, float mu, int dtype, cudaStream_t stream);
 template <int P> int k3_multi_threads(int n, int preagg, int vec);
 
 }  // namespace gar

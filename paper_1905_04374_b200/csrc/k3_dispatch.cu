@@ -17,7 +17,7 @@ cudaError_t launch_k3_p(const float* g, int n, int64_t d, int64_t ld, gar_select
 template <int P> int bulk_ctas_for(int n, int theta, int preagg);
 template <int P>
 cudaError_t launch_k3_multi_p(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg, int vec,
-                              gar_selection_t* sel, int sel_stride, float lr, float mu, cudaStream_t stream);
+                              gar_selection_t* sel, int sel_stride, float lr, float mu, int dtype, cudaStream_t stream);
 template <int P> int k3_multi_threads(int n, int preagg, int vec);
 #define K3_DECL(P)                                                                                              \
     template <>                                                                                                 \
@@ -26,7 +26,7 @@ template <int P> int k3_multi_threads(int n, int preagg, int vec);
     template <> int bulk_ctas_for<P>(int, int, int);                                                            \
     template <>                                                                                                 \
     cudaError_t launch_k3_multi_p<P>(const MultiDesc*, const int*, int, int, int, int, int, gar_selection_t*, int, float, float, \
-                                     cudaStream_t); \
+                                     int, cudaStream_t); \
     template <> int k3_multi_threads<P>(int, int, int);
 K3_P_LIST(K3_DECL)
 #undef K3_DECL
@@ -73,21 +73,26 @@ cudaError_t launch_coordinate(const float* grads, int n, int64_t d, int64_t ld, 
 // and length allow (the batched kernel has no ragged-tail pass, so d must be a multiple too),
 // narrowed as launch_coordinate narrows it for large slot counts.
 int coordinate_multi_vec(const void* grads, const void* out, const void* x, const void* v, int64_t d, int64_t ld, int theta,
-                         int preagg) {
-    const uintptr_t a = reinterpret_cast<uintptr_t>(grads) | reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(x) |
-                        reinterpret_cast<uintptr_t>(v);
+                         int preagg, int dtype) {
+    const uintptr_t g = reinterpret_cast<uintptr_t>(grads);
+    const uintptr_t o = reinterpret_cast<uintptr_t>(out) | reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(v);
     int vec = 1;
-    if (a % 16 == 0 && ld % 4 == 0 && d % 4 == 0) vec = 4;
-    else if (a % 8 == 0 && ld % 2 == 0 && d % 2 == 0) vec = 2;
+    if (dtype == GAR_F32) {
+        if ((g | o) % 16 == 0 && ld % 4 == 0 && d % 4 == 0) vec = 4;
+        else if ((g | o) % 8 == 0 && ld % 2 == 0 && d % 2 == 0) vec = 2;
+    } else {                                              // V 16-bit elements per load, V floats per store
+        if (g % 8 == 0 && o % 16 == 0 && ld % 4 == 0 && d % 4 == 0) vec = 4;
+        else if (g % 4 == 0 && o % 8 == 0 && ld % 2 == 0 && d % 2 == 0) vec = 2;
+    }
     if (vec == 4 && theta > 8) vec = 2;
     if (vec == 2 && theta > (preagg ? 12 : 24)) vec = 1;
     return vec;
 }
 
 cudaError_t launch_coordinate_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
-                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, cudaStream_t stream) {
+                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, int dtype, cudaStream_t stream) {
 #define K3_TRY(P) \
-    if (theta <= P) return launch_k3_multi_p<P>(desc, cta_desc, total_ctas, n, theta, preagg, vec, sel, sel_stride, lr, mu, stream);
+    if (theta <= P) return launch_k3_multi_p<P>(desc, cta_desc, total_ctas, n, theta, preagg, vec, sel, sel_stride, lr, mu, dtype, stream);
     K3_P_LIST(K3_TRY)
 #undef K3_TRY
     return cudaErrorInvalidValue;

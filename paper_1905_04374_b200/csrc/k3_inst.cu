@@ -147,7 +147,7 @@ cudaError_t launch_k3_p<K3_P>(const float* g, int n, int64_t d, int64_t ld, gar_
 // stride and addresses allow V-wide accesses): one CTA per entry of cta_desc.
 template <int P, bool PREAGG, int V>
 static cudaError_t run_multi(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, gar_selection_t* sel,
-                             int sel_stride, float lr, float mu, cudaStream_t stream) {
+                             int sel_stride, float lr, float mu, int dtype, cudaStream_t stream) {
     constexpr bool EXACT = (K3_EXACT != 0);
     int threads = K3_THREADS;
     size_t smem = 0;
@@ -168,7 +168,7 @@ static cudaError_t run_multi(const MultiDesc* desc, const int* cta_desc, int tot
         }
     }
     k3_coordinate_multi<P, EXACT, PREAGG, V><<<unsigned(total_ctas), threads, smem, stream>>>(desc, cta_desc, n, theta, sel, sel_stride,
-                                                                                              loose_cap, lr, mu);
+                                                                                              loose_cap, lr, mu, dtype);
     return cudaGetLastError();
 }
 
@@ -177,17 +177,17 @@ static inline int multi_vec(int vec) { return (vec == 4 && K3_P > 8) ? 2 : vec; 
 
 template <>
 cudaError_t launch_k3_multi_p<K3_P>(const MultiDesc* desc, const int* cta_desc, int total_ctas, int n, int theta, int preagg,
-                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, cudaStream_t stream) {
+                                    int vec, gar_selection_t* sel, int sel_stride, float lr, float mu, int dtype, cudaStream_t stream) {
     constexpr bool kWide = (K3_P <= 8);
     vec = multi_vec(vec);
     if (preagg) {
-        if constexpr (kWide) if (vec == 4) return run_multi<K3_P, true, 4>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, stream);
-        if (vec == 2) return run_multi<K3_P, true, 2>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, stream);
-        return run_multi<K3_P, true, 1>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, stream);
+        if constexpr (kWide) if (vec == 4) return run_multi<K3_P, true, 4>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, dtype, stream);
+        if (vec == 2) return run_multi<K3_P, true, 2>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, dtype, stream);
+        return run_multi<K3_P, true, 1>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, dtype, stream);
     }
-    if constexpr (kWide) if (vec == 4) return run_multi<K3_P, false, 4>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, stream);
-    if (vec == 2) return run_multi<K3_P, false, 2>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, stream);
-    return run_multi<K3_P, false, 1>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, stream);
+    if constexpr (kWide) if (vec == 4) return run_multi<K3_P, false, 4>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, dtype, stream);
+    if (vec == 2) return run_multi<K3_P, false, 2>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, dtype, stream);
+    return run_multi<K3_P, false, 1>(desc, cta_desc, total_ctas, n, theta, sel, sel_stride, lr, mu, dtype, stream);
 }
 
 // Threads per CTA of that launch.

@@ -45,7 +45,7 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
                    'printf("%zu %zu\\n", offsetof(gar_params_t,sgd_params), offsetof(gar_params_t,sgd_lr));'
                    'printf("%zu %zu %zu %zu %zu %zu\\n", sizeof(gar_tensor_t), sizeof(gar_multi_params_t),'
                    'offsetof(gar_multi_params_t,tensors), offsetof(gar_multi_params_t,stream),'
-                   'offsetof(gar_tensor_t,sgd_momentum_buf), offsetof(gar_multi_params_t,sgd_momentum));}')
+                   'offsetof(gar_tensor_t,sgd_momentum_buf), offsetof(gar_multi_params_t,grads_dtype));}')
     exe = tmp_path / "sz"
     subprocess.check_call(["g++", "-I" + os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
     got = [int(v) for v in subprocess.check_output([str(exe)]).split()]
@@ -56,11 +56,11 @@ def test_struct_mirrors_match_the_header(pkg, tmp_path):
                    P.sgd_params.offset, P.sgd_lr.offset,
                    C.sizeof(pkg.GarTensor), C.sizeof(pkg.GarMultiParams), pkg.GarMultiParams.tensors.offset,
                    pkg.GarMultiParams.stream.offset, pkg.GarTensor.sgd_momentum_buf.offset,
-                   pkg.GarMultiParams.sgd_momentum.offset]
+                   pkg.GarMultiParams.grads_dtype.offset]
 
 
 def test_version_and_strings(pkg):
-    assert pkg.gar_version() == 104
+    assert pkg.gar_version() == 105
     assert pkg.gar_status_string(0) == "ok"
     assert pkg.gar_last_cuda_error() == (0, "cudaSuccess")      # nothing has failed in this thread yet
     assert "4f+3" in pkg.gar_status_string(2)
@@ -161,6 +161,8 @@ def test_errors_before_any_launch(pkg):
     assert L.gar_aggregate_multi(C.byref(q)) == 1
     tensors[1].sgd_params, tensors[1].out = 1 << 34, None                  # a fused step without the aggregate: fine
     assert L.gar_aggregate_multi(C.byref(q)) == 4
+    q.grads_dtype = 3                                                      # unknown element type
+    assert L.gar_aggregate_multi(C.byref(q)) == 1
     assert L.gar_reduce_partials(fake, 0, 11, fake, None) == 1 and L.gar_reduce_partials(fake, 2, 65, fake, None) == 3
     assert L.gar_select(5, fake, 11, 2, 0, 0, 0, 3, fake, None) == 1       # unknown even-median mode
     assert L.gar_selftest_bounded_wait(0, fake, None) == 1

@@ -227,3 +227,52 @@ def test_fused_sgd_step_per_tensor(pkg, joint, momentum):
     torch.cuda.synchronize()
     for a, b in zip(outs, gs):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16])
+@pytest.mark.parametrize("cfg", [1, 2])
+@pytest.mark.parametrize("joint", [False, True])
+def test_sixteen_bit_gradients(pkg, dtype, cfg, joint):
+    """bfloat16 / binary16 tensors: every value is widened to fp32 exactly when a kernel loads it,
+    so the oracle fed the same 16-bit values is the reference (exact ties between 16-bit values
+    are frequent: up to 1 % of the coordinates may rest on the tie-aware check)."""
+    wl = pkg.workloads.WORKLOADS[cfg]
+    n, f = wl.n, wl.f
+    dims = [3, 1000, 4099, 65_536, 30_001, 262_144]
+    G32, parts32, _ = layers(pkg, cfg, dims, strided=True)
+    parts = []
+    for k, g in enumerate(parts32):
+        if g.is_contiguous():
+            parts.append(g.to(dtype))
+        else:                                         # keep a strided, misaligned view
+            wide = torch.zeros(n, g.shape[1] + 5, dtype=dtype, device=DEV)
+            wide[:, 3:3 + g.shape[1]] = g.to(dtype)
+            parts.append(wide[:, 3:3 + g.shape[1]])
+    count = len(parts)
+    nsel = 1 if joint else count
+    sels = torch.zeros(nsel * C.sizeof(pkg.GarSelection), dtype=torch.uint8, device=DEV)
+    dist = torch.empty(nsel, n, n, dtype=torch.float64, device=DEV)
+    outs = pkg.gar_aggregate_multi("multi_bulyan", parts, f, joint=joint, dist_out=dist, selection_out=sels)
+    torch.cuda.synchronize()
+    sel_host = read_selections(pkg, sels, nsel)
+    problems = [(torch.cat([p.to(torch.float32) for p in parts], dim=1), torch.cat(outs), 0)] if joint else \
+        [(p.to(torch.float32), o, t) for t, (p, o) in enumerate(zip(parts, outs))]
+    for gh, o, t in problems:
+        Gh = gh.cpu().numpy()
+        got = o.cpu().numpy()
+        want, tab = rule_tables("multi_bulyan", Gh, f)
+        D = dist[t].cpu().numpy()
+        wantD = O.pairwise_sq_distances(Gh)
+        pos = wantD > 0
+        assert np.max(np.abs(D - wantD)[pos] / wantD[pos]) <= 1e-6 and np.all(D[~pos] == 0)
+        sel = sel_host[t]
+        assert sel.status == 0
+        compared = assert_selection_match(sel, tab["rounds"], True)
+        if compared == len(tab["rounds"]):
+            assert_outputs_match(got, want, G=Gh, tables=tab, max_tie_frac=1e-2)
+        else:
+            winners = [sel.winners[r] for r in range(sel.theta)]
+            sets = [[i for i in range(n) if (sel.sets[r] >> i) & 1] for r in range(sel.theta)]
+            want2, gap2 = O.coordinate_phase(Gh, winners, sets, sel.beta)
+            assert_outputs_match(got, want2, G=Gh, tables=dict(winners=winners, sets=sets, beta=sel.beta, gap=gap2),
+                                 max_tie_frac=1e-2)
